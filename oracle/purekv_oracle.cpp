@@ -1,0 +1,249 @@
+// CPU oracle for the PureKV hot path.  TEST INFRASTRUCTURE ONLY: slow, plain,
+// fp64, written from the paper's definitions.  It shares no code with the CUDA
+// library and must never be called from the product path; only the tests, the
+// smoke check and the benchmark's CPU-baseline leg use it.
+//
+// What each function follows:
+//   pko_mask           ST-SpAttn mask, Sec. 3.2 (spatial path: first frame + current
+//                      frame; temporal path: corresponding token of the previous frame
+//                      + first frame), under causal attention (Sec. 3.1/3.2).
+//   pko_prefill        masked softmax attention; the softmax is Eq. 1 restricted to the
+//                      kept keys of each row.
+//   pko_lowlayer_score Eq. 1 (dense causal softmax rows) and Eq. 2 (sum of the recent
+//                      window's rows over the non-recent keys).
+//   pko_vnorm_scores   Eq. 3 / Eq. 4 (C weighted by the L2 norm of each key's V vector).
+//   pko_select         Sec. 3.1: keep the recent window w plus the top-h non-recent keys.
+//   pko_compact        the compacted cache implied by that selection.
+//   pko_budget         integer budget from a keep ratio.
+// Readings taken where the paper is silent (token order inside a frame, prefix
+// tokens always visible, text rows dense, mean over the query heads of a GQA
+// group, tie-break by position) are listed in the repository's design notes.
+//
+// Parity pins: every function here is pinned by the CPU tests against brute
+// force, closed forms, invariants or library special cases.  Nothing numeric is
+// printed by the paper for these operations, so agreement with the authors' own
+// (unpublished) implementation is "parity unpinned".
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <limits>
+#include <numeric>
+#include <vector>
+
+extern "C" {
+
+struct pko_mask_params {
+  int32_t grid_h, grid_w;
+  int32_t anchor_frames;    // first frames every visual query sees (paper: 1)
+  int32_t spatial_radius;   // -1: whole current frame (paper); else Chebyshev radius
+  int32_t temporal_depth;   // number of linked earlier frames (paper: 1), -1: all
+  int32_t temporal_stride;  // linked frames are f-s, f-2s, ... (paper: 1)
+  int32_t temporal_radius;  // 0: same grid cell only (paper); -1: whole linked frame
+  int32_t dense_causal;     // nonzero: plain causal attention
+};
+
+// Sec. 3.2.  Positions are relative to the request; len = n_prefix + n_frames*N + n_suffix.
+// Returns 1 when query i may attend key j.
+int32_t pko_mask(const pko_mask_params* p, int32_t len, int32_t n_prefix, int32_t n_frames,
+                 int32_t i, int32_t j) {
+  if (i < 0 || j < 0 || i >= len || j >= len) return 0;
+  if (j > i) return 0;                           // causal attention
+  if (p->dense_causal) return 1;
+  const int32_t n = p->grid_h * p->grid_w;
+  const int32_t vis_end = n_prefix + n_frames * n;
+  const bool i_visual = i >= n_prefix && i < vis_end;
+  if (!i_visual) return 1;                       // text queries: dense causal
+  if (j < n_prefix) return 1;                    // prefix keys: always visible
+  // both visual (j <= i < vis_end and j >= n_prefix)
+  const int32_t fi = (i - n_prefix) / n, pi = (i - n_prefix) % n;
+  const int32_t fj = (j - n_prefix) / n, pj = (j - n_prefix) % n;
+  const int32_t yi = pi / p->grid_w, xi = pi % p->grid_w;
+  const int32_t yj = pj / p->grid_w, xj = pj % p->grid_w;
+  const int32_t rho = std::max(std::abs(yi - yj), std::abs(xi - xj));
+  const int32_t df = fi - fj;
+  // (1) attention to the first frame(s): both paths keep it
+  if (fj < p->anchor_frames) return 1;
+  // (2) spatial path: the current frame
+  if (df == 0 && (p->spatial_radius < 0 || rho <= p->spatial_radius)) return 1;
+  // (3) temporal path: the corresponding token of the previous frame(s)
+  if (df >= 1 && p->temporal_stride >= 1 && df % p->temporal_stride == 0 &&
+      (p->temporal_depth < 0 || df <= (int64_t)p->temporal_depth * p->temporal_stride) &&
+      (p->temporal_radius < 0 || rho <= p->temporal_radius))
+    return 1;
+  return 0;
+}
+
+void pko_mask_matrix(const pko_mask_params* p, int32_t len, int32_t n_prefix, int32_t n_frames,
+                     uint8_t* out /* [len*len] */) {
+  for (int32_t i = 0; i < len; ++i)
+    for (int32_t j = 0; j < len; ++j)
+      out[(int64_t)i * len + j] = (uint8_t)pko_mask(p, len, n_prefix, n_frames, i, j);
+}
+
+static inline double dot_fd(const float* a, const float* b, int32_t d) {
+  double s = 0.0;
+  for (int32_t c = 0; c < d; ++c) s += (double)a[c] * (double)b[c];
+  return s;
+}
+
+// Masked softmax attention for a list of rows and heads.
+// q [T,H,d], k,v [T,H_kv,d] float32 (bf16 inputs are passed widened, which is exact).
+// rows: absolute token indices (NULL = all T rows); heads: query heads (NULL = all).
+// out [n_rows, n_heads, d] float64, lse [n_heads, n_rows] float64 (natural log).
+// scale <= 0 means 1/sqrt(d) (Eq. 1).
+void pko_prefill(const float* q, const float* k, const float* v,
+                 int32_t n_req, const int32_t* cu_seqlens, const int32_t* n_prefix,
+                 const int32_t* n_frames, const pko_mask_params* mp,
+                 int32_t n_q_heads, int32_t n_kv_heads, int32_t d, double scale,
+                 const int64_t* rows, int64_t n_rows, const int32_t* heads, int32_t n_heads,
+                 double* out, double* lse) {
+  const int64_t T = cu_seqlens[n_req];
+  if (!rows) n_rows = T;
+  if (!heads) n_heads = n_q_heads;
+  if (scale <= 0.0) scale = 1.0 / std::sqrt((double)d);
+  const int32_t G = n_q_heads / n_kv_heads;
+#pragma omp parallel for schedule(dynamic, 4)
+  for (int64_t ri = 0; ri < n_rows; ++ri) {
+    const int64_t t = rows ? rows[ri] : ri;
+    int32_t r = 0;
+    while (r + 1 < n_req && t >= cu_seqlens[r + 1]) ++r;
+    const int64_t base = cu_seqlens[r];
+    const int32_t len = cu_seqlens[r + 1] - cu_seqlens[r];
+    const int32_t i = (int32_t)(t - base);
+    std::vector<double> s(i + 1);
+    std::vector<uint8_t> keep(i + 1);
+    for (int32_t j = 0; j <= i; ++j) keep[j] = (uint8_t)pko_mask(mp, len, n_prefix[r], n_frames[r], i, j);
+    for (int32_t hi = 0; hi < n_heads; ++hi) {
+      const int32_t hq = heads ? heads[hi] : hi;
+      const int32_t g = hq / G;
+      const float* qi = q + ((int64_t)t * n_q_heads + hq) * d;
+      double m = -std::numeric_limits<double>::infinity();
+      for (int32_t j = 0; j <= i; ++j) {
+        if (!keep[j]) continue;
+        s[j] = scale * dot_fd(qi, k + ((base + j) * n_kv_heads + g) * d, d);
+        m = std::max(m, s[j]);
+      }
+      double z = 0.0;
+      double* o = out + ((int64_t)ri * n_heads + hi) * d;
+      for (int32_t c = 0; c < d; ++c) o[c] = 0.0;
+      for (int32_t j = 0; j <= i; ++j) {
+        if (!keep[j]) continue;
+        const double e = std::exp(s[j] - m);
+        z += e;
+        const float* vj = v + ((base + j) * n_kv_heads + g) * d;
+        for (int32_t c = 0; c < d; ++c) o[c] += e * (double)vj[c];
+      }
+      for (int32_t c = 0; c < d; ++c) o[c] /= z;
+      if (lse) lse[(int64_t)hi * n_rows + ri] = m + std::log(z);
+    }
+  }
+}
+
+// Eq. 1 + Eq. 2.  For every request and KV head g:
+//   C[g, j] = (1/G) sum_{hq in group g} sum_{i=l-w}^{l-1} A^{hq}_{i,j},  0 <= j < l-w,
+// with A the dense causal softmax (row i normalised over all j' <= i).  The mean
+// over the group's query heads is this build's reading (the paper is silent on GQA).
+// c_out [H_kv, T] float64; entries of each request's last w positions are set to 0.
+// The window is clipped to the request length.
+void pko_lowlayer_score(const float* q, const float* k,
+                        int32_t n_req, const int32_t* cu_seqlens, int32_t window,
+                        int32_t n_q_heads, int32_t n_kv_heads, int32_t d, double scale,
+                        double* c_out) {
+  const int64_t T = cu_seqlens[n_req];
+  if (scale <= 0.0) scale = 1.0 / std::sqrt((double)d);
+  const int32_t G = n_q_heads / n_kv_heads;
+  for (int64_t x = 0; x < (int64_t)n_kv_heads * T; ++x) c_out[x] = 0.0;
+  for (int32_t r = 0; r < n_req; ++r) {
+    const int64_t base = cu_seqlens[r];
+    const int32_t len = cu_seqlens[r + 1] - cu_seqlens[r];
+    const int32_t w = std::min(window, len);
+    const int32_t nr = len - w;                       // non-recent keys: 0 .. nr-1
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t g = 0; g < n_kv_heads; ++g) {
+      std::vector<double> s(len), acc(std::max(nr, 1), 0.0);
+      for (int32_t hq = g * G; hq < (g + 1) * G; ++hq) {
+        for (int32_t i = len - w; i < len; ++i) {
+          const float* qi = q + ((base + i) * n_q_heads + hq) * d;
+          double m = -std::numeric_limits<double>::infinity();
+          for (int32_t j = 0; j <= i; ++j) {
+            s[j] = scale * dot_fd(qi, k + ((base + j) * n_kv_heads + g) * d, d);
+            m = std::max(m, s[j]);
+          }
+          double z = 0.0;
+          for (int32_t j = 0; j <= i; ++j) { s[j] = std::exp(s[j] - m); z += s[j]; }
+          for (int32_t j = 0; j < nr; ++j) acc[j] += s[j] / z;
+        }
+      }
+      for (int32_t j = 0; j < nr; ++j) c_out[(int64_t)g * T + base + j] = acc[j] / (double)G;
+    }
+  }
+}
+
+// Eq. 3 / Eq. 4 for one layer: S[g, t] = C[g, t] * ||V[t, g, :]||_2.
+void pko_vnorm_scores(const double* c /* [H_kv,T] */, const float* v /* [T,H_kv,d] */,
+                      int64_t T, int32_t n_kv_heads, int32_t d, double* s_out /* [H_kv,T] */) {
+#pragma omp parallel for
+  for (int64_t t = 0; t < T; ++t)
+    for (int32_t g = 0; g < n_kv_heads; ++g) {
+      const float* vv = v + (t * n_kv_heads + g) * d;
+      s_out[(int64_t)g * T + t] = c[(int64_t)g * T + t] * std::sqrt(dot_fd(vv, vv, d));
+    }
+}
+
+// Sec. 3.1 selection for one layer.  For request r and KV head g: the h_keep[r]
+// non-recent positions with the largest score (ties: lower position first), written
+// in ascending position order, followed by the recent window l-w .. l-1.
+// s [H_kv, T]; idx_out [H_kv, K_tot], K_tot = cu_kept[n_req]; positions request-relative.
+// kth_out (nullable) [H_kv, n_req]: the h-th largest score (NaN when h == 0).
+void pko_select(const double* s, int32_t n_req, const int32_t* cu_seqlens, int32_t window,
+                const int32_t* h_keep, const int32_t* cu_kept, int32_t n_kv_heads,
+                int32_t* idx_out, double* kth_out) {
+  const int64_t T = cu_seqlens[n_req];
+  const int64_t K_tot = cu_kept[n_req];
+  for (int32_t g = 0; g < n_kv_heads; ++g)
+    for (int32_t r = 0; r < n_req; ++r) {
+      const int64_t base = cu_seqlens[r];
+      const int32_t len = cu_seqlens[r + 1] - cu_seqlens[r];
+      const int32_t w = std::min(window, len);
+      const int32_t nr = len - w;
+      const int32_t h = h_keep[r];
+      const double* sg = s + (int64_t)g * T + base;
+      std::vector<int32_t> order(nr);
+      std::iota(order.begin(), order.end(), 0);
+      std::stable_sort(order.begin(), order.end(),
+                       [&](int32_t a, int32_t b) { return sg[a] > sg[b]; });   // stable: ties keep position order
+      std::vector<int32_t> chosen(order.begin(), order.begin() + h);
+      std::sort(chosen.begin(), chosen.end());
+      int32_t* o = idx_out + (int64_t)g * K_tot + cu_kept[r];
+      for (int32_t t = 0; t < h; ++t) o[t] = chosen[t];
+      for (int32_t t = 0; t < w; ++t) o[h + t] = nr + t;
+      if (kth_out) kth_out[(int64_t)g * n_req + r] = h > 0 ? sg[order[h - 1]] : std::nan("");
+    }
+}
+
+// Compacted cache of one layer: out[cu_kept[r]+t, g, :] = src[cu_seqlens[r] + idx[g, cu_kept[r]+t], g, :].
+// Rows are row_bytes = d * element size bytes; a pure byte copy.
+void pko_compact(const uint8_t* src /* [T,H_kv,row_bytes] */, const int32_t* idx /* [H_kv,K_tot] */,
+                 int32_t n_req, const int32_t* cu_seqlens, const int32_t* cu_kept,
+                 int32_t n_kv_heads, int64_t row_bytes, uint8_t* out /* [K_tot,H_kv,row_bytes] */) {
+  const int64_t K_tot = cu_kept[n_req];
+  for (int32_t r = 0; r < n_req; ++r)
+    for (int32_t t = cu_kept[r]; t < cu_kept[r + 1]; ++t)
+      for (int32_t g = 0; g < n_kv_heads; ++g) {
+        const int64_t srow = (int64_t)cu_seqlens[r] + idx[(int64_t)g * K_tot + t];
+        std::memcpy(out + ((int64_t)t * n_kv_heads + g) * row_bytes,
+                    src + (srow * n_kv_heads + g) * row_bytes, (size_t)row_bytes);
+      }
+}
+
+// Budget: w <- min(w, l); k = max(w, floor(keep*l)) capped at l; h = k - w.
+void pko_budget(int32_t len, int32_t window, double keep_ratio, int32_t* h_out, int32_t* k_out) {
+  const int32_t w = std::min(window, len);
+  int32_t k = (int32_t)std::floor(keep_ratio * (double)len);
+  k = std::min(len, std::max(w, k));
+  *h_out = k - w;
+  *k_out = k;
+}
+
+}  // extern "C"
