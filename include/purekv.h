@@ -1,0 +1,175 @@
+/* purekv.h -- C ABI of the PureKV hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, as hand-written CUDA kernels, the data-parallel part of
+ * PureKV: Spatial-Temporal Sparse Attention (ST-SpAttn) prefill (Sec. 3.2) and the
+ * KV-cache compression it feeds (Sec. 3.1): window attention scores of a low layer
+ * (Eq. 1-2), V-norm weighting (Eq. 3-4), selection of the recent window plus the
+ * top-h non-recent keys, and the gather of the surviving K/V rows.
+ *
+ * Conventions
+ *  - Every function returns a purekv_status; nothing throws across the ABI.
+ *  - The caller owns every buffer.  Pointers are DEVICE pointers unless the name
+ *    starts with h_ (host).  Nothing is allocated or freed by the library, and no
+ *    call synchronises the device unless its comment says so.
+ *  - `stream` is a cudaStream_t passed as void*; all device work is enqueued on it.
+ *  - Packed variable-length layout ("THD"): Q and O are [T, H, d], K and V are
+ *    [T, H_kv, d], row-major, contiguous; T = total tokens over all requests and
+ *    request r owns tokens cu_seqlens[r] .. cu_seqlens[r+1]-1.  Query head hq uses KV
+ *    head hq / (H / H_kv).
+ *  - A request's tokens are ordered [n_prefix text][n_frames x (grid_h x grid_w) visual,
+ *    raster order inside a frame][suffix text].
+ *  - dtype is the element type of Q/K/V/O; accumulation, softmax and scores are fp32.
+ */
+#ifndef PUREKV_H_
+#define PUREKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PUREKV_OK = 0,
+  PUREKV_ERR_INVALID_ARG = 1, /* null pointer, negative size, inconsistent descriptors   */
+  PUREKV_ERR_UNSUPPORTED = 2, /* head_dim / dtype / tile combination without a kernel    */
+  PUREKV_ERR_WORKSPACE = 3,   /* plan or workspace buffer too small                      */
+  PUREKV_ERR_CUDA = 4,        /* a CUDA call failed; text in purekv_last_error           */
+  PUREKV_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (purekv_poll_status) */
+} purekv_status;
+
+typedef enum { PUREKV_BF16 = 0, PUREKV_FP32 = 1 } purekv_dtype;
+
+#define PUREKV_FLAG_DENSE_CAUSAL 1u
+
+/* The ST-SpAttn mask (Sec. 3.2).  The paper's mask is {anchor_frames 1, spatial_radius -1,
+ * temporal_depth 1, temporal_stride 1, temporal_radius 0}: a visual query attends the first
+ * frame, its own frame, and its own grid cell in the previous frame, all under causality.
+ * Other values are this library's extension.  Text queries are dense causal and prefix keys
+ * are visible to every query.  The mask is token-exact; `tile` only sets the granularity at
+ * which fully masked key blocks are skipped. */
+typedef struct {
+  int32_t grid_h, grid_w;  /* per-frame token grid                                         */
+  int32_t anchor_frames;   /* first frames every visual query sees                         */
+  int32_t spatial_radius;  /* -1: whole current frame; else Chebyshev radius in the grid   */
+  int32_t temporal_depth;  /* number of linked earlier frames; -1: all                     */
+  int32_t temporal_stride; /* linked frames are f-s, f-2s, ... (>= 1)                      */
+  int32_t temporal_radius; /* 0: same grid cell; r: Chebyshev radius; -1: whole frame      */
+  int32_t tile;            /* key-block size for skipping: 16, 32, 64 or 128               */
+  uint32_t flags;          /* PUREKV_FLAG_DENSE_CAUSAL: plain causal attention             */
+} purekv_st_params;
+
+/* Packed batch.  Device arrays feed kernels; host mirrors feed planning and launch sizing.
+ * Both must hold the same values. */
+typedef struct {
+  int32_t n_req;
+  int64_t total_tokens;        /* T = h_cu_seqlens[n_req]                                  */
+  const int32_t *cu_seqlens;   /* device [n_req+1]                                         */
+  const int32_t *h_cu_seqlens; /* host   [n_req+1]                                         */
+  const int32_t *h_n_prefix;   /* host   [n_req] text tokens before the video              */
+  const int32_t *h_n_frames;   /* host   [n_req]; suffix = len - n_prefix - n_frames*N     */
+} purekv_batch;
+
+/* Host-side summary of a built plan; filled by purekv_plan_build, read by
+ * purekv_st_sparse_prefill. */
+typedef struct {
+  int32_t tile_q, tile_k;   /* rows per query tile, keys per key tile                      */
+  int32_t n_qtiles;         /* query tiles over all requests                               */
+  int32_t max_list;         /* longest kept-tile list of a query tile                      */
+  int64_t tiles_kept;       /* key tiles kept (summed over query tiles)                    */
+  int64_t tiles_causal;     /* key tiles a dense causal mask would keep                    */
+  int64_t pairs_kept;       /* (query, key) pairs the mask keeps                           */
+  int64_t tiles_full, tiles_diag, tiles_general; /* kept tiles by predicate class          */
+  int64_t bytes_used;       /* bytes of the plan buffer actually written                   */
+  int32_t dtype, head_dim;  /* what the plan was built for                                 */
+} purekv_plan_info;
+
+const char *purekv_version(void);
+/* Copies the calling thread's last error text (NUL-terminated) into buf. */
+void purekv_last_error(char *buf, size_t buf_bytes);
+
+/* Budget rule: w <- min(window, len); k = min(len, max(w, floor(keep_ratio*len))); h = k - w.
+ * Host only.  (Sec. 3.1: recent window w plus top-h non-recent keys; budgets are quoted as a
+ * fraction of the cache, Tables 1-2.) */
+purekv_status purekv_budget(int32_t len, int32_t window, double keep_ratio, int32_t *h_out, int32_t *k_out);
+
+/* ---- planning (host work + one host-to-device copy) --------------------------------- */
+/* Upper bound of the plan buffer size in bytes for this batch and mask; 0 on invalid input. */
+size_t purekv_plan_bytes(const purekv_batch *batch, const purekv_st_params *params,
+                         purekv_dtype dtype, int32_t head_dim);
+/* Builds, on the host, the per-query-tile lists of key tiles the mask keeps (each tagged
+ * full / causal-only / general), a longest-first work order and per-token grid coordinates,
+ * then copies them into `plan` (device, plan_bytes >= purekv_plan_bytes) on `stream` and
+ * waits for that copy.  A plan depends only on the batch shape and mask, not on Q/K/V, and
+ * serves every layer and head. */
+purekv_status purekv_plan_build(const purekv_batch *batch, const purekv_st_params *params,
+                                purekv_dtype dtype, int32_t head_dim, void *plan, size_t plan_bytes,
+                                purekv_plan_info *h_info, void *stream);
+
+/* Same planning, written to a HOST buffer h_plan (plan_bytes >= purekv_plan_bytes); makes no
+ * CUDA call.  The bytes may be copied to the device by the caller and used as `plan`. */
+purekv_status purekv_plan_build_host(const purekv_batch *batch, const purekv_st_params *params,
+                                     purekv_dtype dtype, int32_t head_dim, void *h_plan, size_t plan_bytes,
+                                     purekv_plan_info *h_info);
+
+/* ---- ST-SpAttn prefill, one layer (Sec. 3.2; softmax of Eq. 1 over the kept keys) ------
+ * O[i,hq,:] = sum_{j<=i, M(i,j)} softmax_j(scale * q_i.k_j) v_j.   lse (nullable) [H, T] fp32
+ * receives log-sum-exp (natural log) of each row's kept logits.  softmax_scale 0 means
+ * 1/sqrt(head_dim).  bf16 with head_dim 128 and tile 64/128 runs on the tcgen05 tensor
+ * cores; other supported shapes (head_dim 32, 64, 128 or 256) run on CUDA cores.
+ * `status` (nullable) is a device int32 the kernel sets to PUREKV_ERR_TIMEOUT if a bounded
+ * wait expires; the caller zeroes it and reads it (purekv_poll_status). */
+purekv_status purekv_st_sparse_prefill(const void *q, const void *k, const void *v, void *o, float *lse,
+                                       const purekv_batch *batch, const void *plan,
+                                       const purekv_plan_info *h_info, int32_t n_q_heads,
+                                       int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                       float softmax_scale, int32_t *status, void *stream);
+
+/* ---- low-layer window scores (Eq. 1-2) -------------------------------------------------
+ * For request r of length l, w = min(window, l), KV head g, key j < l-w:
+ *   C[g, j] = (1/G) sum_{hq in group g} sum_{i=l-w}^{l-1} A^{hq}[i, j],
+ * A = dense causal softmax (each row normalised over all keys j' <= i).  c_out [H_kv, T]
+ * fp32; the last w entries of each request are written as 0.  The attention matrix is never
+ * stored.  ws: device workspace of purekv_score_ws_bytes. */
+size_t purekv_score_ws_bytes(const purekv_batch *batch, int32_t window, int32_t n_q_heads);
+purekv_status purekv_lowlayer_score(const void *q, const void *k, float *c_out, const purekv_batch *batch,
+                                    int32_t window, int32_t n_q_heads, int32_t n_kv_heads,
+                                    int32_t head_dim, purekv_dtype dtype, float softmax_scale,
+                                    void *ws, size_t ws_bytes, void *stream);
+
+/* ---- V-norm weighting and top-h selection, n_layers layers per call (Eq. 3-4) ----------
+ * S[L, g, j] = C[g, j] * ||V_L[j, g, :]||_2 for non-recent j; idx[L, g, cu_kept[r] + t] lists,
+ * for request r, the h_keep[r] positions with the largest S (ties: lower position), in
+ * ascending position order, followed by the window positions l-w .. l-1.  Positions are
+ * relative to the request.  v is [n_layers][T, H_kv, d] with v_layer_stride elements between
+ * layers.  idx_out [n_layers, H_kv, K_tot] int32, K_tot = h_cu_kept[n_req];
+ * cu_kept[r+1]-cu_kept[r] must equal h_keep[r] + min(window, l_r).
+ * s_out (nullable) [n_layers, H_kv, T] fp32 receives S.  ws: purekv_select_ws_bytes. */
+size_t purekv_select_ws_bytes(const purekv_batch *batch, int32_t n_layers, int32_t n_kv_heads);
+purekv_status purekv_select_topk(const float *c, const void *v, int64_t v_layer_stride, int32_t n_layers,
+                                 const purekv_batch *batch, int32_t window, const int32_t *keep /* device [n_req] */,
+                                 const int32_t *h_keep, const int32_t *cu_kept /* device [n_req+1] */,
+                                 const int32_t *h_cu_kept, int32_t n_kv_heads, int32_t head_dim,
+                                 purekv_dtype dtype, int32_t *idx_out, float *s_out, void *ws,
+                                 size_t ws_bytes, void *stream);
+
+/* ---- compaction (the compressed cache of Sec. 3.1) -------------------------------------
+ * k_out[L, cu_kept[r]+t, g, :] = k[L, cu_seqlens[r] + idx[L, g, cu_kept[r]+t], g, :], same for v.
+ * k, v: [n_layers][T, H_kv, d] with layer_stride elements between layers; outputs
+ * [n_layers][K_tot, H_kv, d] with out_layer_stride.  Pure copy, 128-bit vectorised; d * element
+ * size must be a multiple of 16 bytes and all bases 16-byte aligned. */
+purekv_status purekv_compact_kv(const void *k, const void *v, int64_t layer_stride, int32_t n_layers,
+                                const int32_t *idx, const purekv_batch *batch, const int32_t *cu_kept,
+                                const int32_t *h_cu_kept, int32_t n_kv_heads, int32_t head_dim,
+                                purekv_dtype dtype, void *k_out, void *v_out, int64_t out_layer_stride,
+                                void *stream);
+
+/* Synchronises `stream`, copies the device status word to *h_status_out and returns
+ * PUREKV_ERR_TIMEOUT if it is non-zero, PUREKV_ERR_CUDA if the stream reported an error. */
+purekv_status purekv_poll_status(const int32_t *status, int32_t *h_status_out, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PUREKV_H_ */

@@ -1,0 +1,323 @@
+// Host-side planning for ST-SpAttn prefill (Sec. 3.2): turns the batch shape and the mask
+// parameters into per-query-tile lists of kept key tiles, each classified as
+//   full    -- every (row, key) pair of the tile is kept: no predicate in the kernel,
+//   diag    -- exactly the causal pairs j <= i are kept: only the causal compare,
+//   general -- the token predicate is evaluated.
+// Work per query tile is O(rows x intervals): each row's kept keys are a union of a few
+// position intervals (prefix + first frames, spans of the current frame, spans or single cells
+// of linked earlier frames), accumulated into per-key-tile pair counts.
+#include <algorithm>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+namespace purekv {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+purekv_status check_batch(const purekv_batch* b, bool need_device) {
+  PK_REQUIRE(b != nullptr, PUREKV_ERR_INVALID_ARG, "batch is null");
+  PK_REQUIRE(b->n_req >= 0 && b->total_tokens >= 0, PUREKV_ERR_INVALID_ARG, "negative batch size");
+  PK_REQUIRE(b->h_cu_seqlens != nullptr, PUREKV_ERR_INVALID_ARG, "h_cu_seqlens is null");
+  PK_REQUIRE(!need_device || b->cu_seqlens != nullptr || b->n_req == 0, PUREKV_ERR_INVALID_ARG,
+             "cu_seqlens (device) is null");
+  PK_REQUIRE(b->h_cu_seqlens[0] == 0, PUREKV_ERR_INVALID_ARG, "cu_seqlens[0] must be 0");
+  for (int r = 0; r < b->n_req; ++r)
+    PK_REQUIRE(b->h_cu_seqlens[r + 1] >= b->h_cu_seqlens[r], PUREKV_ERR_INVALID_ARG,
+               "cu_seqlens must be non-decreasing (request %d)", r);
+  PK_REQUIRE(b->h_cu_seqlens[b->n_req] == b->total_tokens, PUREKV_ERR_INVALID_ARG,
+             "total_tokens %lld != cu_seqlens[n_req] %d", (long long)b->total_tokens,
+             b->h_cu_seqlens[b->n_req]);
+  return PUREKV_OK;
+}
+
+static int64_t align16(int64_t x) { return (x + 15) & ~int64_t(15); }
+
+static purekv_status check_params(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
+                                  int32_t head_dim, int* tile_q, int* tile_k) {
+  purekv_status st = check_batch(b, false);
+  if (st != PUREKV_OK) return st;
+  PK_REQUIRE(p != nullptr, PUREKV_ERR_INVALID_ARG, "params is null");
+  PK_REQUIRE(b->h_n_prefix && b->h_n_frames, PUREKV_ERR_INVALID_ARG, "h_n_prefix / h_n_frames is null");
+  PK_REQUIRE(p->grid_h >= 1 && p->grid_w >= 1 && p->grid_h <= 32767 && p->grid_w <= 32767,
+             PUREKV_ERR_INVALID_ARG, "grid %dx%d out of range", p->grid_h, p->grid_w);
+  PK_REQUIRE(p->tile == 16 || p->tile == 32 || p->tile == 64 || p->tile == 128, PUREKV_ERR_UNSUPPORTED,
+             "tile %d not in {16,32,64,128}", p->tile);
+  PK_REQUIRE(p->anchor_frames >= 0 && p->spatial_radius >= -1 && p->temporal_depth >= -1 &&
+                 p->temporal_radius >= -1 && p->temporal_stride >= 1 && p->temporal_stride <= 32767 &&
+                 p->temporal_depth <= 32767,
+             PUREKV_ERR_INVALID_ARG, "mask parameter out of range");
+  PK_REQUIRE(dtype == PUREKV_BF16 || dtype == PUREKV_FP32, PUREKV_ERR_INVALID_ARG, "unknown dtype");
+  const int64_t n = (int64_t)p->grid_h * p->grid_w;
+  for (int r = 0; r < b->n_req; ++r) {
+    const int64_t len = b->h_cu_seqlens[r + 1] - b->h_cu_seqlens[r];
+    PK_REQUIRE(b->h_n_prefix[r] >= 0 && b->h_n_frames[r] >= 0 && b->h_n_frames[r] <= 32767 &&
+                   b->h_n_prefix[r] + b->h_n_frames[r] * n <= len,
+               PUREKV_ERR_INVALID_ARG, "request %d: prefix %d + %d frames of %lld tokens exceed length %lld", r,
+               b->h_n_prefix[r], b->h_n_frames[r], (long long)n, (long long)len);
+  }
+  // Tensor-core kernel: 128 query rows per tile, keys per tile = the skip granularity.
+  const bool tc = dtype == PUREKV_BF16 && head_dim == 128 && (p->tile == 64 || p->tile == 128);
+  *tile_k = p->tile;
+  *tile_q = tc ? 128 : std::min(p->tile, 64);  // CUDA-core kernel: at most 64 rows per tile
+  return PUREKV_OK;
+}
+
+static void layout(const purekv_batch* b, int tile_q, int tile_k, int64_t* n_qtiles, int64_t* max_entries) {
+  int64_t nq = 0, ne = 0;
+  for (int r = 0; r < b->n_req; ++r) {
+    const int64_t len = b->h_cu_seqlens[r + 1] - b->h_cu_seqlens[r];
+    const int64_t q = (len + tile_q - 1) / tile_q;
+    nq += q;
+    for (int64_t t = 0; t < q; ++t) ne += (std::min(len, (t + 1) * tile_q) + tile_k - 1) / tile_k;
+  }
+  *n_qtiles = nq;
+  *max_entries = ne;
+}
+
+struct Span { int32_t a, b; };  // inclusive request-relative positions
+
+}  // namespace purekv
+
+using namespace purekv;
+
+extern "C" {
+
+const char* purekv_version(void) { return "purekv-b200 0.1.0 (sm_100a)"; }
+
+void purekv_last_error(char* buf, size_t n) {
+  if (!buf || n == 0) return;
+  strncpy(buf, g_err, n - 1);
+  buf[n - 1] = 0;
+}
+
+purekv_status purekv_budget(int32_t len, int32_t window, double keep_ratio, int32_t* h_out, int32_t* k_out) {
+  PK_REQUIRE(len >= 0 && window >= 0 && keep_ratio >= 0.0 && h_out && k_out, PUREKV_ERR_INVALID_ARG,
+             "purekv_budget: bad argument");
+  const int32_t w = std::min(window, len);
+  const double kf = keep_ratio * (double)len;
+  int32_t k = kf >= (double)len ? len : (int32_t)kf;  // floor of a non-negative value
+  k = std::min(len, std::max(w, k));
+  *h_out = k - w;
+  *k_out = k;
+  return PUREKV_OK;
+}
+
+size_t purekv_plan_bytes(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype, int32_t head_dim) {
+  int tq, tk;
+  if (check_params(b, p, dtype, head_dim, &tq, &tk) != PUREKV_OK) return 0;
+  int64_t nq, ne;
+  layout(b, tq, tk, &nq, &ne);
+  return (size_t)(align16(sizeof(PlanHeader)) + align16(nq * (int64_t)sizeof(QTile)) + align16(nq * 4) +
+                  align16(ne * 4) + align16(b->total_tokens * 8) + 64);
+}
+
+static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
+                                int32_t head_dim, size_t plan_bytes, purekv_plan_info* info,
+                                std::vector<uint8_t>& host) {
+  int tq, tk;
+  purekv_status st = check_params(b, p, dtype, head_dim, &tq, &tk);
+  if (st != PUREKV_OK) return st;
+  PK_REQUIRE(info, PUREKV_ERR_INVALID_ARG, "info is null");
+  PK_REQUIRE(plan_bytes >= purekv_plan_bytes(b, p, dtype, head_dim), PUREKV_ERR_WORKSPACE,
+             "plan buffer of %zu bytes is smaller than purekv_plan_bytes", plan_bytes);
+  const bool dense = (p->flags & PUREKV_FLAG_DENSE_CAUSAL) != 0;
+  const int32_t gw = p->grid_w, gh = p->grid_h, n = gw * gh;
+  const int64_t T = b->total_tokens;
+
+  int64_t nq_tot, ne_max;
+  layout(b, tq, tk, &nq_tot, &ne_max);
+  std::vector<QTile> qtiles;
+  qtiles.reserve((size_t)nq_tot);
+  std::vector<int32_t> entries;
+  entries.reserve((size_t)ne_max);
+  std::vector<int2> meta((size_t)T);
+  memset(info, 0, sizeof(*info));
+
+  std::vector<int64_t> cnt, diff;
+  std::vector<Span> spans;
+  for (int r = 0; r < b->n_req; ++r) {
+    const int32_t base = b->h_cu_seqlens[r];
+    const int32_t len = b->h_cu_seqlens[r + 1] - base;
+    const int32_t npre = b->h_n_prefix[r], nfr = b->h_n_frames[r];
+    const int32_t vis_end = npre + nfr * n;
+    for (int32_t i = 0; i < len; ++i) {
+      int2 m;
+      if (i < npre) m = make_int2(0, 0);
+      else if (i >= vis_end) m = make_int2(2, 0);
+      else {
+        const int32_t f = (i - npre) / n, c = (i - npre) % n;
+        m = make_int2(1 | (f << 2) | ((f % p->temporal_stride) << 17), (c / gw) | ((c % gw) << 16));
+      }
+      meta[(size_t)base + i] = m;
+    }
+    const int32_t nkt = (len + tk - 1) / tk;
+    cnt.assign((size_t)nkt + 1, 0);
+    diff.assign((size_t)nkt + 2, 0);
+    const int32_t anchor_end = std::min<int64_t>(vis_end, npre + (int64_t)p->anchor_frames * n);  // exclusive
+    for (int32_t q0 = 0; q0 < len; q0 += tq) {
+      const int32_t q1 = std::min(len, q0 + tq);  // exclusive
+      std::fill(cnt.begin(), cnt.end(), 0);
+      std::fill(diff.begin(), diff.end(), 0);
+      auto add_span = [&](int32_t a, int32_t bb) {  // inclusive, a <= bb
+        const int32_t ta = a / tk, tb = bb / tk;
+        if (ta == tb) { cnt[ta] += bb - a + 1; return; }
+        cnt[ta] += (ta + 1) * tk - a;
+        cnt[tb] += bb - tb * tk + 1;
+        diff[ta + 1] += tk;
+        diff[tb] -= tk;
+      };
+      for (int32_t i = q0; i < q1; ++i) {
+        const bool visual = i >= npre && i < vis_end;
+        if (dense || !visual) { add_span(0, i); continue; }
+        spans.clear();
+        if (anchor_end > 0) spans.push_back({0, std::min(i, anchor_end - 1)});  // prefix + first frames
+        const int32_t f = (i - npre) / n, c = (i - npre) % n, y = c / gw, x = c % gw;
+        const int32_t fs = npre + f * n;
+        if (p->spatial_radius < 0) spans.push_back({fs, i});
+        else {
+          const int32_t rr = p->spatial_radius;
+          for (int32_t yy = std::max(0, y - rr); yy <= y; ++yy) {
+            const int32_t xa = std::max(0, x - rr), xb = yy == y ? x : std::min(gw - 1, x + rr);
+            spans.push_back({fs + yy * gw + xa, fs + yy * gw + xb});
+          }
+        }
+        for (int32_t m = 1;; ++m) {
+          const int64_t fj = (int64_t)f - (int64_t)m * p->temporal_stride;
+          if (fj < 0 || (p->temporal_depth >= 0 && m > p->temporal_depth)) break;
+          const int32_t fjs = npre + (int32_t)fj * n;
+          if (p->temporal_radius < 0) spans.push_back({fjs, fjs + n - 1});
+          else {
+            const int32_t rr = p->temporal_radius;
+            for (int32_t yy = std::max(0, y - rr); yy <= std::min(gh - 1, y + rr); ++yy)
+              spans.push_back({fjs + yy * gw + std::max(0, x - rr), fjs + yy * gw + std::min(gw - 1, x + rr)});
+          }
+        }
+        std::sort(spans.begin(), spans.end(), [](const Span& u, const Span& v) { return u.a < v.a; });
+        int32_t ca = spans[0].a, cb = spans[0].b;
+        for (size_t s = 1; s < spans.size(); ++s) {
+          if (spans[s].a <= cb + 1) cb = std::max(cb, spans[s].b);
+          else { add_span(ca, cb); ca = spans[s].a; cb = spans[s].b; }
+        }
+        add_span(ca, cb);
+      }
+      QTile qt;
+      qt.q_start = base + q0;
+      qt.q_rows = q1 - q0;
+      qt.req_start = base;
+      qt.req_len = len;
+      qt.entry_begin = (int32_t)entries.size();
+      qt.pad[0] = qt.pad[1] = 0;
+      int64_t run = 0;
+      const int32_t kt_hi = (q1 - 1) / tk;  // last key tile a causal mask reaches
+      for (int32_t kt = 0; kt <= kt_hi; ++kt) {
+        run += diff[kt];
+        const int64_t c = cnt[kt] + run;
+        info->tiles_causal++;
+        if (c == 0) continue;
+        const int32_t j0 = kt * tk;
+        const int64_t full = (int64_t)(q1 - q0) * tk;
+        int64_t causal = full;  // pairs with j <= i inside this tile
+        if (j0 + tk - 1 > q0) {
+          causal = 0;
+          for (int32_t i = q0; i < q1; ++i) causal += std::max(0, std::min(tk, i - j0 + 1));
+        }
+        int32_t cls = kTileGeneral;
+        if (c == full && j0 + tk <= len) cls = kTileFull;
+        else if (c == causal) cls = kTileDiag;
+        entries.push_back((kt << 2) | cls);
+        info->pairs_kept += c;
+        info->tiles_kept++;
+        (cls == kTileFull ? info->tiles_full : cls == kTileDiag ? info->tiles_diag : info->tiles_general)++;
+      }
+      qt.entry_count = (int32_t)entries.size() - qt.entry_begin;
+      info->max_list = std::max(info->max_list, qt.entry_count);
+      qtiles.push_back(qt);
+    }
+  }
+  const int32_t nq = (int32_t)qtiles.size();
+  std::vector<int32_t> order((size_t)nq);
+  for (int32_t i = 0; i < nq; ++i) order[i] = i;
+  std::stable_sort(order.begin(), order.end(),
+                   [&](int32_t u, int32_t v) { return qtiles[u].entry_count > qtiles[v].entry_count; });
+
+  PlanHeader h;
+  memset(&h, 0, sizeof(h));
+  h.magic = kPlanMagic;
+  h.tile_q = tq;
+  h.tile_k = tk;
+  h.n_qtiles = nq;
+  h.total_tokens = T;
+  h.n_entries = (int64_t)entries.size();
+  h.off_qtiles = align16(sizeof(PlanHeader));
+  h.off_order = h.off_qtiles + align16((int64_t)nq * sizeof(QTile));
+  h.off_entries = h.off_order + align16((int64_t)nq * 4);
+  h.off_meta = h.off_entries + align16(h.n_entries * 4);
+  h.anchor_frames = p->anchor_frames;
+  h.spatial_radius = p->spatial_radius;
+  h.temporal_depth = p->temporal_depth;
+  h.temporal_stride = p->temporal_stride;
+  h.temporal_radius = p->temporal_radius;
+  h.dense_causal = dense ? 1 : 0;
+  const int64_t total = h.off_meta + align16(T * 8);
+  PK_REQUIRE((size_t)total <= plan_bytes, PUREKV_ERR_WORKSPACE, "plan needs %lld bytes", (long long)total);
+
+  host.assign((size_t)total, 0);
+  memcpy(host.data(), &h, sizeof(h));
+  if (nq) memcpy(host.data() + h.off_qtiles, qtiles.data(), (size_t)nq * sizeof(QTile));
+  if (nq) memcpy(host.data() + h.off_order, order.data(), (size_t)nq * 4);
+  if (!entries.empty()) memcpy(host.data() + h.off_entries, entries.data(), entries.size() * 4);
+  if (T) memcpy(host.data() + h.off_meta, meta.data(), (size_t)T * 8);
+
+  info->tile_q = tq;
+  info->tile_k = tk;
+  info->n_qtiles = nq;
+  info->bytes_used = total;
+  info->dtype = (int32_t)dtype;
+  info->head_dim = head_dim;
+  return PUREKV_OK;
+}
+
+purekv_status purekv_plan_build_host(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
+                                     int32_t head_dim, void* h_plan, size_t plan_bytes, purekv_plan_info* info) {
+  PK_REQUIRE(h_plan, PUREKV_ERR_INVALID_ARG, "h_plan is null");
+  std::vector<uint8_t> host;
+  purekv_status st = build_plan(b, p, dtype, head_dim, plan_bytes, info, host);
+  if (st != PUREKV_OK) return st;
+  memcpy(h_plan, host.data(), host.size());
+  return PUREKV_OK;
+}
+
+purekv_status purekv_plan_build(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
+                                int32_t head_dim, void* plan, size_t plan_bytes, purekv_plan_info* info,
+                                void* stream) {
+  PK_REQUIRE(plan, PUREKV_ERR_INVALID_ARG, "plan is null");
+  std::vector<uint8_t> host;
+  purekv_status st = build_plan(b, p, dtype, head_dim, plan_bytes, info, host);
+  if (st != PUREKV_OK) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  PK_CUDA(cudaMemcpyAsync(plan, host.data(), host.size(), cudaMemcpyHostToDevice, s));
+  PK_CUDA(cudaStreamSynchronize(s));
+  return PUREKV_OK;
+}
+
+purekv_status purekv_poll_status(const int32_t* status, int32_t* h_out, void* stream) {
+  cudaStream_t s = (cudaStream_t)stream;
+  PK_CUDA(cudaStreamSynchronize(s));
+  int32_t v = 0;
+  if (status) PK_CUDA(cudaMemcpy(&v, status, sizeof(v), cudaMemcpyDeviceToHost));
+  if (h_out) *h_out = v;
+  PK_REQUIRE(v == 0, PUREKV_ERR_TIMEOUT, "device status word is %d: a bounded device-side wait expired", v);
+  return PUREKV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,28 @@
+// purekv_st_sparse_prefill: argument checks and dispatch to the tensor-core or CUDA-core kernel.
+#include "prefill.cuh"
+
+using namespace purekv;
+
+extern "C" purekv_status purekv_st_sparse_prefill(const void* q, const void* k, const void* v, void* o, float* lse,
+                                                  const purekv_batch* batch, const void* plan,
+                                                  const purekv_plan_info* info, int32_t n_q_heads, int32_t n_kv_heads,
+                                                  int32_t head_dim, purekv_dtype dtype, float softmax_scale,
+                                                  int32_t* status, void* stream) {
+  purekv_status st = check_batch(batch, false);
+  if (st != PUREKV_OK) return st;
+  PK_REQUIRE(q && k && v && o && plan && info, PUREKV_ERR_INVALID_ARG, "purekv_st_sparse_prefill: null pointer");
+  PK_REQUIRE(n_q_heads >= 1 && n_kv_heads >= 1 && n_q_heads % n_kv_heads == 0 && n_q_heads <= 65535,
+             PUREKV_ERR_INVALID_ARG, "n_q_heads %d must be a positive multiple of n_kv_heads %d", n_q_heads,
+             n_kv_heads);
+  PK_REQUIRE(dtype == PUREKV_BF16 || dtype == PUREKV_FP32, PUREKV_ERR_INVALID_ARG, "unknown dtype");
+  PK_REQUIRE(info->dtype == (int32_t)dtype && info->head_dim == head_dim, PUREKV_ERR_INVALID_ARG,
+             "plan was built for dtype %d head_dim %d, call has dtype %d head_dim %d", info->dtype, info->head_dim,
+             (int)dtype, head_dim);
+  PK_REQUIRE(((uintptr_t)q | (uintptr_t)k | (uintptr_t)v | (uintptr_t)o | (uintptr_t)plan) % 16 == 0,
+             PUREKV_ERR_INVALID_ARG, "Q/K/V/O/plan must be 16-byte aligned");
+  if (info->n_qtiles == 0) return PUREKV_OK;
+  PrefillArgs a{q, k, v, o, lse, batch, plan, info, n_q_heads, n_kv_heads, head_dim, dtype,
+                softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim), status, (cudaStream_t)stream};
+  if (dtype == PUREKV_BF16 && head_dim == 128 && info->tile_q == 128) return launch_prefill_tc(a);
+  return launch_prefill_simt(a);
+}

@@ -1,0 +1,273 @@
+// purekv_lowlayer_score: window attention scores of the low layer (Eq. 1-2).
+//
+// For each request and KV head g the G*w query rows of the recent window (G query heads of
+// the group x w positions) are stacked; row (hl, iw) is query head g*G+hl at position
+// i = l-w+iw.  Pass 1 streams the keys once per 32-row block and keeps a running
+// (max, sum of exponentials) per row -> log-sum-exp over all causal keys j <= i (Eq. 1's row
+// normaliser).  Pass 2 gives each CTA one block of 64 non-recent keys: it recomputes the
+// logits of every stacked row against those keys, forms exp(s - lse) and sums down the rows
+// (Eq. 2), so the attention matrix never leaves the SM and no atomics are needed.
+// Logits are fp32 FMA chains over exact products; exponentials use exp2f.
+#include <algorithm>
+
+#include "common.cuh"
+
+namespace purekv {
+
+constexpr int kRB = 32;        // stacked rows per block
+constexpr int kKB = 64;        // keys per block
+constexpr int kThreads = 256;  // thread (ty, tx): rows 2*ty, 2*ty+1; keys tx, tx+16, tx+32, tx+48
+
+template <typename T>
+__device__ __forceinline__ void load_row_f32(float* dst, const T* src, int d, int lane_in_group, int group_size) {
+  for (int c = lane_in_group; c < d; c += group_size) dst[c] = to_f32(src[c]);
+}
+
+// s[a][b] = <q row 2*ty+a, key tx+16*b> over d, both tiles in shared memory with row stride ld.
+__device__ __forceinline__ void tile_dots(const float* qs, const float* ks, int d, int ld, int ty, int tx,
+                                          float s[2][4]) {
+#pragma unroll
+  for (int a = 0; a < 2; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) s[a][b] = 0.f;
+  const float4* q0 = reinterpret_cast<const float4*>(qs + (2 * ty) * ld);
+  const float4* q1 = reinterpret_cast<const float4*>(qs + (2 * ty + 1) * ld);
+  for (int c = 0; c < d / 4; ++c) {
+    const float4 a0 = q0[c], a1 = q1[c];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const float4 kk = reinterpret_cast<const float4*>(ks + (tx + 16 * b) * ld)[c];
+      s[0][b] = fmaf(a0.x, kk.x, s[0][b]);
+      s[0][b] = fmaf(a0.y, kk.y, s[0][b]);
+      s[0][b] = fmaf(a0.z, kk.z, s[0][b]);
+      s[0][b] = fmaf(a0.w, kk.w, s[0][b]);
+      s[1][b] = fmaf(a1.x, kk.x, s[1][b]);
+      s[1][b] = fmaf(a1.y, kk.y, s[1][b]);
+      s[1][b] = fmaf(a1.z, kk.z, s[1][b]);
+      s[1][b] = fmaf(a1.w, kk.w, s[1][b]);
+    }
+  }
+}
+
+// Pass 1.  grid (row blocks, n_kv_heads, n_req).  lse2 [n_req][H][window] in log2 units of the
+// scaled logits (s * scale * log2 e).
+template <typename T>
+__global__ void __launch_bounds__(kThreads) score_lse_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                             const int32_t* __restrict__ cu_seqlens, int32_t window,
+                                                             int32_t n_q_heads, int32_t n_kv_heads, int32_t d,
+                                                             float scale_log2, float* __restrict__ lse2) {
+  extern __shared__ __align__(16) float smem[];
+  const int ld = d + 4;
+  float* qs = smem;             // [kRB][ld]
+  float* ks = smem + kRB * ld;  // [kKB][ld]
+  const int32_t r = blockIdx.z, g = blockIdx.y;
+  const int32_t G = n_q_heads / n_kv_heads;
+  const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
+  const int32_t w = min(window, len);
+  const int32_t n_rows = G * w;
+  const int32_t row0 = blockIdx.x * kRB;
+  if (row0 >= n_rows) return;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  // stage the query rows (rows past n_rows are zero)
+  for (int rr = tid >> 3; rr < kRB; rr += kThreads / 8) {
+    const int32_t row = row0 + rr;
+    float* dst = qs + rr * ld;
+    if (row < n_rows) {
+      const int32_t hq = g * G + row / w, i = len - w + row % w;
+      load_row_f32(dst, q + ((int64_t)(base + i) * n_q_heads + hq) * d, d, tid & 7, 8);
+    } else {
+      for (int c = tid & 7; c < d; c += 8) dst[c] = 0.f;
+    }
+  }
+  int32_t my_i[2];
+#pragma unroll
+  for (int a = 0; a < 2; ++a) {
+    const int32_t row = row0 + 2 * ty + a;
+    my_i[a] = row < n_rows ? len - w + row % w : -1;
+  }
+  // last key any row of this block needs
+  const int32_t last_row = min(n_rows, row0 + kRB) - 1;
+  int32_t i_max = 0;
+  if (row0 / w == last_row / w) i_max = len - w + last_row % w; else i_max = len - 1;
+  float m[2] = {-INFINITY, -INFINITY}, l[2] = {0.f, 0.f};
+  for (int32_t j0 = 0; j0 <= i_max; j0 += kKB) {
+    __syncthreads();
+    for (int rr = tid >> 3; rr < kKB; rr += kThreads / 8) {
+      const int32_t j = j0 + rr;
+      float* dst = ks + rr * ld;
+      if (j < len) load_row_f32(dst, k + ((int64_t)(base + j) * n_kv_heads + g) * d, d, tid & 7, 8);
+      else for (int c = tid & 7; c < d; c += 8) dst[c] = 0.f;
+    }
+    __syncthreads();
+    float s[2][4];
+    tile_dots(qs, ks, d, ld, ty, tx, s);
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+      float tmax = -INFINITY;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int32_t j = j0 + tx + 16 * b;
+        s[a][b] = j <= my_i[a] ? s[a][b] * scale_log2 : -INFINITY;
+        tmax = fmaxf(tmax, s[a][b]);
+      }
+      if (tmax > -INFINITY) {
+        const float mn = fmaxf(m[a], tmax);
+        float add = 0.f;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) add += exp2f(s[a][b] - mn);
+        l[a] = l[a] * exp2f(m[a] - mn) + add;
+        m[a] = mn;
+      }
+    }
+  }
+  // combine the 16 threads (tx) that share a row: lanes differ in the low 4 bits
+#pragma unroll
+  for (int a = 0; a < 2; ++a) {
+#pragma unroll
+    for (int off = 8; off >= 1; off >>= 1) {
+      const float mo = __shfl_xor_sync(0xffffffffu, m[a], off), lo = __shfl_xor_sync(0xffffffffu, l[a], off);
+      const float mn = fmaxf(m[a], mo);
+      if (mn > -INFINITY) {
+        l[a] = l[a] * exp2f(m[a] - mn) + lo * exp2f(mo - mn);
+        m[a] = mn;
+      }
+    }
+    const int32_t row = row0 + 2 * ty + a;
+    if (tx == 0 && row < n_rows)
+      lse2[((int64_t)r * n_q_heads + g * G + row / w) * window + row % w] = m[a] + log2f(l[a]);
+  }
+}
+
+// Pass 2.  grid (key blocks over the longest request, n_kv_heads, n_req).
+template <typename T>
+__global__ void __launch_bounds__(kThreads) score_colsum_kernel(const T* __restrict__ q, const T* __restrict__ k,
+                                                                const int32_t* __restrict__ cu_seqlens,
+                                                                int32_t window, int32_t n_q_heads,
+                                                                int32_t n_kv_heads, int32_t d, float scale_log2,
+                                                                const float* __restrict__ lse2, int64_t n_tokens,
+                                                                float* __restrict__ c_out) {
+  extern __shared__ __align__(16) float smem[];
+  __shared__ float red[kThreads / 16][kKB];
+  const int ld = d + 4;
+  float* qs = smem;
+  float* ks = smem + kRB * ld;
+  const int32_t r = blockIdx.z, g = blockIdx.y;
+  const int32_t G = n_q_heads / n_kv_heads;
+  const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
+  const int32_t w = min(window, len);
+  const int32_t nr = len - w;  // non-recent keys
+  const int32_t j0 = blockIdx.x * kKB;
+  if (j0 >= len) return;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  float* cg = c_out + (int64_t)g * n_tokens + base;
+  if (j0 >= nr) {  // block inside the window: defined as 0
+    for (int c = tid; c < kKB; c += kThreads)
+      if (j0 + c < len) cg[j0 + c] = 0.f;
+    return;
+  }
+  for (int rr = tid >> 3; rr < kKB; rr += kThreads / 8) {
+    const int32_t j = j0 + rr;
+    float* dst = ks + rr * ld;
+    if (j < len) load_row_f32(dst, k + ((int64_t)(base + j) * n_kv_heads + g) * d, d, tid & 7, 8);
+    else for (int c = tid & 7; c < d; c += 8) dst[c] = 0.f;
+  }
+  const int32_t n_rows = G * w;
+  float col[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int32_t row0 = 0; row0 < n_rows; row0 += kRB) {
+    __syncthreads();
+    for (int rr = tid >> 3; rr < kRB; rr += kThreads / 8) {
+      const int32_t row = row0 + rr;
+      float* dst = qs + rr * ld;
+      if (row < n_rows) {
+        const int32_t hq = g * G + row / w, i = len - w + row % w;
+        load_row_f32(dst, q + ((int64_t)(base + i) * n_q_heads + hq) * d, d, tid & 7, 8);
+      } else {
+        for (int c = tid & 7; c < d; c += 8) dst[c] = 0.f;
+      }
+    }
+    __syncthreads();
+    float s[2][4];
+    tile_dots(qs, ks, d, ld, ty, tx, s);
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+      const int32_t row = row0 + 2 * ty + a;
+      if (row < n_rows) {
+        const float lse = __ldg(lse2 + ((int64_t)r * n_q_heads + g * G + row / w) * window + row % w);
+        // every non-recent key precedes every window row, so causality holds for all of them
+#pragma unroll
+        for (int b = 0; b < 4; ++b) col[b] += exp2f(s[a][b] * scale_log2 - lse);
+      }
+    }
+  }
+#pragma unroll
+  for (int b = 0; b < 4; ++b) red[ty][tx + 16 * b] = col[b];
+  __syncthreads();
+  if (tid < kKB) {
+    float sum = 0.f;
+#pragma unroll
+    for (int t = 0; t < kThreads / 16; ++t) sum += red[t][tid];
+    const int32_t j = j0 + tid;
+    if (j < len) cg[j] = j < nr ? sum / (float)G : 0.f;
+  }
+}
+
+static int32_t max_len(const purekv_batch* b) {
+  int32_t m = 0;
+  for (int r = 0; r < b->n_req; ++r) m = std::max(m, b->h_cu_seqlens[r + 1] - b->h_cu_seqlens[r]);
+  return m;
+}
+
+template <typename T>
+static purekv_status launch_score(const void* q, const void* k, float* c_out, const purekv_batch* b, int32_t window,
+                                  int32_t H, int32_t Hkv, int32_t d, float scale, float* lse2, cudaStream_t sm) {
+  const int32_t ml = max_len(b);
+  const int32_t w = std::min(window, ml);
+  const int32_t G = H / Hkv;
+  const size_t smem = (size_t)(kRB + kKB) * (d + 4) * sizeof(float);
+  PK_CUDA(cudaFuncSetAttribute(score_lse_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  PK_CUDA(cudaFuncSetAttribute(score_colsum_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const float scale_log2 = scale * 1.4426950408889634f;
+  dim3 g1((unsigned)((G * w + kRB - 1) / kRB), (unsigned)Hkv, (unsigned)b->n_req);
+  score_lse_kernel<T><<<g1, kThreads, smem, sm>>>((const T*)q, (const T*)k, b->cu_seqlens, window, H, Hkv, d, scale_log2,
+                                                  lse2);
+  PK_CUDA(cudaGetLastError());
+  dim3 g2((unsigned)((ml + kKB - 1) / kKB), (unsigned)Hkv, (unsigned)b->n_req);
+  score_colsum_kernel<T><<<g2, kThreads, smem, sm>>>((const T*)q, (const T*)k, b->cu_seqlens, window, H, Hkv, d,
+                                                     scale_log2, lse2, b->total_tokens, c_out);
+  PK_CUDA(cudaGetLastError());
+  return PUREKV_OK;
+}
+
+}  // namespace purekv
+
+using namespace purekv;
+
+extern "C" size_t purekv_score_ws_bytes(const purekv_batch* batch, int32_t window, int32_t n_q_heads) {
+  if (!batch || window < 0 || n_q_heads < 0) return 0;
+  return (size_t)batch->n_req * n_q_heads * (size_t)std::max(window, 1) * sizeof(float) + 256;
+}
+
+extern "C" purekv_status purekv_lowlayer_score(const void* q, const void* k, float* c_out, const purekv_batch* batch,
+                                               int32_t window, int32_t n_q_heads, int32_t n_kv_heads,
+                                               int32_t head_dim, purekv_dtype dtype, float softmax_scale, void* ws,
+                                               size_t ws_bytes, void* stream) {
+  purekv_status st = check_batch(batch, true);
+  if (st != PUREKV_OK) return st;
+  PK_REQUIRE(q && k && c_out, PUREKV_ERR_INVALID_ARG, "purekv_lowlayer_score: null pointer");
+  PK_REQUIRE(n_q_heads >= 1 && n_kv_heads >= 1 && n_q_heads % n_kv_heads == 0, PUREKV_ERR_INVALID_ARG,
+             "n_q_heads %d must be a positive multiple of n_kv_heads %d", n_q_heads, n_kv_heads);
+  PK_REQUIRE(window >= 1, PUREKV_ERR_INVALID_ARG, "window must be >= 1");
+  PK_REQUIRE(head_dim >= 4 && head_dim % 4 == 0 && head_dim <= 256, PUREKV_ERR_UNSUPPORTED,
+             "head_dim %d: need a multiple of 4 up to 256", head_dim);
+  PK_REQUIRE(dtype == PUREKV_BF16 || dtype == PUREKV_FP32, PUREKV_ERR_INVALID_ARG, "unknown dtype");
+  PK_REQUIRE(n_kv_heads <= 65535 && batch->n_req <= 65535, PUREKV_ERR_UNSUPPORTED, "too many heads or requests");
+  if (batch->n_req == 0 || batch->total_tokens == 0) return PUREKV_OK;
+  PK_REQUIRE(ws && ws_bytes >= purekv_score_ws_bytes(batch, window, n_q_heads), PUREKV_ERR_WORKSPACE,
+             "purekv_lowlayer_score: workspace of %zu bytes is too small", ws_bytes);
+  float* lse2 = (float*)(((uintptr_t)ws + 255) & ~(uintptr_t)255);
+  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+  cudaStream_t sm = (cudaStream_t)stream;
+  if (dtype == PUREKV_BF16)
+    return launch_score<__nv_bfloat16>(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
+  return launch_score<float>(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
+}

@@ -1,0 +1,273 @@
+// purekv_select_topk: V-norm weighting (Eq. 3 / Eq. 4) and budgeted top-h selection (Sec. 3.1).
+//
+// Two kernels.  vnorm_score_kernel streams V once (the only large traffic of this step):
+// a warp owns 32 consecutive tokens of one KV head, each half-warp reads one 16-byte-chunked
+// row per step, reduces the squared norm with shuffles, and the warp writes 32 consecutive
+// scores S = C * ||V||.  select_kernel then handles one (layer, KV head, request) segment per
+// CTA: a 4 x 8-bit MSB-first radix select over the fp32 bit patterns finds the h-th largest
+// score, and a block-scan compaction emits the chosen positions in ascending order; among
+// scores equal to the threshold the lowest positions win, so the result is deterministic.
+#include <algorithm>
+
+#include "common.cuh"
+
+namespace purekv {
+
+template <typename T>
+struct Chunk;  // one 16-byte load
+template <>
+struct Chunk<float> {
+  static __device__ __forceinline__ float sumsq(uint4 u) {
+    const float a = __uint_as_float(u.x), b = __uint_as_float(u.y), c = __uint_as_float(u.z),
+                d = __uint_as_float(u.w);
+    return a * a + b * b + c * c + d * d;
+  }
+};
+template <>
+struct Chunk<__nv_bfloat16> {
+  static __device__ __forceinline__ float sumsq(uint4 u) {
+    float s = 0.f;
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+      s = fmaf(lo, lo, s);
+      s = fmaf(hi, hi, s);
+    }
+    return s;
+  }
+};
+
+// grid: (ceil(T/32) token blocks split over x, n_kv_heads, n_layers); block: 256 threads = 8 warps.
+template <typename T>
+__global__ void __launch_bounds__(256) vnorm_score_kernel(const uint4* __restrict__ v, int64_t layer_stride_c,
+                                                          const float* __restrict__ c, int64_t n_tokens,
+                                                          int32_t n_kv_heads, int32_t chunks_per_row,
+                                                          float* __restrict__ s_out) {
+  const int32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int32_t g = blockIdx.y, layer = blockIdx.z;
+  const uint4* vl = v + layer * layer_stride_c;
+  float* so = s_out + ((int64_t)layer * n_kv_heads + g) * n_tokens;
+  const float* cg = c + (int64_t)g * n_tokens;
+  const int64_t n_blocks = (n_tokens + 31) / 32;
+  for (int64_t blk = (int64_t)blockIdx.x * 8 + warp; blk < n_blocks; blk += (int64_t)gridDim.x * 8) {
+    const int64_t t0 = blk * 32;
+    float mine = 0.f;
+    if (chunks_per_row == 16) {
+      // 256-byte rows: a half-warp covers one row per step, 16 steps cover 32 tokens.
+      const int32_t half = lane >> 4, ch = lane & 15;
+      float part[16];
+#pragma unroll
+      for (int it = 0; it < 16; ++it) {
+        const int64_t t = t0 + it * 2 + half;
+        uint4 u = make_uint4(0, 0, 0, 0);
+        if (t < n_tokens) u = __ldg(vl + (t * n_kv_heads + g) * 16 + ch);
+        part[it] = Chunk<T>::sumsq(u);
+      }
+#pragma unroll
+      for (int it = 0; it < 16; ++it) {
+        float p = part[it];
+        p += __shfl_xor_sync(0xffffffffu, p, 8);
+        p += __shfl_xor_sync(0xffffffffu, p, 4);
+        p += __shfl_xor_sync(0xffffffffu, p, 2);
+        p += __shfl_xor_sync(0xffffffffu, p, 1);
+        // lanes 0..15 now hold token 2*it's sum, lanes 16..31 token 2*it+1's; lane L keeps token L
+        const float v0 = __shfl_sync(0xffffffffu, p, 0), v1 = __shfl_sync(0xffffffffu, p, 16);
+        if (lane == it * 2) mine = v0;
+        if (lane == it * 2 + 1) mine = v1;
+      }
+    } else {
+      // generic row length: one token per lane, sequential chunks
+      const int64_t t = t0 + lane;
+      if (t < n_tokens) {
+        const uint4* row = vl + (t * n_kv_heads + g) * chunks_per_row;
+        for (int32_t ch = 0; ch < chunks_per_row; ++ch) mine += Chunk<T>::sumsq(__ldg(row + ch));
+      }
+    }
+    const int64_t t = t0 + lane;
+    if (t < n_tokens) so[t] = __ldg(cg + t) * sqrtf(mine);
+  }
+}
+
+__device__ __forceinline__ uint32_t order_key(float f) {
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelItems = 4;
+
+// One CTA per (request, KV head, layer).
+__global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ s, int64_t n_tokens,
+                                                             const int32_t* __restrict__ cu_seqlens,
+                                                             const int32_t* __restrict__ cu_kept,
+                                                             const int32_t* __restrict__ keep, int32_t window,
+                                                             int32_t k_tot, int32_t n_kv_heads,
+                                                             int32_t* __restrict__ idx_out) {
+  __shared__ int32_t hist[256];
+  __shared__ uint32_t sh_prefix;
+  __shared__ int32_t sh_need;
+  __shared__ int32_t warp_gt[32], warp_eq[32];
+  __shared__ int32_t carry_gt, carry_eq;
+
+  const int32_t r = blockIdx.x, g = blockIdx.y, layer = blockIdx.z;
+  const int32_t base = cu_seqlens[r];
+  const int32_t len = cu_seqlens[r + 1] - base;
+  const int32_t w = min(window, len);
+  const int32_t nr = len - w;
+  const int32_t h = keep[r];
+  const float* seg = s + ((int64_t)layer * n_kv_heads + g) * n_tokens + base;
+  int32_t* out = idx_out + ((int64_t)layer * n_kv_heads + g) * k_tot + cu_kept[r];
+  const int32_t tid = threadIdx.x;
+
+  for (int32_t t = tid; t < w; t += kSelThreads) out[h + t] = nr + t;  // the recent window
+  if (h <= 0) return;
+
+  // ---- radix select: the h-th largest key --------------------------------------------
+  uint32_t prefix = 0, mask = 0;
+  int32_t need = h;  // rank still to find among keys matching the prefix
+  for (int32_t shift = 24; shift >= 0; shift -= 8) {
+    if (tid < 256) hist[tid] = 0;
+    __syncthreads();
+    for (int32_t j = tid; j < nr; j += kSelThreads) {
+      const uint32_t key = order_key(__ldg(seg + j));
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+    }
+    __syncthreads();
+    if (tid == 0) {
+      int32_t acc = 0, b = 255;
+      for (; b > 0; --b) {
+        if (acc + hist[b] >= need) break;
+        acc += hist[b];
+      }
+      sh_prefix = prefix | ((uint32_t)b << shift);
+      sh_need = need - acc;
+    }
+    __syncthreads();
+    prefix = sh_prefix;
+    need = sh_need;
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t thr = prefix;  // key of the h-th largest score
+  const int32_t need_eq = need; // how many keys equal to thr are taken (lowest positions first)
+
+  // ---- ordered compaction --------------------------------------------------------------
+  if (tid == 0) { carry_gt = 0; carry_eq = 0; }
+  __syncthreads();
+  const int32_t lane = tid & 31, warp = tid >> 5;
+  for (int32_t c0 = 0; c0 < nr; c0 += kSelThreads * kSelItems) {
+    const int32_t j0 = c0 + tid * kSelItems;
+    uint32_t keys[kSelItems];
+    int32_t n_gt = 0, n_eq = 0;
+#pragma unroll
+    for (int i = 0; i < kSelItems; ++i) {
+      keys[i] = (j0 + i < nr) ? order_key(__ldg(seg + j0 + i)) : 0u;
+      const bool valid = j0 + i < nr;
+      n_gt += (valid && keys[i] > thr);
+      n_eq += (valid && keys[i] == thr);
+    }
+    int32_t inc_gt = n_gt, inc_eq = n_eq;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int32_t a = __shfl_up_sync(0xffffffffu, inc_gt, d), b = __shfl_up_sync(0xffffffffu, inc_eq, d);
+      if (lane >= d) { inc_gt += a; inc_eq += b; }
+    }
+    if (lane == 31) { warp_gt[warp] = inc_gt; warp_eq[warp] = inc_eq; }
+    __syncthreads();
+    if (warp == 0) {
+      int32_t a = warp_gt[lane], b = warp_eq[lane];
+      const int32_t ta = a, tb = b;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int32_t x = __shfl_up_sync(0xffffffffu, a, d), y = __shfl_up_sync(0xffffffffu, b, d);
+        if (lane >= d) { a += x; b += y; }
+      }
+      warp_gt[lane] = a - ta;  // exclusive
+      warp_eq[lane] = b - tb;
+    }
+    __syncthreads();
+    int32_t pos_gt = carry_gt + warp_gt[warp] + inc_gt - n_gt;  // exclusive counts before this thread
+    int32_t pos_eq = carry_eq + warp_eq[warp] + inc_eq - n_eq;
+#pragma unroll
+    for (int i = 0; i < kSelItems; ++i) {
+      if (j0 + i < nr) {
+        if (keys[i] > thr) {
+          out[pos_gt + min(pos_eq, need_eq)] = j0 + i;
+          ++pos_gt;
+        } else if (keys[i] == thr) {
+          if (pos_eq < need_eq) out[pos_gt + pos_eq] = j0 + i;
+          ++pos_eq;
+        }
+      }
+    }
+    __syncthreads();
+    if (tid == kSelThreads - 1) { carry_gt = pos_gt; carry_eq = pos_eq; }
+    __syncthreads();
+  }
+}
+
+}  // namespace purekv
+
+using namespace purekv;
+
+extern "C" size_t purekv_select_ws_bytes(const purekv_batch* batch, int32_t n_layers, int32_t n_kv_heads) {
+  if (!batch || n_layers < 0 || n_kv_heads < 0) return 0;
+  return (size_t)n_layers * n_kv_heads * batch->total_tokens * sizeof(float) + 256;
+}
+
+extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64_t v_layer_stride, int32_t n_layers,
+                                            const purekv_batch* batch, int32_t window, const int32_t* keep,
+                                            const int32_t* h_keep, const int32_t* cu_kept, const int32_t* h_cu_kept,
+                                            int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                            int32_t* idx_out, float* s_out, void* ws, size_t ws_bytes, void* stream) {
+  purekv_status st = check_batch(batch, true);
+  if (st != PUREKV_OK) return st;
+  PK_REQUIRE(c && v && keep && h_keep && cu_kept && h_cu_kept && idx_out, PUREKV_ERR_INVALID_ARG,
+             "purekv_select_topk: null pointer");
+  PK_REQUIRE(n_layers >= 0 && n_layers <= 65535 && n_kv_heads >= 1 && n_kv_heads <= 65535 && head_dim >= 1 &&
+                 window >= 0,
+             PUREKV_ERR_INVALID_ARG, "purekv_select_topk: bad sizes");
+  PK_REQUIRE(dtype == PUREKV_BF16 || dtype == PUREKV_FP32, PUREKV_ERR_INVALID_ARG, "unknown dtype");
+  const int64_t esz = dtype == PUREKV_BF16 ? 2 : 4;
+  PK_REQUIRE((head_dim * esz) % 16 == 0, PUREKV_ERR_UNSUPPORTED, "V row of %lld bytes is not a multiple of 16",
+             (long long)(head_dim * esz));
+  PK_REQUIRE((v_layer_stride * esz) % 16 == 0 && (uintptr_t)v % 16 == 0, PUREKV_ERR_INVALID_ARG,
+             "V base and layer stride must be 16-byte aligned");
+  PK_REQUIRE(h_cu_kept[0] == 0, PUREKV_ERR_INVALID_ARG, "cu_kept[0] must be 0");
+  for (int r = 0; r < batch->n_req; ++r) {
+    const int32_t len = batch->h_cu_seqlens[r + 1] - batch->h_cu_seqlens[r];
+    const int32_t w = std::min(window, len);
+    PK_REQUIRE(h_keep[r] >= 0 && h_keep[r] <= len - w, PUREKV_ERR_INVALID_ARG,
+               "request %d: h = %d outside [0, %d]", r, h_keep[r], len - w);
+    PK_REQUIRE(h_cu_kept[r + 1] - h_cu_kept[r] == h_keep[r] + w, PUREKV_ERR_INVALID_ARG,
+               "request %d: cu_kept step %d != h + w = %d", r, h_cu_kept[r + 1] - h_cu_kept[r], h_keep[r] + w);
+  }
+  const int64_t T = batch->total_tokens;
+  if (n_layers == 0 || T == 0 || batch->n_req == 0) return PUREKV_OK;
+  float* s_buf = s_out;
+  if (!s_buf) {
+    PK_REQUIRE(ws && ws_bytes >= purekv_select_ws_bytes(batch, n_layers, n_kv_heads), PUREKV_ERR_WORKSPACE,
+               "purekv_select_topk: workspace of %zu bytes is too small", ws_bytes);
+    s_buf = (float*)(((uintptr_t)ws + 255) & ~(uintptr_t)255);
+  }
+  cudaStream_t sm = (cudaStream_t)stream;
+  const int32_t cpr = (int32_t)(head_dim * esz / 16);
+  const int64_t n_blocks = (T + 31) / 32;
+  // 148 SMs x 8 resident CTAs shared by the (head, layer) planes of the grid.
+  const int64_t planes = (int64_t)n_kv_heads * n_layers;
+  const int64_t want = std::max<int64_t>(1, (148 * 8 + planes - 1) / planes);
+  dim3 g1((unsigned)std::min<int64_t>((n_blocks + 7) / 8, want), (unsigned)n_kv_heads, (unsigned)n_layers);
+  if (dtype == PUREKV_BF16)
+    vnorm_score_kernel<__nv_bfloat16><<<g1, 256, 0, sm>>>((const uint4*)v, v_layer_stride * esz / 16, c, T, n_kv_heads,
+                                                          cpr, s_buf);
+  else
+    vnorm_score_kernel<float><<<g1, 256, 0, sm>>>((const uint4*)v, v_layer_stride * esz / 16, c, T, n_kv_heads, cpr,
+                                                  s_buf);
+  PK_CUDA(cudaGetLastError());
+  dim3 g2((unsigned)batch->n_req, (unsigned)n_kv_heads, (unsigned)n_layers);
+  select_kernel<<<g2, kSelThreads, 0, sm>>>(s_buf, T, batch->cu_seqlens, cu_kept, keep, window, h_cu_kept[batch->n_req],
+                                            n_kv_heads, idx_out);
+  PK_CUDA(cudaGetLastError());
+  return PUREKV_OK;
+}

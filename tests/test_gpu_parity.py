@@ -1,0 +1,175 @@
+"""GPU parity: the CUDA path (through the C-ABI binding) against the fp64 oracle."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import purekv_oracle as po
+from paper_2510_25600_b200 import inputs
+from tests import gpu_common as gc
+
+pytestmark = pytest.mark.gpu
+
+
+def make_wl(dtype, H, Hkv, d, n_prefix, n_frames, n_suffix, gh, gw, tile, window=8, keep=0.3, seed=11, **mask_kw):
+    batch = inputs.make_batch(n_prefix, n_frames, n_suffix, gh, gw)
+    return inputs.Workload("t", seed, dtype, H, Hkv, d, 1, (0,), (0,), batch, inputs.STMask(gh, gw, tile=tile, **mask_kw),
+                           window, keep)
+
+
+# ---------------------------------------------------------------- prefill ---------------
+@pytest.mark.parametrize("mask_kw", [{}, dict(dense_causal=True),
+                                     dict(anchor_frames=2, spatial_radius=1, temporal_depth=2, temporal_stride=2, temporal_radius=1)])
+@pytest.mark.parametrize("dtype,d,tile", [("fp32", 64, 16), ("fp32", 32, 32), ("bf16", 64, 64), ("fp32", 128, 64)])
+def test_prefill_cuda_core_kernel(dtype, d, tile, mask_kw):
+    wl = make_wl(dtype, 4, 2, d, [5, 0, 9], [4, 3, 0], [7, 33, 3], 5, 6, tile, **mask_kw)
+    gc.check_prefill(wl, inputs.make_qkv(wl, 0))
+
+
+@pytest.mark.parametrize("mask_kw", [{}, dict(dense_causal=True),
+                                     dict(anchor_frames=0, spatial_radius=2, temporal_depth=-1, temporal_stride=2, temporal_radius=-1),
+                                     dict(anchor_frames=2, spatial_radius=-1, temporal_depth=3, temporal_radius=1)])
+@pytest.mark.parametrize("tile", [64, 128])
+def test_prefill_tensor_core_kernel(tile, mask_kw):
+    # several requests, lengths that are not multiples of the tile, frames that straddle tiles
+    wl = make_wl("bf16", 4, 2, 128, [37, 0, 5, 1], [5, 3, 1, 0], [29, 140, 0, 2], 9, 11, tile, **mask_kw)
+    gc.check_prefill(wl, inputs.make_qkv(wl, 0))
+
+
+def test_prefill_tensor_core_single_token_and_tiny_requests():
+    wl = make_wl("bf16", 2, 1, 128, [1, 0, 3], [0, 1, 0], [0, 0, 126], 1, 1, 128)
+    gc.check_prefill(wl, inputs.make_qkv(wl, 0))
+
+
+def test_prefill_cfg0():
+    wl = inputs.workload(0)
+    err, plan = gc.check_prefill(wl, inputs.make_qkv(wl, 0))
+    assert (plan.info.tiles_kept, plan.info.tiles_causal) == (131, 171)
+
+
+def test_prefill_is_deterministic():
+    wl = make_wl("bf16", 4, 2, 128, [10], [6], [50], 8, 8, 128)
+    x = inputs.make_qkv(wl, 0)
+    a, la, _ = gc.gpu_prefill(wl, x)
+    b, lb, _ = gc.gpu_prefill(wl, x)
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16)) and torch.equal(la, lb)
+
+
+# ------------------------------------------------- score / select / compact -------------
+def run_compress(wl, layers_x, window, keep):
+    """layers_x: list of per-layer dicts; layer 0 is the scored layer.  Returns everything needed."""
+    P = gc.pk()
+    db = gc.device_batch(wl)
+    bud = P.Budget(db, window, keep)
+    q0, k0 = gc.upload(layers_x[0], "q", wl.dtype), gc.upload(layers_x[0], "k", wl.dtype)
+    c = P.purekv_lowlayer_score(q0, k0, db, window)
+    ks = torch.stack([gc.upload(x, "k", wl.dtype) for x in layers_x])
+    vs = torch.stack([gc.upload(x, "v", wl.dtype) for x in layers_x])
+    s = torch.empty((len(layers_x), wl.n_kv_heads, db.total_tokens), dtype=torch.float32, device="cuda")
+    idx = P.purekv_select_topk(c, vs, db, bud, s_out=s)
+    idx_ws = P.purekv_select_topk(c, vs, db, bud)          # workspace path must agree
+    assert torch.equal(idx, idx_ws)
+    kc, vc = P.purekv_compact_kv(ks, vs, idx, db, bud)
+    torch.cuda.synchronize()
+    return c, s, idx, kc, vc, bud
+
+
+def check_compress(wl, n_layers, window, keep):
+    layers_x = [inputs.make_qkv(wl, l) for l in range(n_layers)]
+    c, s, idx, kc, vc, bud = run_compress(wl, layers_x, window, keep)
+    b = wl.batch
+    cu = b.cu_seqlens
+    c_ref = po.lowlayer_score(layers_x[0]["q"], layers_x[0]["k"], cu, window)
+    assert gc.score_error(c.cpu().numpy(), c_ref) <= gc.SCORE_RTOL
+    hk, ck = po.budgets(b.seq_lens, window, keep)
+    assert np.array_equal(hk, bud.h_keep) and np.array_equal(ck, bud.h_cu_kept)
+    for l in range(n_layers):
+        x = layers_x[l]
+        s_ref = po.vnorm_scores(c_ref, x["v"])
+        s_gpu = s[l].cpu().numpy()
+        assert gc.score_error(s_gpu, s_ref) <= gc.SCORE_RTOL
+        idx_ref, kth = po.select(s_ref, cu, window, hk, ck)
+        idx_gpu = idx[l].cpu().numpy()
+        gc.check_index_sets(idx_gpu, idx_ref, s_ref, kth, wl, hk, ck, window)
+        # selection alone, on the GPU's own fp32 scores: bit-exact against the oracle's selection rule
+        idx_self, _ = po.select(s_gpu.astype(np.float64), cu, window, hk, ck)
+        assert np.array_equal(idx_gpu, idx_self)
+        # compaction: bit-exact against the oracle's gather driven by the GPU's indices
+        bits = "k_bits" if wl.dtype == "bf16" else "k"
+        vbits = "v_bits" if wl.dtype == "bf16" else "v"
+        view = (lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16)) if wl.dtype == "bf16" else (lambda t: t.cpu().numpy())
+        assert np.array_equal(view(kc[l]), po.compact(x[bits], idx_gpu, cu, ck))
+        assert np.array_equal(view(vc[l]), po.compact(x[vbits], idx_gpu, cu, ck))
+
+
+@pytest.mark.parametrize("dtype,d", [("fp32", 64), ("bf16", 128), ("bf16", 64)])
+@pytest.mark.parametrize("window,keep", [(8, 0.3), (1, 0.1), (40, 0.5), (8, 1.0), (500, 0.2)])
+def test_compress_small(dtype, d, window, keep):
+    wl = make_wl(dtype, 6, 2, d, [5, 0, 9], [4, 3, 0], [17, 45, 30], 5, 6, 64)
+    check_compress(wl, 3, window, keep)
+
+
+def test_compress_cfg0():
+    wl = inputs.workload(0)
+    check_compress(wl, 1, wl.window, wl.keep_ratio)
+
+
+def test_select_with_ties_picks_lowest_positions():
+    P = gc.pk()
+    db = P.Batch([4100], [0], [0])
+    bud = P.Budget(db, 100, 0.5)
+    T = 4100
+    c = torch.ones((1, T), dtype=torch.float32, device="cuda")
+    v = torch.ones((1, T, 1, 8), dtype=torch.float32, device="cuda")          # every score equal
+    idx = P.purekv_select_topk(c, v, db, bud).cpu().numpy()[0, 0]
+    h = int(bud.h_keep[0])
+    assert np.array_equal(idx[:h], np.arange(h)) and np.array_equal(idx[h:], np.arange(4000, 4100))
+    c[0, 1000:1010] = 2.0
+    c[0, 3000] = 0.5
+    idx = P.purekv_select_topk(c, v, db, bud).cpu().numpy()[0, 0]
+    want = np.sort(np.concatenate([np.arange(1000, 1010), np.arange(0, h - 10)]))
+    assert np.array_equal(idx[:h], want)
+
+
+def test_compact_keep_all_is_identity_and_guard_bands_survive():
+    P = gc.pk()
+    wl = make_wl("bf16", 2, 2, 128, [3, 1], [2, 1], [9, 4], 4, 4, 64)
+    x = inputs.make_qkv(wl, 0)
+    db = gc.device_batch(wl)
+    bud = P.Budget(db, 4, 1.0)
+    k = gc.upload(x, "k", "bf16")[None].contiguous()
+    v = gc.upload(x, "v", "bf16")[None].contiguous()
+    c = P.purekv_lowlayer_score(gc.upload(x, "q", "bf16"), k[0], db, 4)
+    idx = P.purekv_select_topk(c, v, db, bud)
+    n = k.numel()
+    guard = torch.full((2, n + 512), 0x7B7B, dtype=torch.int16, device="cuda")
+    ko = guard[0, 256:256 + n].view(torch.bfloat16).view(k.shape)
+    vo = guard[1, 256:256 + n].view(torch.bfloat16).view(k.shape)
+    P.purekv_compact_kv(k, v, idx, db, bud, k_out=ko, v_out=vo)
+    torch.cuda.synchronize()
+    assert torch.equal(ko.view(torch.int16), k.view(torch.int16)) and torch.equal(vo.view(torch.int16), v.view(torch.int16))
+    assert (guard[:, :256] == 0x7B7B).all() and (guard[:, 256 + n:] == 0x7B7B).all()
+
+
+def test_empty_inputs_and_bad_arguments():
+    P = gc.pk()
+    db = P.Batch([], [], [])
+    bud = P.Budget(db, 4, 0.5)
+    z = torch.empty((0, 2, 128), dtype=torch.bfloat16, device="cuda")
+    plan = P.purekv_plan_build(db, P.st_params(inputs.STMask(4, 4, tile=64)), P.BF16, 128)
+    P.purekv_st_sparse_prefill(z, z, z, db, plan)
+    c = P.purekv_lowlayer_score(z, z, db, 4)
+    idx = P.purekv_select_topk(c, z[None], db, bud)
+    P.purekv_compact_kv(z[None], z[None], idx, db, bud)
+    torch.cuda.synchronize()
+    db = P.Batch([40], [0], [0])
+    q = torch.zeros((40, 3, 128), dtype=torch.bfloat16, device="cuda")
+    kv = torch.zeros((40, 2, 128), dtype=torch.bfloat16, device="cuda")
+    plan = P.purekv_plan_build(db, P.st_params(inputs.STMask(4, 4, tile=64)), P.BF16, 128)
+    with pytest.raises(P.PureKVError) as e:
+        P.purekv_st_sparse_prefill(q, kv, kv, db, plan)          # 3 query heads, 2 KV heads
+    assert e.value.status == P.ERR_INVALID_ARG
+    with pytest.raises(P.PureKVError) as e:
+        P.purekv_lowlayer_score(q[:, :2].contiguous(), kv, db, 4, ws=torch.empty(8, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == P.ERR_WORKSPACE

@@ -1,0 +1,154 @@
+"""CPU tests of the C-ABI library's host side: it loads, exports what include/purekv.h
+declares, validates arguments, and its plan builder agrees with the oracle's mask."""
+import ctypes as C
+import os
+import re
+import struct
+
+import numpy as np
+import pytest
+
+from oracle import purekv_oracle as po
+from paper_2510_25600_b200 import binding as pk
+from paper_2510_25600_b200 import inputs
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    text = open(os.path.join(ROOT, "include", "purekv.h")).read()
+    declared = set(re.findall(r"\b(purekv_[a-z_0-9]+)\s*\(", text))
+    assert declared == set(pk.EXPORTS)
+    lib = C.CDLL(pk.LIB_PATH)
+    for name in declared:
+        assert hasattr(lib, name), name
+    assert "sm_100a" in pk.purekv_version()
+
+
+def test_budget_matches_oracle_rule():
+    for length in [0, 1, 7, 57, 288, 2432, 8320, 37120, 12393]:
+        for window in [1, 16, 64, 256, 100000]:
+            for keep in [0.0, 0.05, 0.1, 0.2, 0.35, 0.5, 0.999, 1.0]:
+                assert pk.purekv_budget(length, window, keep) == po.budget(length, window, keep)
+
+
+def parse_plan(buf: np.ndarray):
+    raw = buf.tobytes()
+    magic, tq, tk, nq, T, ne, oq, oo, oe, om, A, rs, D, st, rt, dense = struct.unpack_from("<Iiiiqqqqqqiiiiii", raw, 0)
+    assert magic == 0x504B5631
+    qt = np.frombuffer(raw, dtype=np.int32, count=nq * 8, offset=oq).reshape(nq, 8)
+    order = np.frombuffer(raw, dtype=np.int32, count=nq, offset=oo)
+    entries = np.frombuffer(raw, dtype=np.int32, count=ne, offset=oe)
+    meta = np.frombuffer(raw, dtype=np.int32, count=2 * T, offset=om).reshape(T, 2)
+    return dict(tq=tq, tk=tk, nq=nq, T=T, qt=qt, order=order, entries=entries, meta=meta,
+                params=(A, rs, D, st, rt, dense))
+
+
+def check_plan(batch: inputs.Batch, mask: inputs.STMask, dtype, head_dim):
+    b = pk.Batch(batch.seq_lens, batch.n_prefix, batch.n_frames, device=None)
+    buf, info = pk.purekv_plan_build_host(b, pk.st_params(mask), dtype, head_dim)
+    p = parse_plan(buf)
+    tq, tk = p["tq"], p["tk"]
+    assert (tq, tk) == (info.tile_q, info.tile_k)
+    mp = po.mask_params(mask)
+    cu = batch.cu_seqlens
+    pairs = kept = full = diag = gen = causal_tiles = 0
+    qi = 0
+    n = mask.grid_h * mask.grid_w
+    for r in range(batch.n_req):
+        l = batch.seq_lens[r]
+        mm = po.mask_matrix(mp, l, batch.n_prefix[r], batch.n_frames[r])
+        pairs += int(mm.sum())
+        # per-token coordinates
+        for i in range(l):
+            mx, my = p["meta"][cu[r] + i]
+            v = i - batch.n_prefix[r]
+            if v < 0:
+                assert mx & 3 == 0
+            elif v >= batch.n_frames[r] * n:
+                assert mx & 3 == 2
+            else:
+                f, c = divmod(v, n)
+                assert mx & 3 == 1 and (mx >> 2) & 0x7FFF == f and (mx >> 17) & 0x7FFF == f % mask.temporal_stride
+                assert my & 0xFFFF == c // mask.grid_w and (my >> 16) & 0xFFFF == c % mask.grid_w
+        for q0 in range(0, l, tq):
+            q1 = min(l, q0 + tq)
+            row = p["qt"][qi]
+            qi += 1
+            assert row[0] == cu[r] + q0 and row[1] == q1 - q0 and row[2] == cu[r] and row[3] == l
+            ents = p["entries"][row[4]:row[4] + row[5]]
+            listed = {int(e) >> 2: int(e) & 3 for e in ents}
+            assert len(listed) == len(ents) and list(listed) == sorted(listed)
+            nkt = (q1 - 1) // tk + 1
+            causal_tiles += nkt
+            for kt in range(nkt):
+                j0, j1 = kt * tk, min(l, kt * tk + tk)
+                sub = mm[q0:q1, j0:j1]
+                cnt = int(sub.sum())
+                if cnt == 0:
+                    assert kt not in listed
+                    continue
+                kept += 1
+                cls = listed[kt]
+                causal_cnt = int(np.tril(np.ones((l, l), dtype=bool))[q0:q1, j0:j1].sum())
+                if cnt == (q1 - q0) * tk:
+                    assert cls == 0
+                    full += 1
+                elif cnt == causal_cnt:
+                    assert cls == 1
+                    diag += 1
+                else:
+                    assert cls == 2
+                    gen += 1
+    assert qi == p["nq"] == info.n_qtiles
+    assert (info.pairs_kept, info.tiles_kept, info.tiles_causal) == (pairs, kept, causal_tiles)
+    assert (info.tiles_full, info.tiles_diag, info.tiles_general) == (full, diag, gen)
+    order = p["order"]
+    assert sorted(order.tolist()) == list(range(p["nq"]))
+    counts = p["qt"][order, 5]
+    assert (np.diff(counts) <= 0).all()
+    return info
+
+
+@pytest.mark.parametrize("tile", [16, 64])
+@pytest.mark.parametrize("mask_kw", [{}, dict(dense_causal=True), dict(anchor_frames=2, spatial_radius=1, temporal_depth=2,
+                                                                       temporal_stride=2, temporal_radius=1),
+                                     dict(anchor_frames=0, spatial_radius=0, temporal_depth=-1, temporal_radius=-1),
+                                     dict(temporal_depth=-1, temporal_stride=3, temporal_radius=0)])
+def test_plan_matches_oracle_mask(tile, mask_kw):
+    batch = inputs.make_batch([5, 0, 20], [6, 3, 0], [9, 40, 3], 5, 7)
+    check_plan(batch, inputs.STMask(5, 7, tile=tile, **mask_kw), pk.FP32, 64)
+
+
+def test_plan_for_tensor_core_shapes_and_workload_counts():
+    batch = inputs.make_batch([64, 3], [5, 2], [64, 130], 12, 12)
+    for tile in (64, 128):
+        info = check_plan(batch, inputs.STMask(12, 12, tile=tile), pk.BF16, 128)
+        assert info.tile_q == 128 and info.tile_k == tile
+    # cfg 0: pair count of the paper's mask (closed form) and the block density quoted for 16-tiles
+    wl = inputs.workload(0)
+    info = check_plan(wl.batch, wl.mask, pk.FP32, 64)
+    assert info.pairs_kept == 29456 and (info.tiles_kept, info.tiles_causal) == (131, 171)
+
+
+def test_plan_pair_counts_on_the_large_workloads():
+    # pairs kept = closed-form pair count of the paper's mask (derived in tests/test_oracle_mask.py)
+    for cfg, pairs in [(1, 783264), (2, 4148800), (3, 41042944)]:
+        wl = inputs.workload(cfg)
+        b = pk.Batch(wl.batch.seq_lens, wl.batch.n_prefix, wl.batch.n_frames, device=None)
+        _, info = pk.purekv_plan_build_host(b, pk.st_params(wl.mask), pk.BF16, 128)
+        assert info.pairs_kept == pairs
+        assert info.tile_q == 128 and 0 < info.tiles_kept < info.tiles_causal
+
+
+def test_argument_errors():
+    b = pk.Batch([10], [2], [1], device=None)
+    with pytest.raises(pk.PureKVError) as e:
+        pk.purekv_plan_build_host(b, pk.st_params(inputs.STMask(4, 4)), pk.FP32, 64)     # 2 + 16 > 10
+    assert e.value.status == pk.ERR_INVALID_ARG
+    b = pk.Batch([30], [2], [1], device=None)
+    with pytest.raises(pk.PureKVError) as e:
+        pk.purekv_plan_build_host(b, pk.st_params(inputs.STMask(4, 4, tile=48)), pk.FP32, 64)
+    assert e.value.status == pk.ERR_UNSUPPORTED
+    with pytest.raises(pk.PureKVError):
+        pk.purekv_budget(-1, 4, 0.5)
