@@ -19,6 +19,8 @@
  *  - A request's tokens are ordered [n_prefix text][n_frames x (grid_h x grid_w) visual,
  *    raster order inside a frame][suffix text].
  *  - dtype is the element type of Q/K/V/O; accumulation, softmax and scores are fp32.
+ *  - A batch with no requests or no tokens is valid everywhere: the call returns PUREKV_OK
+ *    without touching any buffer (tensor pointers may then be null).
  */
 #ifndef PUREKV_H_
 #define PUREKV_H_

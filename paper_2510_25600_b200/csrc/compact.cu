@@ -50,6 +50,7 @@ extern "C" purekv_status purekv_compact_kv(const void* k, const void* v, int64_t
                                            void* stream) {
   purekv_status st = check_batch(batch, true);
   if (st != PUREKV_OK) return st;
+  if (batch->total_tokens == 0 || batch->n_req == 0) return PUREKV_OK;  // empty batch: nothing to do
   PK_REQUIRE(k && v && idx && cu_kept && h_cu_kept && k_out && v_out, PUREKV_ERR_INVALID_ARG,
              "purekv_compact_kv: null pointer");
   PK_REQUIRE(n_layers >= 0 && n_kv_heads >= 1 && head_dim >= 1, PUREKV_ERR_INVALID_ARG,

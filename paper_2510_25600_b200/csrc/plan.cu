@@ -28,7 +28,7 @@ purekv_status check_batch(const purekv_batch* b, bool need_device) {
   PK_REQUIRE(b != nullptr, PUREKV_ERR_INVALID_ARG, "batch is null");
   PK_REQUIRE(b->n_req >= 0 && b->total_tokens >= 0, PUREKV_ERR_INVALID_ARG, "negative batch size");
   PK_REQUIRE(b->h_cu_seqlens != nullptr, PUREKV_ERR_INVALID_ARG, "h_cu_seqlens is null");
-  PK_REQUIRE(!need_device || b->cu_seqlens != nullptr || b->n_req == 0, PUREKV_ERR_INVALID_ARG,
+  PK_REQUIRE(!need_device || b->cu_seqlens != nullptr || b->n_req == 0 || b->total_tokens == 0, PUREKV_ERR_INVALID_ARG,
              "cu_seqlens (device) is null");
   PK_REQUIRE(b->h_cu_seqlens[0] == 0, PUREKV_ERR_INVALID_ARG, "cu_seqlens[0] must be 0");
   for (int r = 0; r < b->n_req; ++r)

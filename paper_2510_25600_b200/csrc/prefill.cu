@@ -10,6 +10,7 @@ extern "C" purekv_status purekv_st_sparse_prefill(const void* q, const void* k, 
                                                   int32_t* status, void* stream) {
   purekv_status st = check_batch(batch, false);
   if (st != PUREKV_OK) return st;
+  if (batch->total_tokens == 0 || batch->n_req == 0) return PUREKV_OK;  // empty batch: nothing to do
   PK_REQUIRE(q && k && v && o && plan && info, PUREKV_ERR_INVALID_ARG, "purekv_st_sparse_prefill: null pointer");
   PK_REQUIRE(n_q_heads >= 1 && n_kv_heads >= 1 && n_q_heads % n_kv_heads == 0 && n_q_heads <= 65535,
              PUREKV_ERR_INVALID_ARG, "n_q_heads %d must be a positive multiple of n_kv_heads %d", n_q_heads,

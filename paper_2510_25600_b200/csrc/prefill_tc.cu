@@ -172,7 +172,8 @@ struct __align__(8) Barriers {
   uint64_t q_full;
   uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
   uint64_t s_full[2], p_full[2];
-  uint64_t o_done;
+  uint64_t o_done;   // one completion per P.V product (tile m completes phase m)
+  uint64_t o_final;  // completes once, after the last P.V product
   uint64_t drain;
 };
 
@@ -222,6 +223,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       mbar_init(smem_u32(&bars.p_full[b]), 128);
     }
     mbar_init(smem_u32(&bars.o_done), 1);
+    mbar_init(smem_u32(&bars.o_final), 1);
     mbar_init(smem_u32(&bars.drain), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -308,6 +310,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         if (n >= 1 && !issue_pv(n - 1)) { ok = false; break; }
       }
       if (ok) ok = issue_pv(nt - 1);
+      if (ok) tc_commit(smem_u32(&bars.o_final));
       if (!ok) {
         // leaving early: let every issued MMA finish before TMEM is released
         tc_commit(smem_u32(&bars.drain));
@@ -404,6 +407,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       // rescale O and the running sum where the reference moved (warp-uniform decision)
       const float alpha = grow ? (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_use)) : 1.f;
       if (n > 0 && __any_sync(0xffffffffu, grow)) {
+        // S[b] of tile n is complete, hence so is P.V of tile n-2: o_done is in phase n-1 or n
         if (!wait_w(smem_u32(&bars.o_done), (n - 1) & 1)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll
@@ -422,7 +426,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       tc_fence_before();
       mbar_arrive(smem_u32(&bars.p_full[b]));
     }
-    if (ok) ok = wait_w(smem_u32(&bars.o_done), (nt - 1) & 1);
+    // The per-tile o_done barrier may still be two phases behind here (nothing orders the last
+    // softmax step after the second-to-last P.V), which a parity wait cannot tell apart; the
+    // dedicated single-phase barrier can.
+    if (ok) ok = wait_w(smem_u32(&bars.o_final), 0);
     if (ok) {
       tc_fence_after();
       const float inv = 1.f / l_sum;

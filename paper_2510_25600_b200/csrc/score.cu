@@ -253,6 +253,7 @@ extern "C" purekv_status purekv_lowlayer_score(const void* q, const void* k, flo
                                                size_t ws_bytes, void* stream) {
   purekv_status st = check_batch(batch, true);
   if (st != PUREKV_OK) return st;
+  if (batch->total_tokens == 0 || batch->n_req == 0) return PUREKV_OK;  // empty batch: nothing to do
   PK_REQUIRE(q && k && c_out, PUREKV_ERR_INVALID_ARG, "purekv_lowlayer_score: null pointer");
   PK_REQUIRE(n_q_heads >= 1 && n_kv_heads >= 1 && n_q_heads % n_kv_heads == 0, PUREKV_ERR_INVALID_ARG,
              "n_q_heads %d must be a positive multiple of n_kv_heads %d", n_q_heads, n_kv_heads);

@@ -223,6 +223,7 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
                                             int32_t* idx_out, float* s_out, void* ws, size_t ws_bytes, void* stream) {
   purekv_status st = check_batch(batch, true);
   if (st != PUREKV_OK) return st;
+  if (batch->total_tokens == 0 || batch->n_req == 0) return PUREKV_OK;  // empty batch: nothing to do
   PK_REQUIRE(c && v && keep && h_keep && cu_kept && h_cu_kept && idx_out, PUREKV_ERR_INVALID_ARG,
              "purekv_select_topk: null pointer");
   PK_REQUIRE(n_layers >= 0 && n_layers <= 65535 && n_kv_heads >= 1 && n_kv_heads <= 65535 && head_dim >= 1 &&

@@ -125,10 +125,11 @@ def test_select_with_ties_picks_lowest_positions():
     idx = P.purekv_select_topk(c, v, db, bud).cpu().numpy()[0, 0]
     h = int(bud.h_keep[0])
     assert np.array_equal(idx[:h], np.arange(h)) and np.array_equal(idx[h:], np.arange(4000, 4100))
-    c[0, 1000:1010] = 2.0
-    c[0, 3000] = 0.5
+    c[0, 3000:3010] = 2.0
+    c[0, 5] = 0.5
     idx = P.purekv_select_topk(c, v, db, bud).cpu().numpy()[0, 0]
-    want = np.sort(np.concatenate([np.arange(1000, 1010), np.arange(0, h - 10)]))
+    ties = np.setdiff1d(np.arange(0, h - 10 + 1), [5])           # the h-10 lowest positions among the ties
+    want = np.sort(np.concatenate([np.arange(3000, 3010), ties]))
     assert np.array_equal(idx[:h], want)
 
 
