@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the PureKV hot path on B200.
+
+A step = one pass of the whole hot path over one synthetic batch: planning, ST-SpAttn prefill
+of every layer (dense causal up to the CLIE layer), low-layer window scores, V-norm top-h
+selection and K/V compaction of the compressed layers.  Default workload: the
+VideoLLaMA2-shaped one (32 layers, 32/8 heads, head_dim 128, 2432 tokens, bf16).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--cfg 1] [--impl reference]
+
+Prints ONE JSON line (rank 0).  `value` = prefill tokens/s of the whole job with inputs
+resident in HBM; `e2e` = the same with inputs in pinned host memory and the compact cache read
+back; `roofline` describes the dominant kernel (tensor-core prefill); `cpu_baseline` is the
+fp64 oracle timed on this machine's host cores on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "st_spattn_prefill_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample(wl, layers_x, budget_s: float = 20.0):
+    """Times the oracle on a bounded sample of the step; returns (tokens/s extrapolated to the whole step,
+    cores, description).  Prefill: all heads of a row sample of one ST layer and of the dense layer; score,
+    selection and compaction of one layer in full."""
+    from oracle import purekv_oracle as po
+    b = wl.batch
+    cu = b.cu_seqlens
+    t_tot = b.total_tokens
+    rng = np.random.default_rng(wl.seed)
+    cores = len(os.sched_getaffinity(0))
+    x0 = layers_x[0]
+    x1 = next((x for x in layers_x[1:] if "q" in x), x0)
+    dense = type(wl.mask)(wl.mask.grid_h, wl.mask.grid_w, tile=wl.mask.tile, dense_causal=True)
+    n_rows = min(t_tot, 256)
+    rows = np.sort(rng.choice(t_tot, size=n_rows, replace=False))
+    t = time.perf_counter()
+    po.prefill(x1["q"], x1["k"], x1["v"], cu, b.n_prefix, b.n_frames, po.mask_params(wl.mask), rows=rows)
+    t_st = (time.perf_counter() - t) * t_tot / n_rows
+    t = time.perf_counter()
+    po.prefill(x0["q"], x0["k"], x0["v"], cu, b.n_prefix, b.n_frames, po.mask_params(dense), rows=rows)
+    t_dense = (time.perf_counter() - t) * t_tot / n_rows
+    t = time.perf_counter()
+    c = po.lowlayer_score(x0["q"], x0["k"], cu, wl.window)
+    t_score = time.perf_counter() - t
+    hk, ck = po.budgets(b.seq_lens, wl.window, wl.keep_ratio)
+    t = time.perf_counter()
+    s = po.vnorm_scores(c, x1["v"])
+    idx, _ = po.select(s, cu, wl.window, hk, ck)
+    po.compact(x1["k"], idx, cu, ck)
+    po.compact(x1["v"], idx, cu, ck)
+    t_comp = time.perf_counter() - t
+    n_dense = max(wl.scored_layers) + 1
+    n_st = wl.n_layers - n_dense
+    total = n_dense * t_dense + n_st * t_st + len(wl.scored_layers) * t_score + len(wl.compacted_layers) * t_comp
+    desc = (f"{n_rows} seeded rows x all {wl.n_q_heads} heads of one ST layer and one dense layer, full score / select / "
+            f"compact of one layer; extrapolated to {n_dense} dense + {n_st} ST layers, {len(wl.scored_layers)} scored, "
+            f"{len(wl.compacted_layers)} compacted")
+    return t_tot / total, cores, desc, total
+
+
+def run_reference(args, wl):
+    """--impl reference: the oracle as it stands, on host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import purekv_oracle as po
+    from paper_2510_25600_b200 import inputs
+    po.build()
+    pool = ThreadPoolExecutor(len(os.sched_getaffinity(0)))
+    layers_x = [inputs.make_qkv(wl, l, pool=pool) for l in range(min(2, wl.n_layers))]
+    vals, tot = [], 0.0
+    for i in range(args.warmup + args.steps):
+        v, cores, desc, total = oracle_sample(wl, layers_x)
+        if i >= args.warmup:
+            vals.append(v)
+            tot += total
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / max(1, args.steps),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "tokens": wl.batch.total_tokens, "layers": wl.n_layers},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--cfg", type=int, default=1)
+    ap.add_argument("--impl", default="purekv")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
+
+    from paper_2510_25600_b200 import inputs
+    wl = inputs.workload(args.cfg)
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2510_25600_b200 import binding as P
+    from paper_2510_25600_b200.pipeline import PureKVPipeline
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks, peak_kind = load_peaks()
+
+    # ---- inputs: generated on the host from the seed, then resident in HBM -------------------------------
+    b = wl.batch
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    kv_layers = max(wl.n_layers, wl.compacted_layers[-1] + 1)
+    pipe = PureKVPipeline(b.seq_lens, b.n_prefix, b.n_frames, wl.mask, wl.n_layers, wl.n_q_heads, wl.n_kv_heads,
+                          wl.head_dim, tdt, wl.scored_layers, wl.compacted_layers, wl.window, wl.keep_ratio, kv_layers)
+    (hq, hk, hv), h_out = pipe.alloc_host_io()
+    pool = ThreadPoolExecutor(len(os.sched_getaffinity(0)))
+    keep_for_oracle = []
+    for layer in range(kv_layers):
+        x = inputs.make_qkv(wl, layer, which="qkv" if layer < wl.n_layers else "kv", pool=pool)
+        key = "_bits" if wl.dtype == "bf16" else ""
+        view = (lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)) if wl.dtype == "bf16" else torch.from_numpy
+        if layer < wl.n_layers:
+            hq[layer].copy_(view(x["q" + key]))
+        hk[layer].copy_(view(x["k" + key]))
+        hv[layer].copy_(view(x["v" + key]))
+        if layer < 2:
+            keep_for_oracle.append(x)
+    d_in = tuple(t.cuda() for t in (hq, hk, hv))
+    torch.cuda.synchronize()
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing ---------------------------------------------------------------------------
+    events = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(wl.n_layers)]
+              for _ in range(args.steps)]
+    for _ in range(args.warmup):
+        pipe.run_device(*d_in)
+    pipe.check_status()
+    sampler = ClockSampler(local)
+    sampler.start()
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for s in range(args.steps):
+        pipe.run_device(*d_in, events=events[s])
+    e1.record()
+    sync_all()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    pipe.check_status()
+    t_max = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t_max, op=dist.ReduceOp.MAX)
+    ms_step = float(t_max.item()) / args.steps
+    tokens = b.total_tokens
+    value = world * tokens / (ms_step * 1e-3)
+
+    # ---- roofline of the dominant kernel (tensor-core prefill), from events around each launch -------------
+    info_d, info_s = pipe.plan_dense.info, pipe.plan_st.info
+    n_dense = pipe.clie + 1
+    flops_tile = 4.0 * info_s.tile_q * info_s.tile_k * wl.head_dim * wl.n_q_heads
+    flops_step = flops_tile * (n_dense * info_d.tiles_kept + (wl.n_layers - n_dense) * info_s.tiles_kept)
+    k_ms = np.array([[ev[0].elapsed_time(ev[1]) for ev in step] for step in events])      # [steps, layers]
+    prefill_ms_step = float(k_ms.sum(axis=1).mean())
+    achieved = flops_step / (prefill_ms_step * 1e-3) / 1e12
+    peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
+    roofline = {"kernel": f"prefill_tc_kernel<{info_s.tile_k}>", "bound": "tensor", "achieved": achieved, "peak": peak,
+                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                "peak_kind": f"{peak_kind} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']}, nominal dense 2250)",
+                "flops_per_step": flops_step, "launches_per_step": wl.n_layers, "avg_launch_ms": prefill_ms_step / wl.n_layers,
+                "st_layer_ms": float(k_ms[:, n_dense:].mean()) if wl.n_layers > n_dense else None,
+                "dense_layer_ms": float(k_ms[:, :n_dense].mean()),
+                "tiles_kept_st": info_s.tiles_kept, "tiles_causal": info_s.tiles_causal,
+                "useful_flops_per_step": 4.0 * wl.head_dim * wl.n_q_heads *
+                (n_dense * info_d.pairs_kept + (wl.n_layers - n_dense) * info_s.pairs_kept)}
+
+    # ---- per-step breakdown of the HBM-bound steps (separately timed, cold L2: inputs exceed L2) -----------
+    def time_call(fn, reps=5):
+        out = []
+        for _ in range(reps):
+            flush.zero_()
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            c.record()
+            torch.cuda.synchronize()
+            out.append(a.elapsed_time(c))
+        return float(np.median(out))
+
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    q, k, v = d_in
+    esz = 2 if wl.dtype == "bf16" else 4
+    lo, hi = pipe.compacted[0], pipe.compacted[-1] + 1
+    nc = hi - lo
+    sl = pipe.scored[-1]
+    t_score = time_call(lambda: P.purekv_lowlayer_score(q[sl], k[sl], pipe.batch, wl.window, c_out=pipe.c[0], ws=pipe.score_ws))
+    t_select = time_call(lambda: P.purekv_select_topk(pipe.c[len(pipe.scored) - 1], v[lo:hi], pipe.batch, pipe.budget,
+                                                      idx_out=pipe.idx, ws=pipe.select_ws))
+    t_compact = time_call(lambda: P.purekv_compact_kv(k[lo:hi], v[lo:hi], pipe.idx, pipe.batch, pipe.budget,
+                                                      k_out=pipe.k_c, v_out=pipe.v_c))
+    t_plan = time.perf_counter()
+    pipe.build_plans()
+    t_plan = (time.perf_counter() - t_plan) * 1e3
+    row = wl.n_kv_heads * wl.head_dim * esz
+    kt = pipe.budget.total_kept
+    bytes_score = tokens * row + min(wl.window, tokens) * wl.n_q_heads * wl.head_dim * esz * b.n_req + wl.n_kv_heads * tokens * 4
+    bytes_select = nc * (tokens * row + wl.n_kv_heads * tokens * 4 + wl.n_kv_heads * kt * 4)
+    bytes_compact = nc * (4 * kt * row + wl.n_kv_heads * kt * 4)
+    hbm = float(peaks["hbm_gbs"])
+    steps_detail = {
+        "plan_build_ms": t_plan,
+        "score": {"ms": t_score, "GBps": bytes_score / t_score / 1e6, "frac_hbm": bytes_score / t_score / 1e6 / hbm},
+        "select": {"ms": t_select, "GBps": bytes_select / t_select / 1e6, "frac_hbm": bytes_select / t_select / 1e6 / hbm},
+        "compact": {"ms": t_compact, "GBps": bytes_compact / t_compact / 1e6, "frac_hbm": bytes_compact / t_compact / 1e6 / hbm},
+        "hbm_peak_GBps": hbm, "hbm_peak_kind": peak_kind, "timing": "cold L2 (256 MiB flush before each call), median of 5",
+    }
+
+    # ---- end to end: pinned host inputs, compact cache read back ---------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        n_e2e = max(3, min(args.steps, 10))
+        pipe.run_host((hq, hk, hv), h_out, d_in)
+        sync_all()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            pipe.run_host((hq, hk, hv), h_out, d_in)
+        sync_all()
+        dt = time.perf_counter() - t0
+        t_e = torch.tensor([dt], dtype=torch.float64, device="cuda")
+        if world > 1:
+            dist.all_reduce(t_e, op=dist.ReduceOp.MAX)
+        h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
+        d2h = sum(t.numel() * t.element_size() for t in h_out)
+        e2e = {"value": world * tokens / (float(t_e.item()) / n_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": 1e3 * float(t_e.item()) / n_e2e}
+    pipe.check_status()
+
+    # ---- the oracle on this machine's host cores (rank 0, N = 1 only) ---------------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import purekv_oracle as po
+        po.build()
+        v_cpu, cores, desc, _ = oracle_sample(wl, keep_for_oracle)
+        cpu = {"value": v_cpu, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+                "config": {"workload": wl.name, "tokens": tokens, "layers": wl.n_layers, "heads": [wl.n_q_heads, wl.n_kv_heads],
+                           "head_dim": wl.head_dim, "tile": wl.mask.tile, "window": wl.window, "keep_ratio": wl.keep_ratio,
+                           "l2": "inputs larger than L2 (each layer reads its own Q/K/V; %.0f MB per step)" %
+                                 (sum(t.numel() * t.element_size() for t in d_in) / 1e6),
+                           "multi_gpu": "replicas only (the path has no exchange step)",
+                           "step": "plan build + %d prefill layers + score + select + compact" % wl.n_layers},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": pipe.launches_per_step * args.steps,
+                "roofline": roofline, "cpu_baseline": cpu, "steps_detail": steps_detail}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

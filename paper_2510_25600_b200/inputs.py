@@ -199,7 +199,7 @@ def salient_directions(seed: int, layer: int, n_kv_heads: int, head_dim: int) ->
     return z / np.sqrt((z * z).sum(axis=1, keepdims=True))
 
 
-_CHUNK_TOKENS = 1 << 11
+_CHUNK_TOKENS = 1 << 8
 
 
 def _draw(key: np.uint64, t0: int, t1: int, n_heads: int, d: int) -> np.ndarray:

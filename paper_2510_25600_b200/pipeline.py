@@ -1,0 +1,108 @@
+"""One pass of the PureKV hot path over a batch: the sequence of C-ABI calls a caller makes.
+
+    layers <= CLIE layer : dense causal prefill; the CLIE layer also yields the window scores C
+    higher layers        : ST-SpAttn prefill
+    then                 : V-norm weighting + top-h selection and K/V compaction of the
+                           compressed layers
+
+This module only sequences calls of `binding` and owns the device buffers (torch); it does
+no arithmetic of the method.  `run_host` is the end-to-end form: inputs start in pinned host
+memory and the compact cache is read back to the host.
+"""
+from __future__ import annotations
+
+from typing import Optional, Sequence
+
+import torch
+
+from . import binding as P
+
+
+class PureKVPipeline:
+    def __init__(self, seq_lens: Sequence[int], n_prefix: Sequence[int], n_frames: Sequence[int], mask,
+                 n_layers: int, n_q_heads: int, n_kv_heads: int, head_dim: int, dtype: torch.dtype,
+                 scored_layers: Sequence[int], compacted_layers: Sequence[int], window: int, keep_ratio: float,
+                 kv_layers: Optional[int] = None):
+        """`mask` has the STMask attributes.  Layers up to max(scored_layers) run dense causal attention,
+        the rest ST-SpAttn.  K/V exist for kv_layers >= n_layers layers (default n_layers)."""
+        self.mask, self.n_layers = mask, n_layers
+        self.h, self.hkv, self.d, self.dtype = n_q_heads, n_kv_heads, head_dim, dtype
+        self.code = P.BF16 if dtype == torch.bfloat16 else P.FP32
+        self.clie = max(scored_layers)
+        self.scored = tuple(scored_layers)
+        self.compacted = tuple(compacted_layers)
+        assert self.compacted == tuple(range(self.compacted[0], self.compacted[-1] + 1)), "compacted layers must be contiguous"
+        self.kv_layers = kv_layers if kv_layers is not None else max(n_layers, self.compacted[-1] + 1)
+        self.window, self.keep_ratio = window, keep_ratio
+        self.batch = P.Batch(seq_lens, n_prefix, n_frames)
+        self.budget = P.Budget(self.batch, window, keep_ratio)
+        t = self.batch.total_tokens
+        dev = "cuda"
+        params_dense = P.st_params(mask)
+        params_dense.flags |= P.FLAG_DENSE_CAUSAL
+        self.params_dense, self.params_st = params_dense, P.st_params(mask)
+        self.plan_buf_dense = torch.empty(max(1, P.purekv_plan_bytes(self.batch, params_dense, self.code, head_dim)),
+                                          dtype=torch.uint8, device=dev)
+        self.plan_buf_st = torch.empty(max(1, P.purekv_plan_bytes(self.batch, self.params_st, self.code, head_dim)),
+                                       dtype=torch.uint8, device=dev)
+        self.o = torch.empty((n_layers, t, n_q_heads, head_dim), dtype=dtype, device=dev)
+        self.c = torch.empty((len(self.scored), n_kv_heads, t), dtype=torch.float32, device=dev)
+        self.score_ws = torch.empty(P.purekv_score_ws_bytes(self.batch, window, n_q_heads), dtype=torch.uint8, device=dev)
+        nc = len(self.compacted)
+        self.select_ws = torch.empty(P.purekv_select_ws_bytes(self.batch, nc, n_kv_heads), dtype=torch.uint8, device=dev)
+        self.idx = torch.empty((nc, n_kv_heads, self.budget.total_kept), dtype=torch.int32, device=dev)
+        self.k_c = torch.empty((nc, self.budget.total_kept, n_kv_heads, head_dim), dtype=dtype, device=dev)
+        self.v_c = torch.empty_like(self.k_c)
+        self.status = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.plan_dense = self.plan_st = None
+        self.launches_per_step = n_layers + 2 * len(self.scored) + 2 + 1   # prefill, score (2 kernels), select (2), compact
+
+    def build_plans(self) -> None:
+        self.plan_dense = P.purekv_plan_build(self.batch, self.params_dense, self.code, self.d, self.plan_buf_dense)
+        self.plan_st = P.purekv_plan_build(self.batch, self.params_st, self.code, self.d, self.plan_buf_st)
+
+    def prefill_layer(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor) -> None:
+        plan = self.plan_dense if layer <= self.clie else self.plan_st
+        P.purekv_st_sparse_prefill(q, k, v, self.batch, plan, out=self.o[layer], status=self.status)
+
+    def run_device(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, events=None) -> None:
+        """q [n_layers,T,H,d], k,v [kv_layers,T,H_kv,d] on the GPU.  Results in self.o / idx / k_c / v_c.
+        `events`, if given, is a list of (start, end) torch.cuda.Event pairs, one per prefill launch."""
+        self.build_plans()
+        for layer in range(self.n_layers):
+            if events is not None:
+                events[layer][0].record()
+            self.prefill_layer(layer, q[layer], k[layer], v[layer])
+            if events is not None:
+                events[layer][1].record()
+        for n, layer in enumerate(self.scored):
+            P.purekv_lowlayer_score(q[layer], k[layer], self.batch, self.window, c_out=self.c[n], ws=self.score_ws)
+        lo, hi = self.compacted[0], self.compacted[-1] + 1
+        P.purekv_select_topk(self.c[len(self.scored) - 1], v[lo:hi], self.batch, self.budget, idx_out=self.idx,
+                             ws=self.select_ws)
+        P.purekv_compact_kv(k[lo:hi], v[lo:hi], self.idx, self.batch, self.budget, k_out=self.k_c, v_out=self.v_c)
+
+    def alloc_host_io(self):
+        """Pinned host buffers for run_host: (q, k, v) inputs and (k_c, v_c, o_last) outputs."""
+        t = self.batch.total_tokens
+        pin = dict(dtype=self.dtype, pin_memory=True)
+        ins = (torch.empty((self.n_layers, t, self.h, self.d), **pin),
+               torch.empty((self.kv_layers, t, self.hkv, self.d), **pin),
+               torch.empty((self.kv_layers, t, self.hkv, self.d), **pin))
+        outs = (torch.empty(tuple(self.k_c.shape), **pin), torch.empty(tuple(self.v_c.shape), **pin),
+                torch.empty((t, self.h, self.d), **pin))
+        return ins, outs
+
+    def run_host(self, h_in, h_out, d_in) -> None:
+        """End to end: pinned host Q/K/V -> device (d_in, caller-owned staging) -> hot path -> compact cache and
+        the last layer's O back in pinned host memory.  Synchronises before returning."""
+        for src, dst in zip(h_in, d_in):
+            dst.copy_(src, non_blocking=True)
+        self.run_device(*d_in)
+        h_out[0].copy_(self.k_c, non_blocking=True)
+        h_out[1].copy_(self.v_c, non_blocking=True)
+        h_out[2].copy_(self.o[self.n_layers - 1], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    def check_status(self) -> None:
+        P.purekv_poll_status(self.status)
