@@ -39,9 +39,9 @@ __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 
 // ---- plan buffer layout (device memory, written by purekv_plan_build) -------------------
-// [PlanHeader][QTile x n_qtiles][order int32 x n_qtiles][entries int32 x n_entries][meta int2 x T]
+// [PlanHeader][QTile x n_qtiles][order int32 x n_qtiles][entries int2 x n_entries][masks uint32 x n_mask_words]
 // all sections 16-byte aligned.
-constexpr uint32_t kPlanMagic = 0x504B5631u;  // "PKV1"
+constexpr uint32_t kPlanMagic = 0x504B5632u;  // "PKV2"
 
 enum TileClass : int32_t { kTileFull = 0, kTileDiag = 1, kTileGeneral = 2 };
 
@@ -51,11 +51,10 @@ struct PlanHeader {
   int32_t n_qtiles;
   int64_t total_tokens;
   int64_t n_entries;
-  int64_t off_qtiles, off_order, off_entries, off_meta;  // byte offsets from the plan base
-  // mask parameters the kernels evaluate for general tiles
-  int32_t anchor_frames, spatial_radius, temporal_depth, temporal_stride, temporal_radius;
-  int32_t dense_causal;
-  int32_t pad[2];
+  int64_t n_mask_words;
+  int64_t off_qtiles, off_order, off_entries, off_masks;  // byte offsets from the plan base
+  int32_t words_per_row;                                  // max(1, tile_k / 32)
+  int32_t pad[3];
 };
 
 struct QTile {
@@ -67,35 +66,10 @@ struct QTile {
   int32_t entry_count;
   int32_t pad[2];
 };
-// entry = (key tile index inside the request << 2) | TileClass;  key tile kt covers request
+// entry.x = (key tile index inside the request << 2) | TileClass;  key tile kt covers request
 // positions kt*tile_k .. kt*tile_k + tile_k - 1.
-
-// Per-token coordinates, int2:  x = kind | frame << 2 | (frame mod stride) << 17,  y = gy | gx << 16
-// kind: 0 prefix text, 1 visual, 2 suffix text.
-__host__ __device__ __forceinline__ int meta_kind(int mx) { return mx & 3; }
-__host__ __device__ __forceinline__ int meta_frame(int mx) { return (mx >> 2) & 0x7FFF; }
-__host__ __device__ __forceinline__ int meta_fmod(int mx) { return (mx >> 17) & 0x7FFF; }
-__host__ __device__ __forceinline__ int meta_gy(int my) { return my & 0xFFFF; }
-__host__ __device__ __forceinline__ int meta_gx(int my) { return (my >> 16) & 0xFFFF; }
-
-struct MaskConsts {
-  int32_t anchor_frames, spatial_radius, temporal_depth, temporal_stride, temporal_radius;
-};
-
-// Token-level mask of Sec. 3.2 for request-relative positions j <= i is checked by the caller.
-// qm/km are the per-token coordinates of the query and the key.
-__host__ __device__ __forceinline__ bool st_keep(const MaskConsts& mc, int2 qm, int2 km) {
-  if (meta_kind(qm.x) != 1) return true;   // text query: dense
-  if (meta_kind(km.x) == 0) return true;   // prefix key
-  const int fq = meta_frame(qm.x), fk = meta_frame(km.x);
-  if (fk < mc.anchor_frames) return true;  // first frame(s)
-  const int dy = abs(meta_gy(qm.y) - meta_gy(km.y)), dx = abs(meta_gx(qm.y) - meta_gx(km.y));
-  const int rho = dy > dx ? dy : dx;
-  const int df = fq - fk;
-  if (df == 0) return mc.spatial_radius < 0 || rho <= mc.spatial_radius;   // current frame
-  const bool linked = meta_fmod(qm.x) == meta_fmod(km.x) &&
-                      (mc.temporal_depth < 0 || df <= mc.temporal_depth * mc.temporal_stride);
-  return linked && (mc.temporal_radius < 0 || rho <= mc.temporal_radius);  // previous frame(s)
-}
+// entry.y = for a general tile, the index of its first mask word: row r of the query tile owns
+// words [entry.y + r*words_per_row, +words_per_row), bit c of word w = key 32*w + c of the tile
+// (causality already applied; rows past q_rows are zero); -1 otherwise.
 
 }  // namespace purekv

@@ -2,10 +2,11 @@
 // parameters into per-query-tile lists of kept key tiles, each classified as
 //   full    -- every (row, key) pair of the tile is kept: no predicate in the kernel,
 //   diag    -- exactly the causal pairs j <= i are kept: only the causal compare,
-//   general -- the token predicate is evaluated.
+//   general -- the kernel reads a bit mask (one bit per row and key) stored in the plan.
 // Work per query tile is O(rows x intervals): each row's kept keys are a union of a few
 // position intervals (prefix + first frames, spans of the current frame, spans or single cells
-// of linked earlier frames), accumulated into per-key-tile pair counts.
+// of linked earlier frames), accumulated into per-key-tile pair counts; general tiles get their
+// bits from the same intervals.  The kernels therefore never evaluate the mask's definition.
 #include <algorithm>
 #include <cstring>
 #include <string>
@@ -72,18 +73,6 @@ static purekv_status check_params(const purekv_batch* b, const purekv_st_params*
   return PUREKV_OK;
 }
 
-static void layout(const purekv_batch* b, int tile_q, int tile_k, int64_t* n_qtiles, int64_t* max_entries) {
-  int64_t nq = 0, ne = 0;
-  for (int r = 0; r < b->n_req; ++r) {
-    const int64_t len = b->h_cu_seqlens[r + 1] - b->h_cu_seqlens[r];
-    const int64_t q = (len + tile_q - 1) / tile_q;
-    nq += q;
-    for (int64_t t = 0; t < q; ++t) ne += (std::min(len, (t + 1) * tile_q) + tile_k - 1) / tile_k;
-  }
-  *n_qtiles = nq;
-  *max_entries = ne;
-}
-
 struct Span { int32_t a, b; };  // inclusive request-relative positions
 
 }  // namespace purekv
@@ -112,63 +101,43 @@ purekv_status purekv_budget(int32_t len, int32_t window, double keep_ratio, int3
   return PUREKV_OK;
 }
 
-size_t purekv_plan_bytes(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype, int32_t head_dim) {
-  int tq, tk;
-  if (check_params(b, p, dtype, head_dim, &tq, &tk) != PUREKV_OK) return 0;
-  int64_t nq, ne;
-  layout(b, tq, tk, &nq, &ne);
-  return (size_t)(align16(sizeof(PlanHeader)) + align16(nq * (int64_t)sizeof(QTile)) + align16(nq * 4) +
-                  align16(ne * 4) + align16(b->total_tokens * 8) + 64);
-}
-
 static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
-                                int32_t head_dim, size_t plan_bytes, purekv_plan_info* info,
-                                std::vector<uint8_t>& host) {
+                                int32_t head_dim, purekv_plan_info* info, std::vector<uint8_t>& host) {
   int tq, tk;
   purekv_status st = check_params(b, p, dtype, head_dim, &tq, &tk);
   if (st != PUREKV_OK) return st;
   PK_REQUIRE(info, PUREKV_ERR_INVALID_ARG, "info is null");
-  PK_REQUIRE(plan_bytes >= purekv_plan_bytes(b, p, dtype, head_dim), PUREKV_ERR_WORKSPACE,
-             "plan buffer of %zu bytes is smaller than purekv_plan_bytes", plan_bytes);
   const bool dense = (p->flags & PUREKV_FLAG_DENSE_CAUSAL) != 0;
   const int32_t gw = p->grid_w, gh = p->grid_h, n = gw * gh;
   const int64_t T = b->total_tokens;
+  const int32_t wpr = std::max(1, tk / 32);  // mask words per row of a general tile
 
-  int64_t nq_tot, ne_max;
-  layout(b, tq, tk, &nq_tot, &ne_max);
   std::vector<QTile> qtiles;
-  qtiles.reserve((size_t)nq_tot);
-  std::vector<int32_t> entries;
-  entries.reserve((size_t)ne_max);
-  std::vector<int2> meta((size_t)T);
+  std::vector<int2> entries;
+  std::vector<uint32_t> masks;
   memset(info, 0, sizeof(*info));
 
   std::vector<int64_t> cnt, diff;
-  std::vector<Span> spans;
+  std::vector<Span> spans, row_spans;
+  std::vector<int32_t> row_off;
   for (int r = 0; r < b->n_req; ++r) {
     const int32_t base = b->h_cu_seqlens[r];
     const int32_t len = b->h_cu_seqlens[r + 1] - base;
     const int32_t npre = b->h_n_prefix[r], nfr = b->h_n_frames[r];
     const int32_t vis_end = npre + nfr * n;
-    for (int32_t i = 0; i < len; ++i) {
-      int2 m;
-      if (i < npre) m = make_int2(0, 0);
-      else if (i >= vis_end) m = make_int2(2, 0);
-      else {
-        const int32_t f = (i - npre) / n, c = (i - npre) % n;
-        m = make_int2(1 | (f << 2) | ((f % p->temporal_stride) << 17), (c / gw) | ((c % gw) << 16));
-      }
-      meta[(size_t)base + i] = m;
-    }
     const int32_t nkt = (len + tk - 1) / tk;
     cnt.assign((size_t)nkt + 1, 0);
     diff.assign((size_t)nkt + 2, 0);
-    const int32_t anchor_end = std::min<int64_t>(vis_end, npre + (int64_t)p->anchor_frames * n);  // exclusive
+    const int32_t anchor_end = (int32_t)std::min<int64_t>(vis_end, npre + (int64_t)p->anchor_frames * n);  // exclusive
     for (int32_t q0 = 0; q0 < len; q0 += tq) {
       const int32_t q1 = std::min(len, q0 + tq);  // exclusive
-      std::fill(cnt.begin(), cnt.end(), 0);
-      std::fill(diff.begin(), diff.end(), 0);
+      const int32_t kt_hi = (q1 - 1) / tk;        // last key tile a causal mask reaches
+      std::fill(cnt.begin(), cnt.begin() + kt_hi + 1, 0);
+      std::fill(diff.begin(), diff.begin() + kt_hi + 2, 0);
+      row_spans.clear();
+      row_off.assign(1, 0);
       auto add_span = [&](int32_t a, int32_t bb) {  // inclusive, a <= bb
+        row_spans.push_back({a, bb});
         const int32_t ta = a / tk, tb = bb / tk;
         if (ta == tb) { cnt[ta] += bb - a + 1; return; }
         cnt[ta] += (ta + 1) * tk - a;
@@ -176,39 +145,46 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
         diff[ta + 1] += tk;
         diff[tb] -= tk;
       };
+      // each row's kept keys as disjoint ascending spans (Sec. 3.2)
       for (int32_t i = q0; i < q1; ++i) {
         const bool visual = i >= npre && i < vis_end;
-        if (dense || !visual) { add_span(0, i); continue; }
-        spans.clear();
-        if (anchor_end > 0) spans.push_back({0, std::min(i, anchor_end - 1)});  // prefix + first frames
-        const int32_t f = (i - npre) / n, c = (i - npre) % n, y = c / gw, x = c % gw;
-        const int32_t fs = npre + f * n;
-        if (p->spatial_radius < 0) spans.push_back({fs, i});
-        else {
-          const int32_t rr = p->spatial_radius;
-          for (int32_t yy = std::max(0, y - rr); yy <= y; ++yy) {
-            const int32_t xa = std::max(0, x - rr), xb = yy == y ? x : std::min(gw - 1, x + rr);
-            spans.push_back({fs + yy * gw + xa, fs + yy * gw + xb});
+        if (dense || !visual) {
+          add_span(0, i);  // text rows and the dense mask: plain causal
+        } else {
+          spans.clear();
+          if (anchor_end > 0) spans.push_back({0, std::min(i, anchor_end - 1)});  // prefix + first frame(s)
+          const int32_t f = (i - npre) / n, c = (i - npre) % n, y = c / gw, x = c % gw;
+          const int32_t fs = npre + f * n;
+          if (p->spatial_radius < 0) {
+            spans.push_back({fs, i});  // the current frame, causal
+          } else {
+            const int32_t rr = p->spatial_radius;
+            for (int32_t yy = std::max(0, y - rr); yy <= y; ++yy) {
+              const int32_t xa = std::max(0, x - rr), xb = yy == y ? x : std::min(gw - 1, x + rr);
+              spans.push_back({fs + yy * gw + xa, fs + yy * gw + xb});
+            }
           }
-        }
-        for (int32_t m = 1;; ++m) {
-          const int64_t fj = (int64_t)f - (int64_t)m * p->temporal_stride;
-          if (fj < 0 || (p->temporal_depth >= 0 && m > p->temporal_depth)) break;
-          const int32_t fjs = npre + (int32_t)fj * n;
-          if (p->temporal_radius < 0) spans.push_back({fjs, fjs + n - 1});
-          else {
-            const int32_t rr = p->temporal_radius;
-            for (int32_t yy = std::max(0, y - rr); yy <= std::min(gh - 1, y + rr); ++yy)
-              spans.push_back({fjs + yy * gw + std::max(0, x - rr), fjs + yy * gw + std::min(gw - 1, x + rr)});
+          for (int32_t m = 1;; ++m) {  // linked earlier frames: the corresponding cell (or a window / the frame)
+            const int64_t fj = (int64_t)f - (int64_t)m * p->temporal_stride;
+            if (fj < 0 || (p->temporal_depth >= 0 && m > p->temporal_depth)) break;
+            const int32_t fjs = npre + (int32_t)fj * n;
+            if (p->temporal_radius < 0) {
+              spans.push_back({fjs, fjs + n - 1});
+            } else {
+              const int32_t rr = p->temporal_radius;
+              for (int32_t yy = std::max(0, y - rr); yy <= std::min(gh - 1, y + rr); ++yy)
+                spans.push_back({fjs + yy * gw + std::max(0, x - rr), fjs + yy * gw + std::min(gw - 1, x + rr)});
+            }
           }
+          std::sort(spans.begin(), spans.end(), [](const Span& u, const Span& v) { return u.a < v.a; });
+          int32_t ca = spans[0].a, cb = spans[0].b;
+          for (size_t s = 1; s < spans.size(); ++s) {
+            if (spans[s].a <= cb + 1) cb = std::max(cb, spans[s].b);
+            else { add_span(ca, cb); ca = spans[s].a; cb = spans[s].b; }
+          }
+          add_span(ca, cb);
         }
-        std::sort(spans.begin(), spans.end(), [](const Span& u, const Span& v) { return u.a < v.a; });
-        int32_t ca = spans[0].a, cb = spans[0].b;
-        for (size_t s = 1; s < spans.size(); ++s) {
-          if (spans[s].a <= cb + 1) cb = std::max(cb, spans[s].b);
-          else { add_span(ca, cb); ca = spans[s].a; cb = spans[s].b; }
-        }
-        add_span(ca, cb);
+        row_off.push_back((int32_t)row_spans.size());
       }
       QTile qt;
       qt.q_start = base + q0;
@@ -218,7 +194,6 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
       qt.entry_begin = (int32_t)entries.size();
       qt.pad[0] = qt.pad[1] = 0;
       int64_t run = 0;
-      const int32_t kt_hi = (q1 - 1) / tk;  // last key tile a causal mask reaches
       for (int32_t kt = 0; kt <= kt_hi; ++kt) {
         run += diff[kt];
         const int64_t c = cnt[kt] + run;
@@ -231,10 +206,29 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
           causal = 0;
           for (int32_t i = q0; i < q1; ++i) causal += std::max(0, std::min(tk, i - j0 + 1));
         }
-        int32_t cls = kTileGeneral;
+        int32_t cls = kTileGeneral, mask_at = -1;
         if (c == full && j0 + tk <= len) cls = kTileFull;
         else if (c == causal) cls = kTileDiag;
-        entries.push_back((kt << 2) | cls);
+        if (cls == kTileGeneral) {
+          // one bit per (row, key) of the tile, rows past q_rows stay zero
+          PK_REQUIRE(masks.size() + (size_t)tq * wpr < (size_t)INT32_MAX, PUREKV_ERR_UNSUPPORTED,
+                     "mask table exceeds 2^31 words");
+          mask_at = (int32_t)masks.size();
+          masks.resize(masks.size() + (size_t)tq * wpr, 0u);
+          uint32_t* mw = masks.data() + mask_at;
+          for (int32_t i = q0; i < q1; ++i)
+            for (int32_t s = row_off[i - q0]; s < row_off[i - q0 + 1]; ++s) {
+              const int32_t a = std::max(row_spans[s].a, j0), bb = std::min(row_spans[s].b, j0 + tk - 1);
+              if (a > bb) continue;
+              const int32_t lo = a - j0, hi = bb - j0;  // bit range inside the tile row
+              uint32_t* rw = mw + (i - q0) * wpr;
+              for (int32_t w = lo >> 5; w <= (hi >> 5); ++w) {
+                const int32_t b0 = std::max(lo - 32 * w, 0), b1 = std::min(hi - 32 * w, 31);
+                rw[w] |= (b1 - b0 == 31) ? 0xFFFFFFFFu : (((1u << (b1 - b0 + 1)) - 1u) << b0);
+              }
+            }
+        }
+        entries.push_back(make_int2((kt << 2) | cls, mask_at));
         info->pairs_kept += c;
         info->tiles_kept++;
         (cls == kTileFull ? info->tiles_full : cls == kTileDiag ? info->tiles_diag : info->tiles_general)++;
@@ -258,25 +252,20 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   h.n_qtiles = nq;
   h.total_tokens = T;
   h.n_entries = (int64_t)entries.size();
+  h.n_mask_words = (int64_t)masks.size();
+  h.words_per_row = wpr;
   h.off_qtiles = align16(sizeof(PlanHeader));
   h.off_order = h.off_qtiles + align16((int64_t)nq * sizeof(QTile));
   h.off_entries = h.off_order + align16((int64_t)nq * 4);
-  h.off_meta = h.off_entries + align16(h.n_entries * 4);
-  h.anchor_frames = p->anchor_frames;
-  h.spatial_radius = p->spatial_radius;
-  h.temporal_depth = p->temporal_depth;
-  h.temporal_stride = p->temporal_stride;
-  h.temporal_radius = p->temporal_radius;
-  h.dense_causal = dense ? 1 : 0;
-  const int64_t total = h.off_meta + align16(T * 8);
-  PK_REQUIRE((size_t)total <= plan_bytes, PUREKV_ERR_WORKSPACE, "plan needs %lld bytes", (long long)total);
+  h.off_masks = h.off_entries + align16(h.n_entries * 8);
+  const int64_t total = h.off_masks + align16(h.n_mask_words * 4);
 
   host.assign((size_t)total, 0);
   memcpy(host.data(), &h, sizeof(h));
   if (nq) memcpy(host.data() + h.off_qtiles, qtiles.data(), (size_t)nq * sizeof(QTile));
   if (nq) memcpy(host.data() + h.off_order, order.data(), (size_t)nq * 4);
-  if (!entries.empty()) memcpy(host.data() + h.off_entries, entries.data(), entries.size() * 4);
-  if (T) memcpy(host.data() + h.off_meta, meta.data(), (size_t)T * 8);
+  if (!entries.empty()) memcpy(host.data() + h.off_entries, entries.data(), entries.size() * 8);
+  if (!masks.empty()) memcpy(host.data() + h.off_masks, masks.data(), masks.size() * 4);
 
   info->tile_q = tq;
   info->tile_k = tk;
@@ -287,12 +276,21 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   return PUREKV_OK;
 }
 
+size_t purekv_plan_bytes(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype, int32_t head_dim) {
+  purekv_plan_info info;
+  std::vector<uint8_t> host;
+  if (build_plan(b, p, dtype, head_dim, &info, host) != PUREKV_OK) return 0;
+  return host.size();
+}
+
 purekv_status purekv_plan_build_host(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
                                      int32_t head_dim, void* h_plan, size_t plan_bytes, purekv_plan_info* info) {
   PK_REQUIRE(h_plan, PUREKV_ERR_INVALID_ARG, "h_plan is null");
   std::vector<uint8_t> host;
-  purekv_status st = build_plan(b, p, dtype, head_dim, plan_bytes, info, host);
+  purekv_status st = build_plan(b, p, dtype, head_dim, info, host);
   if (st != PUREKV_OK) return st;
+  PK_REQUIRE(host.size() <= plan_bytes, PUREKV_ERR_WORKSPACE, "plan needs %zu bytes, buffer has %zu", host.size(),
+             plan_bytes);
   memcpy(h_plan, host.data(), host.size());
   return PUREKV_OK;
 }
@@ -302,8 +300,10 @@ purekv_status purekv_plan_build(const purekv_batch* b, const purekv_st_params* p
                                 void* stream) {
   PK_REQUIRE(plan, PUREKV_ERR_INVALID_ARG, "plan is null");
   std::vector<uint8_t> host;
-  purekv_status st = build_plan(b, p, dtype, head_dim, plan_bytes, info, host);
+  purekv_status st = build_plan(b, p, dtype, head_dim, info, host);
   if (st != PUREKV_OK) return st;
+  PK_REQUIRE(host.size() <= plan_bytes, PUREKV_ERR_WORKSPACE, "plan needs %zu bytes, buffer has %zu", host.size(),
+             plan_bytes);
   cudaStream_t s = (cudaStream_t)stream;
   PK_CUDA(cudaMemcpyAsync(plan, host.data(), host.size(), cudaMemcpyHostToDevice, s));
   PK_CUDA(cudaStreamSynchronize(s));

@@ -2,7 +2,7 @@
 // fp32 inputs (computed in fp32 throughout) and bf16 with head_dim other than 128.
 //
 // One CTA = one query tile (<= 64 rows) of one query head, walking the plan's list of kept key
-// tiles.  K and V tiles are staged in shared memory as fp32.  A warp owns rows warp, warp+4, ...
+// tiles (general tiles carry a bit mask in the plan).  K and V tiles are staged in shared memory as fp32.  A warp owns rows warp, warp+4, ...
 // of the tile; for a row the lanes split the keys of the tile for q.k, the row's online-softmax
 // state (max, sum, d/32 output values per lane) lives in registers, and probabilities pass
 // through a per-warp shared buffer for the P.V product where the lanes split the head dim.
@@ -26,11 +26,9 @@ __global__ void __launch_bounds__(kSimtThreads) prefill_simt_kernel(
   const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(plan);
   const QTile* qtiles = reinterpret_cast<const QTile*>(plan + hdr->off_qtiles);
   const int32_t* order = reinterpret_cast<const int32_t*>(plan + hdr->off_order);
-  const int32_t* entries = reinterpret_cast<const int32_t*>(plan + hdr->off_entries);
-  const int2* meta = reinterpret_cast<const int2*>(plan + hdr->off_meta);
-  const int32_t tq = hdr->tile_q, tk = hdr->tile_k;
-  const MaskConsts mc{hdr->anchor_frames, hdr->spatial_radius, hdr->temporal_depth, hdr->temporal_stride,
-                      hdr->temporal_radius};
+  const int2* entries = reinterpret_cast<const int2*>(plan + hdr->off_entries);
+  const uint32_t* masks = reinterpret_cast<const uint32_t*>(plan + hdr->off_masks);
+  const int32_t tq = hdr->tile_q, tk = hdr->tile_k, wpr = hdr->words_per_row;
   const QTile qt = qtiles[order[blockIdx.x]];
   const int32_t hq = blockIdx.y, g = hq / (n_q_heads / n_kv_heads);
   const int32_t q_rel0 = qt.q_start - qt.req_start;
@@ -39,7 +37,6 @@ __global__ void __launch_bounds__(kSimtThreads) prefill_simt_kernel(
   float* ks = qs + tq * D;                  // [tk][LD]
   float* vs = ks + tk * LD;                 // [tk][LD]
   float* ps = vs + tk * LD;                 // [warps][tk]
-  int2* kmeta = reinterpret_cast<int2*>(ps + kSimtWarps * tk);  // [tk]
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int x = tid; x < tq * D; x += kSimtThreads) {
@@ -48,20 +45,17 @@ __global__ void __launch_bounds__(kSimtThreads) prefill_simt_kernel(
   }
 
   float m[kMaxRowsPerWarp], l[kMaxRowsPerWarp], acc[kMaxRowsPerWarp][DPL];
-  int2 qm[kMaxRowsPerWarp];
 #pragma unroll
   for (int rr = 0; rr < kMaxRowsPerWarp; ++rr) {
     m[rr] = -INFINITY;
     l[rr] = 0.f;
 #pragma unroll
     for (int c = 0; c < DPL; ++c) acc[rr][c] = 0.f;
-    const int row = warp + kSimtWarps * rr;
-    qm[rr] = row < qt.q_rows ? meta[qt.q_start + row] : make_int2(0, 0);
   }
 
   for (int32_t e = 0; e < qt.entry_count; ++e) {
-    const int32_t ent = entries[qt.entry_begin + e];
-    const int32_t cls = ent & 3, j0 = (ent >> 2) * tk;
+    const int2 ent = entries[qt.entry_begin + e];
+    const int32_t cls = ent.x & 3, j0 = (ent.x >> 2) * tk;
     __syncthreads();
     for (int x = tid; x < tk * D; x += kSimtThreads) {
       const int row = x / D, c = x % D;
@@ -70,9 +64,6 @@ __global__ void __launch_bounds__(kSimtThreads) prefill_simt_kernel(
       ks[row * LD + c] = in ? to_f32(k[src]) : 0.f;
       vs[row * LD + c] = in ? to_f32(v[src]) : 0.f;
     }
-    if (cls == kTileGeneral)
-      for (int x = tid; x < tk; x += kSimtThreads)
-        kmeta[x] = j0 + x < qt.req_len ? meta[qt.req_start + j0 + x] : make_int2(0, 0);
     __syncthreads();
 #pragma unroll
     for (int rr = 0; rr < kMaxRowsPerWarp; ++rr) {
@@ -88,7 +79,7 @@ __global__ void __launch_bounds__(kSimtThreads) prefill_simt_kernel(
         sv[kk] = -INFINITY;
         if (c < tk) {
           bool keep = cls == kTileFull || j0 + c <= i;
-          if (keep && cls == kTileGeneral) keep = st_keep(mc, qm[rr], kmeta[c]);
+          if (cls == kTileGeneral) keep = (__ldg(masks + ent.y + row * wpr + (c >> 5)) >> (c & 31)) & 1u;
           if (keep) {
             float s = 0.f;
             const float* krow = ks + c * LD;
@@ -150,7 +141,7 @@ template <typename T, int DPL>
 static purekv_status launch(const PrefillArgs& a) {
   const int D = 32 * DPL;
   const size_t smem = ((size_t)a.info->tile_q * D + 2 * (size_t)a.info->tile_k * (D + 1) +
-                       (size_t)kSimtWarps * a.info->tile_k) * sizeof(float) + (size_t)a.info->tile_k * sizeof(int2);
+                       (size_t)kSimtWarps * a.info->tile_k) * sizeof(float);
   PK_REQUIRE(smem <= 227 * 1024, PUREKV_ERR_UNSUPPORTED,
              "head_dim %d with tile %d needs %zu bytes of shared memory", D, a.info->tile_k, smem);
   PK_CUDA(cudaFuncSetAttribute(prefill_simt_kernel<T, DPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

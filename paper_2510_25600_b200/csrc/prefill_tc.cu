@@ -1,16 +1,18 @@
 // Tensor-core ST-SpAttn prefill (Sec. 3.2) for bf16, head_dim 128, on sm_100a.
 //
-// One CTA = one 128-row query tile of one query head; it walks the plan's list of kept key
-// tiles, so key blocks the mask removes are never read.  Roles:
-//   warp 0      TMA producer: Q once, then K and V tiles (128B-swizzled, two 64-column panels
-//               each) into a 2-stage ring; only kept tiles are requested from HBM/L2.
-//   warp 1      owns the 512 TMEM columns; one lane issues tcgen05.mma:
-//               S[b] = Q K^T (K-major A and B from shared memory) and
-//               O   += P[b] V (A = bf16 P from TMEM, B = V as MN-major shared-memory operand).
-//   warps 2-5   one thread per query row: read S from TMEM, apply the tile's predicate class
-//               (full / causal / general token predicate), online softmax in the log2 domain
-//               with lazy rescaling of O, write bf16 P back to TMEM, final normalise + store.
-// TMEM columns: S0 [0,128) S1 [128,256) O [256,384) P0 [384,448) P1 [448,512).
+// One CTA = one 128-row query tile of a PAIR of query heads that share a KV head ("slots"), so
+// every K/V tile staged in shared memory feeds two heads.  It walks the plan's list of kept key
+// tiles: key blocks the mask removes are never read.  Roles:
+//   warp 0      TMA producer: Q of both slots once, then K and V tiles (128B-swizzled, two
+//               64-column panels each) into a ring of stages.
+//   warp 1      owns the 512 TMEM columns; one lane issues tcgen05.mma, alternating slots:
+//               S = Q K^T (K-major A and B from shared memory) and
+//               O += P V (A = bf16 P from TMEM, B = V as MN-major shared-memory operand),
+//               so the tensor pipe works on one slot while the other slot's rows are in softmax.
+//   warps 2-9   one thread per query row of a slot: the row of S from TMEM into registers, the
+//               tile's predicate class (full / causal / bit mask from the plan), online softmax in
+//               the log2 domain with lazy rescaling of O, bf16 P written over S, final normalise
+//               and store.
 // Every wait on an mbarrier is bounded in time; on expiry the CTA raises a shared abort flag,
 // sets the device status word, drains, frees TMEM and exits.
 #include <cuda.h>
@@ -22,10 +24,9 @@ namespace tc {
 
 constexpr int kD = 128;
 constexpr int kBQ = 128;
-constexpr int kStages = 2;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 softmax of slot 0, warps 6-9 of slot 1
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256, kColP = 384;
+constexpr uint32_t kColO = 256;
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
 constexpr float kRescaleThreshold = 8.0f;                        // log2 units
 
@@ -56,15 +57,18 @@ __device__ __forceinline__ uint64_t global_ns() {
   return t;
 }
 // Bounded wait: false if the abort flag is up or the time limit passed (then raises the flag).
+// The wall-clock timer is slow to read, so it is consulted only every 1024 failed polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const uint64_t t0 = global_ns();
+  uint64_t t0 = 0;
   uint32_t it = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((++it & 31u) == 0u) {
+    if ((++it & 1023u) == 0u) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      const uint64_t now = global_ns();
+      if (t0 == 0) {
+        t0 = now;
+      } else if (now - t0 > kWaitLimitNs) {
         *abort_flag = 1;
         return false;
       }
@@ -130,6 +134,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
 }
+// Same load into elements OFF .. OFF+31 of a larger register array.
+template <int OFF, int N>
+__device__ __forceinline__ void tmem_ld32_at(uint32_t taddr, uint32_t (&r)[N]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : PK_R8(r, OFF + 0), PK_R8(r, OFF + 8), PK_R8(r, OFF + 16), PK_R8(r, OFF + 24)
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
@@ -168,62 +183,81 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
          ((uint32_t)(128 >> 4) << 24);
 }
 
+template <int BK>
+struct Cfg {
+  static constexpr int kStages = BK == 64 ? 4 : 2;  // K/V ring depth (32 KB resp. 64 KB per stage)
+  static constexpr int kSBuf = BK == 64 ? 2 : 1;    // S buffers per slot: kSBuf * BK = 128 TMEM columns
+};
+
+template <int BK>
 struct __align__(8) Barriers {
+  static constexpr int ST = Cfg<BK>::kStages, SB = Cfg<BK>::kSBuf;
   uint64_t q_full;
-  uint64_t k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  uint64_t s_full[2], p_full[2];
-  uint64_t o_done;   // one completion per P.V product (tile m completes phase m)
-  uint64_t o_final;  // completes once, after the last P.V product
+  uint64_t k_full[ST], k_empty[ST], v_full[ST], v_empty[ST];
+  uint64_t s_full[2][SB];  // MMA -> softmax: S of (slot, buffer) is complete
+  uint64_t p_full[2][SB];  // softmax -> MMA: P written (and O rescaled) by all 128 row threads
+  uint64_t o_done[2];      // one completion per P.V product of the slot
+  uint64_t o_final[2];     // completes once, after the slot's last P.V product
   uint64_t drain;
 };
 
+// TMEM columns: S(slot, buf) at slot*128 + buf*BK (P aliases its first BK/2 columns), O(slot) at 256 + slot*128.
 template <int BK>
 __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
     const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, float* __restrict__ lse,
     const uint8_t* __restrict__ plan, int32_t n_q_heads, int32_t n_kv_heads, float scale_log2,
     int32_t* __restrict__ status) {
-  constexpr uint32_t kPanelQ = kBQ * 128;   // bytes of one 64-column panel of Q
-  constexpr uint32_t kPanelKV = BK * 128;   // bytes of one 64-column panel of a K or V tile
+  constexpr int ST = Cfg<BK>::kStages, SB = Cfg<BK>::kSBuf;
+  constexpr uint32_t kPanelQ = kBQ * 128;  // bytes of one 64-column panel of a Q tile
+  constexpr uint32_t kTileQ = 2 * kPanelQ;
+  constexpr uint32_t kPanelKV = BK * 128;  // bytes of one 64-column panel of a K or V tile
   constexpr uint32_t kTileKV = 2 * kPanelKV;
   extern __shared__ uint8_t smem_raw[];
-  __shared__ Barriers bars;
+  __shared__ Barriers<BK> bars;
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
-  __shared__ int2 kmeta[4][BK];  // per softmax warp: coordinates of the current tile's keys
 
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t sQ = smem0;
-  const uint32_t sK = sQ + 2 * kPanelQ;
-  const uint32_t sV = sK + kStages * kTileKV;
+  const uint32_t sQ = smem0;                 // [2 slots][2 panels][128 rows x 128 B]
+  const uint32_t sK = sQ + 2 * kTileQ;       // [ST][2 panels][BK rows x 128 B]
+  const uint32_t sV = sK + ST * kTileKV;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(plan);
   const QTile* qtiles = reinterpret_cast<const QTile*>(plan + hdr->off_qtiles);
   const int32_t* order = reinterpret_cast<const int32_t*>(plan + hdr->off_order);
-  const int32_t* entries = reinterpret_cast<const int32_t*>(plan + hdr->off_entries);
-  const int2* meta = reinterpret_cast<const int2*>(plan + hdr->off_meta);
-  const QTile qt = qtiles[order[blockIdx.x]];
-  const int32_t hq = blockIdx.y, g = hq / (n_q_heads / n_kv_heads);
+  const int2* entries = reinterpret_cast<const int2*>(plan + hdr->off_entries);
+  const uint32_t* masks = reinterpret_cast<const uint32_t*>(plan + hdr->off_masks);
+  // blockIdx.x = rank of the query tile in the longest-first order * n_pairs + pair, so the long lists of
+  // every head start first.  A pair = (KV head, two of its query heads); the last pair of an odd group is single.
+  const int32_t G = n_q_heads / n_kv_heads, ppg = (G + 1) >> 1, n_pairs = n_kv_heads * ppg;
+  const QTile qt = qtiles[order[blockIdx.x / n_pairs]];
+  const int32_t pair = blockIdx.x % n_pairs;
+  const int32_t g = pair / ppg, pr = pair % ppg;
+  const int32_t hq0 = g * G + 2 * pr;
+  const int32_t n_slots = (2 * pr + 1 < G) ? 2 : 1;
   const int32_t nt = qt.entry_count;
-  const int32_t* ent = entries + qt.entry_begin;
+  const int2* ent = entries + qt.entry_begin;
   volatile int* abort_flag = &abort_s;
 
   if (tid == 0) {
     abort_s = *reinterpret_cast<volatile int32_t*>(status) != 0;  // an earlier CTA already failed
     mbar_init(smem_u32(&bars.q_full), 1);
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < ST; ++s) {
       mbar_init(smem_u32(&bars.k_full[s]), 1);
       mbar_init(smem_u32(&bars.k_empty[s]), 1);
       mbar_init(smem_u32(&bars.v_full[s]), 1);
       mbar_init(smem_u32(&bars.v_empty[s]), 1);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&bars.s_full[b]), 1);
-      mbar_init(smem_u32(&bars.p_full[b]), 128);
+    for (int sl = 0; sl < 2; ++sl) {
+      for (int b = 0; b < SB; ++b) {
+        mbar_init(smem_u32(&bars.s_full[sl][b]), 1);
+        mbar_init(smem_u32(&bars.p_full[sl][b]), 128);
+      }
+      mbar_init(smem_u32(&bars.o_done[sl]), 1);
+      mbar_init(smem_u32(&bars.o_final[sl]), 1);
     }
-    mbar_init(smem_u32(&bars.o_done), 1);
-    mbar_init(smem_u32(&bars.o_final), 1);
     mbar_init(smem_u32(&bars.drain), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -241,20 +275,22 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
   if (start_ok && warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      mbar_expect_tx(smem_u32(&bars.q_full), 2 * kPanelQ);
-      tma_load_3d(sQ, &tm_q, smem_u32(&bars.q_full), 0, hq, qt.q_start);
-      tma_load_3d(sQ + kPanelQ, &tm_q, smem_u32(&bars.q_full), 64, hq, qt.q_start);
+      mbar_expect_tx(smem_u32(&bars.q_full), n_slots * kTileQ);
+      for (int sl = 0; sl < n_slots; ++sl) {
+        tma_load_3d(sQ + sl * kTileQ, &tm_q, smem_u32(&bars.q_full), 0, hq0 + sl, qt.q_start);
+        tma_load_3d(sQ + sl * kTileQ + kPanelQ, &tm_q, smem_u32(&bars.q_full), 64, hq0 + sl, qt.q_start);
+      }
       int32_t issued_k = 0, issued_v = 0;
       for (int32_t n = 0; n < nt; ++n) {
-        const int32_t s = n % kStages;
-        const uint32_t par = ((n / kStages) - 1) & 1;
-        const int32_t tok = qt.req_start + (ent[n] >> 2) * BK;
-        if (n >= kStages && !mbar_wait(smem_u32(&bars.k_empty[s]), par, abort_flag)) break;
+        const int32_t s = n % ST;
+        const uint32_t par = ((n / ST) - 1) & 1;
+        const int32_t tok = qt.req_start + (ent[n].x >> 2) * BK;
+        if (n >= ST && !mbar_wait(smem_u32(&bars.k_empty[s]), par, abort_flag)) break;
         mbar_expect_tx(smem_u32(&bars.k_full[s]), kTileKV);
         tma_load_3d(sK + s * kTileKV, &tm_k, smem_u32(&bars.k_full[s]), 0, g, tok);
         tma_load_3d(sK + s * kTileKV + kPanelKV, &tm_k, smem_u32(&bars.k_full[s]), 64, g, tok);
         issued_k = n + 1;
-        if (n >= kStages && !mbar_wait(smem_u32(&bars.v_empty[s]), par, abort_flag)) break;
+        if (n >= ST && !mbar_wait(smem_u32(&bars.v_empty[s]), par, abort_flag)) break;
         mbar_expect_tx(smem_u32(&bars.v_full[s]), kTileKV);
         tma_load_3d(sV + s * kTileKV, &tm_v, smem_u32(&bars.v_full[s]), 0, g, tok);
         tma_load_3d(sV + s * kTileKV + kPanelKV, &tm_v, smem_u32(&bars.v_full[s]), 64, g, tok);
@@ -263,12 +299,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       if (*abort_flag) {
         // drain: every issued copy must have landed before shared memory is released
         const uint64_t t0 = global_ns();
-        for (int32_t n = max(0, issued_k - kStages); n < issued_k; ++n)
-          while (!mbar_try_wait(smem_u32(&bars.k_full[n % kStages]), (n / kStages) & 1) &&
-                 global_ns() - t0 < kWaitLimitNs) {}
-        for (int32_t n = max(0, issued_v - kStages); n < issued_v; ++n)
-          while (!mbar_try_wait(smem_u32(&bars.v_full[n % kStages]), (n / kStages) & 1) &&
-                 global_ns() - t0 < kWaitLimitNs) {}
+        for (int32_t n = max(0, issued_k - ST); n < issued_k; ++n)
+          while (!mbar_try_wait(smem_u32(&bars.k_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+        for (int32_t n = max(0, issued_v - ST); n < issued_v; ++n)
+          while (!mbar_try_wait(smem_u32(&bars.v_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < kWaitLimitNs) {}
         while (!mbar_try_wait(smem_u32(&bars.q_full), 0) && global_ns() - t0 < kWaitLimitNs) {}
       }
     }
@@ -277,40 +311,48 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(BK, false);
       constexpr uint32_t idesc_pv = instr_desc(kD, true);
-      auto issue_pv = [&](int32_t m) -> bool {
-        const int32_t s = m % kStages, b = m & 1;
-        if (!mbar_wait(smem_u32(&bars.v_full[s]), (m / kStages) & 1, abort_flag)) return false;
-        if (!mbar_wait(smem_u32(&bars.p_full[b]), (m >> 1) & 1, abort_flag)) return false;
+      // S(slot, n) = Q_slot K_n^T; the last slot to read K_n releases its stage
+      auto issue_qk = [&](int32_t sl, int32_t n) -> bool {
+        const int32_t s = n % ST, b = n % SB;
+        if (!mbar_wait(smem_u32(&bars.k_full[s]), (n / ST) & 1, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t p_addr = tmem + kColP + b * 64;
+        const uint32_t d_addr = tmem + sl * 128 + b * BK;
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks) {
+          const uint32_t qoff = sl * kTileQ + (ks >> 2) * kPanelQ + (ks & 3) * 32;
+          const uint32_t koff = s * kTileKV + (ks >> 2) * kPanelKV + (ks & 3) * 32;
+          mma_ss(d_addr, smem_desc(sQ + qoff, 16, 1024), smem_desc(sK + koff, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
+        }
+        if (sl == n_slots - 1) tc_commit(smem_u32(&bars.k_empty[s]));
+        tc_commit(smem_u32(&bars.s_full[sl][b]));
+        return true;
+      };
+      // O(slot) += P(slot, n) V_n; the last slot to read V_n releases its stage
+      auto issue_pv = [&](int32_t sl, int32_t n) -> bool {
+        const int32_t s = n % ST, b = n % SB;
+        if (!mbar_wait(smem_u32(&bars.v_full[s]), (n / ST) & 1, abort_flag)) return false;
+        if (!mbar_wait(smem_u32(&bars.p_full[sl][b]), (n / SB) & 1, abort_flag)) return false;
+        tc_fence_after();
+        const uint32_t p_addr = tmem + sl * 128 + b * BK;
 #pragma unroll
         for (int ks = 0; ks < BK / 16; ++ks) {
           // B = V tile, MN-major: 16 key rows (2 groups of 8, SBO 1024) x 128 dims (2 panels, LBO)
           const uint64_t bdesc = smem_desc(sV + s * kTileKV + ks * 2048, kPanelKV, 1024);
-          mma_ts(tmem + kColO, p_addr + ks * 8, bdesc, idesc_pv, (m > 0 || ks > 0) ? 1u : 0u);
+          mma_ts(tmem + kColO + sl * 128, p_addr + ks * 8, bdesc, idesc_pv, (n > 0 || ks > 0) ? 1u : 0u);
         }
-        tc_commit(smem_u32(&bars.v_empty[s]));
-        tc_commit(smem_u32(&bars.o_done));
+        if (sl == n_slots - 1) tc_commit(smem_u32(&bars.v_empty[s]));
+        tc_commit(smem_u32(&bars.o_done[sl]));
+        if (n == nt - 1) tc_commit(smem_u32(&bars.o_final[sl]));
         return true;
       };
       bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort_flag);
-      for (int32_t n = 0; ok && n < nt; ++n) {
-        const int32_t s = n % kStages, b = n & 1;
-        if (!mbar_wait(smem_u32(&bars.k_full[s]), (n / kStages) & 1, abort_flag)) { ok = false; break; }
-        tc_fence_after();
-#pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-          const uint32_t koff = (ks >> 2) * kPanelQ + (ks & 3) * 32;
-          const uint32_t kboff = (ks >> 2) * kPanelKV + (ks & 3) * 32;
-          mma_ss(tmem + kColS + b * 128, smem_desc(sQ + koff, 16, 1024),
-                 smem_desc(sK + s * kTileKV + kboff, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
+      for (int32_t n = 0; ok && n < SB && n < nt; ++n)
+        for (int32_t sl = 0; ok && sl < n_slots; ++sl) ok = issue_qk(sl, n);
+      for (int32_t n = 0; ok && n < nt; ++n)
+        for (int32_t sl = 0; ok && sl < n_slots; ++sl) {
+          ok = issue_pv(sl, n);
+          if (ok && n + SB < nt) ok = issue_qk(sl, n + SB);  // in order behind P.V of tile n, which frees S(slot, n % SB)
         }
-        tc_commit(smem_u32(&bars.k_empty[s]));
-        tc_commit(smem_u32(&bars.s_full[b]));
-        if (n >= 1 && !issue_pv(n - 1)) { ok = false; break; }
-      }
-      if (ok) ok = issue_pv(nt - 1);
-      if (ok) tc_commit(smem_u32(&bars.o_final));
       if (!ok) {
         // leaving early: let every issued MMA finish before TMEM is released
         tc_commit(smem_u32(&bars.drain));
@@ -318,135 +360,145 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         while (!mbar_try_wait(smem_u32(&bars.drain), 0) && global_ns() - t0 < kWaitLimitNs) {}
       }
     }
-  } else if (start_ok) {
-    // ---------------- softmax / epilogue: one thread per query row ----------------
-    const int quad = warp & 3;            // TMEM lane quadrant this warp may access
+  } else if (start_ok && (warp - 2) / 4 < n_slots) {
+    // ---------------- softmax / epilogue: one thread per query row of one slot ----------------
+    const int sl = (warp - 2) >> 2;
+    const int quad = warp & 3;  // TMEM lane quadrant this warp may access
     const int row = quad * 32 + lane;
-    int2* km = kmeta[warp - 2];
+    const int32_t hq = hq0 + sl;
+    const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
+    const bool row_valid = row < qt.q_rows;
+    const int32_t i_rel = qt.q_start - qt.req_start + row;
+    const int32_t wpr = BK / 32;
     // waits are made warp-uniform: the TMEM loads/stores below need the whole warp
     auto wait_w = [&](uint32_t bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
     };
-    const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
-    const bool row_valid = row < qt.q_rows;
-    const int32_t i_rel = qt.q_start - qt.req_start + row;
-    const int2 qm = row_valid ? meta[qt.q_start + row] : make_int2(0, 0);
-    const MaskConsts mc{hdr->anchor_frames, hdr->spatial_radius, hdr->temporal_depth, hdr->temporal_stride,
-                        hdr->temporal_radius};
     float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = true;
     for (int32_t n = 0; n < nt; ++n) {
-      const int32_t b = n & 1;
-      const int32_t e = ent[n], cls = e & 3, j0 = (e >> 2) * BK;
-      if (!wait_w(smem_u32(&bars.s_full[b]), (n >> 1) & 1)) { ok = false; break; }
-      tc_fence_after();
-      if (cls == kTileGeneral) {  // warp-private copy: no barrier across warps is needed
-        __syncwarp();
-        for (int x = lane; x < BK; x += 32)
-          km[x] = j0 + x < qt.req_len ? meta[qt.req_start + j0 + x] : make_int2(0, 0);
-        __syncwarp();
-      }
+      const int32_t b = n % SB;
+      const int2 e = ent[n];
+      const int32_t cls = e.x & 3, j0 = (e.x >> 2) * BK;
       uint32_t keep[BK / 32];
-      if (cls == kTileFull) {
+      if (cls == kTileGeneral) {  // this row's bits of the tile's mask (read before the wait to hide the latency)
+        const uint32_t* mrow = masks + e.y + row * wpr;
 #pragma unroll
-        for (int c = 0; c < BK / 32; ++c) keep[c] = 0xFFFFFFFFu;
-      } else {
+        for (int c = 0; c < BK / 32; ++c) keep[c] = __ldg(mrow + c);
+      } else if (cls == kTileDiag) {
         const int32_t n_ok = min(BK, max(0, i_rel - j0 + 1));  // causal: columns 0 .. n_ok-1
 #pragma unroll
         for (int c = 0; c < BK / 32; ++c) {
           const int32_t k_in = min(32, max(0, n_ok - 32 * c));
           keep[c] = k_in >= 32 ? 0xFFFFFFFFu : ((1u << k_in) - 1u);
         }
-        if (cls == kTileGeneral) {
+      }
+      if (!wait_w(smem_u32(&bars.s_full[sl][b]), (n / SB) & 1)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t s_addr = t_lane + sl * 128 + b * BK;
+      // Row maximum.  BK = 64: the whole row of S stays in registers; BK = 128: the register file cannot hold
+      // 128 values beside the rest (168 registers per thread at this CTA size), so the row is read twice.
+      constexpr int NR = BK == 64 ? 64 : 32;
+      uint32_t r[NR];
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if constexpr (BK == 64) {
+        tmem_ld32_at<0>(s_addr, r);
+        tmem_ld32_at<32>(s_addr + 32, r);
+        tc_wait_ld();
+        if (cls != kTileFull) {
 #pragma unroll
-          for (int c = 0; c < BK / 32; ++c) {
-            uint32_t bits = 0;
-            for (int x = 0; x < 32; ++x) bits |= (st_keep(mc, qm, km[32 * c + x]) ? 1u : 0u) << x;
-            keep[c] &= bits;
+          for (int x = 0; x < 64; ++x)
+            if (!((keep[x >> 5] >> (x & 31)) & 1u)) r[x] = 0xFF800000u;  // -inf: drops out of max and exp
+        }
+#pragma unroll
+        for (int x = 0; x < 64; ++x) mx[x & 3] = fmaxf(mx[x & 3], __uint_as_float(r[x]));
+      } else {
+#pragma unroll
+        for (int c = 0; c < BK / 32; ++c) {
+          tmem_ld32_at<0>(s_addr + 32 * c, r);
+          tc_wait_ld();
+          if (cls != kTileFull) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x)
+              if (!((keep[c] >> x) & 1u)) r[x] = 0xFF800000u;
           }
+#pragma unroll
+          for (int x = 0; x < 32; ++x) mx[x & 3] = fmaxf(mx[x & 3], __uint_as_float(r[x]));
         }
       }
-      const uint32_t s_addr = t_lane + kColS + b * 128;
-      // pass 1: row maximum over the kept columns
-      float m_tile = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < BK / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(s_addr + 32 * c, r);
-        tc_wait_ld();
-#pragma unroll
-        for (int x = 0; x < 32; ++x)
-          if ((keep[c] >> x) & 1u) m_tile = fmaxf(m_tile, __uint_as_float(r[x]));
-      }
-      m_tile *= scale_log2;  // scale > 0; -inf stays -inf
+      const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
       // lazy rescale: move the reference only when the maximum grew by more than the threshold
       float m_use = m_ref;
       const bool grow = m_tile > m_ref + kRescaleThreshold || (m_ref == -INFINITY && m_tile > -INFINITY);
       if (grow) m_use = m_tile;
       const float m_sub = m_use == -INFINITY ? 0.f : m_use;
-      // pass 2: probabilities -> bf16 P in TMEM, row sum in fp32
-      float l_tile = 0.f;
-      const uint32_t p_addr = t_lane + kColP + b * 64;
-#pragma unroll
-      for (int c = 0; c < BK / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(s_addr + 32 * c, r);
-        tc_wait_ld();
-        uint32_t pk[16];
-#pragma unroll
-        for (int x = 0; x < 32; x += 2) {
-          float p0 = ex2(fmaf(__uint_as_float(r[x]), scale_log2, -m_sub));
-          float p1 = ex2(fmaf(__uint_as_float(r[x + 1]), scale_log2, -m_sub));
-          p0 = ((keep[c] >> x) & 1u) ? p0 : 0.f;
-          p1 = ((keep[c] >> (x + 1)) & 1u) ? p1 : 0.f;
-          l_tile += p0 + p1;
-          pk[x >> 1] = pack_bf16(p0, p1);
-        }
-        tmem_st16(p_addr + 16 * c, pk);
-      }
       // rescale O and the running sum where the reference moved (warp-uniform decision)
       const float alpha = grow ? (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_use)) : 1.f;
       if (n > 0 && __any_sync(0xffffffffu, grow)) {
-        // S[b] of tile n is complete, hence so is P.V of tile n-2: o_done is in phase n-1 or n
-        if (!wait_w(smem_u32(&bars.o_done), (n - 1) & 1)) { ok = false; break; }
+        // O must be quiescent: with one S buffer, S of tile n was issued behind P.V of tile n-1, so it is;
+        // with two, S of tile n only implies P.V of tile n-2 (o_done is then in phase n-1 or n).
+        if (SB > 1 && !wait_w(smem_u32(&bars.o_done[sl]), (n - 1) & 1)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll
         for (int c = 0; c < kD / 32; ++c) {
-          uint32_t r[32];
-          tmem_ld32(t_lane + kColO + 32 * c, r);
+          uint32_t t[32];
+          tmem_ld32(t_lane + kColO + sl * 128 + 32 * c, t);
           tc_wait_ld();
 #pragma unroll
-          for (int x = 0; x < 32; ++x) r[x] = __float_as_uint(__uint_as_float(r[x]) * alpha);
-          tmem_st32(t_lane + kColO + 32 * c, r);
+          for (int x = 0; x < 32; ++x) t[x] = __float_as_uint(__uint_as_float(t[x]) * alpha);
+          tmem_st32(t_lane + kColO + sl * 128 + 32 * c, t);
         }
       }
-      l_sum = l_sum * alpha + l_tile;
+      // probabilities -> bf16 P over the S columns, row sum in fp32
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c = 0; c < BK / 32; ++c) {
+        constexpr int kOff = BK == 64 ? 32 : 0;
+        if constexpr (BK == 128) {
+          tmem_ld32_at<0>(s_addr + 32 * c, r);
+          tc_wait_ld();
+          if (cls != kTileFull) {
+#pragma unroll
+            for (int x = 0; x < 32; ++x)
+              if (!((keep[c] >> x) & 1u)) r[x] = 0xFF800000u;
+          }
+        }
+        uint32_t pk[16];
+#pragma unroll
+        for (int x = 0; x < 32; x += 2) {
+          const float p0 = ex2(fmaf(__uint_as_float(r[kOff * c + x]), scale_log2, -m_sub));
+          const float p1 = ex2(fmaf(__uint_as_float(r[kOff * c + x + 1]), scale_log2, -m_sub));
+          ls[(x >> 1) & 3] += p0 + p1;
+          pk[x >> 1] = pack_bf16(p0, p1);
+        }
+        // P chunk c lands on S columns 16c..16c+15, which this thread has already consumed
+        tmem_st16(s_addr + 16 * c, pk);
+      }
+      l_sum = l_sum * alpha + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
       m_ref = m_use;
       tc_wait_st();
       tc_fence_before();
-      mbar_arrive(smem_u32(&bars.p_full[b]));
+      mbar_arrive(smem_u32(&bars.p_full[sl][b]));
     }
-    // The per-tile o_done barrier may still be two phases behind here (nothing orders the last
-    // softmax step after the second-to-last P.V), which a parity wait cannot tell apart; the
-    // dedicated single-phase barrier can.
-    if (ok) ok = wait_w(smem_u32(&bars.o_final), 0);
+    // o_done may be two phases behind here, which a parity wait cannot tell apart; o_final has one phase.
+    if (ok) ok = wait_w(smem_u32(&bars.o_final[sl]), 0);
     if (ok) {
       tc_fence_after();
       const float inv = 1.f / l_sum;
       __nv_bfloat16* dst = o + ((int64_t)(qt.q_start + row) * n_q_heads + hq) * kD;
 #pragma unroll
       for (int c = 0; c < kD / 32; ++c) {
-        uint32_t r[32];
-        tmem_ld32(t_lane + kColO + 32 * c, r);
+        uint32_t t[32];
+        tmem_ld32(t_lane + kColO + sl * 128 + 32 * c, t);
         tc_wait_ld();
         if (row_valid) {
 #pragma unroll
           for (int x = 0; x < 32; x += 8) {
             uint4 u;
-            u.x = pack_bf16(__uint_as_float(r[x + 0]) * inv, __uint_as_float(r[x + 1]) * inv);
-            u.y = pack_bf16(__uint_as_float(r[x + 2]) * inv, __uint_as_float(r[x + 3]) * inv);
-            u.z = pack_bf16(__uint_as_float(r[x + 4]) * inv, __uint_as_float(r[x + 5]) * inv);
-            u.w = pack_bf16(__uint_as_float(r[x + 6]) * inv, __uint_as_float(r[x + 7]) * inv);
+            u.x = pack_bf16(__uint_as_float(t[x + 0]) * inv, __uint_as_float(t[x + 1]) * inv);
+            u.y = pack_bf16(__uint_as_float(t[x + 2]) * inv, __uint_as_float(t[x + 3]) * inv);
+            u.z = pack_bf16(__uint_as_float(t[x + 4]) * inv, __uint_as_float(t[x + 5]) * inv);
+            u.w = pack_bf16(__uint_as_float(t[x + 6]) * inv, __uint_as_float(t[x + 7]) * inv);
             *reinterpret_cast<uint4*>(dst + 32 * c + x) = u;
           }
         }
@@ -502,9 +554,10 @@ __device__ int32_t g_default_status;
 template <int BK>
 static purekv_status launch(const PrefillArgs& a, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             int32_t* status) {
-  const size_t smem = 1024 + 2 * (size_t)kBQ * 128 + 2 * (size_t)kStages * 2 * BK * 128;
+  const size_t smem = 1024 + 2 * 2 * (size_t)kBQ * 128 + 2 * (size_t)Cfg<BK>::kStages * 2 * BK * 128;
   PK_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  dim3 grid((unsigned)a.info->n_qtiles, (unsigned)a.n_q_heads);
+  const int32_t G = a.n_q_heads / a.n_kv_heads;
+  dim3 grid((unsigned)((int64_t)a.info->n_qtiles * a.n_kv_heads * ((G + 1) / 2)));
   prefill_tc_kernel<BK><<<grid, kThreads, smem, a.stream>>>(mq, mk, mv, (__nv_bfloat16*)a.o, a.lse,
                                                             (const uint8_t*)a.plan, a.n_q_heads, a.n_kv_heads,
                                                             a.scale * 1.4426950408889634f, status);

@@ -34,50 +34,38 @@ def test_budget_matches_oracle_rule():
 
 def parse_plan(buf: np.ndarray):
     raw = buf.tobytes()
-    magic, tq, tk, nq, T, ne, oq, oo, oe, om, A, rs, D, st, rt, dense = struct.unpack_from("<Iiiiqqqqqqiiiiii", raw, 0)
-    assert magic == 0x504B5631
+    magic, tq, tk, nq, T, ne, nm, oq, oo, oe, om, wpr = struct.unpack_from("<Iiiiqqqqqqqi", raw, 0)
+    assert magic == 0x504B5632
     qt = np.frombuffer(raw, dtype=np.int32, count=nq * 8, offset=oq).reshape(nq, 8)
     order = np.frombuffer(raw, dtype=np.int32, count=nq, offset=oo)
-    entries = np.frombuffer(raw, dtype=np.int32, count=ne, offset=oe)
-    meta = np.frombuffer(raw, dtype=np.int32, count=2 * T, offset=om).reshape(T, 2)
-    return dict(tq=tq, tk=tk, nq=nq, T=T, qt=qt, order=order, entries=entries, meta=meta,
-                params=(A, rs, D, st, rt, dense))
+    entries = np.frombuffer(raw, dtype=np.int32, count=2 * ne, offset=oe).reshape(ne, 2)
+    masks = np.frombuffer(raw, dtype=np.uint32, count=nm, offset=om)
+    return dict(tq=tq, tk=tk, nq=nq, T=T, qt=qt, order=order, entries=entries, masks=masks, wpr=wpr)
 
 
 def check_plan(batch: inputs.Batch, mask: inputs.STMask, dtype, head_dim):
     b = pk.Batch(batch.seq_lens, batch.n_prefix, batch.n_frames, device=None)
     buf, info = pk.purekv_plan_build_host(b, pk.st_params(mask), dtype, head_dim)
+    assert pk.purekv_plan_bytes(b, pk.st_params(mask), dtype, head_dim) == info.bytes_used == len(buf)
     p = parse_plan(buf)
-    tq, tk = p["tq"], p["tk"]
-    assert (tq, tk) == (info.tile_q, info.tile_k)
+    tq, tk, wpr = p["tq"], p["tk"], p["wpr"]
+    assert (tq, tk) == (info.tile_q, info.tile_k) and wpr == max(1, tk // 32)
     mp = po.mask_params(mask)
     cu = batch.cu_seqlens
     pairs = kept = full = diag = gen = causal_tiles = 0
     qi = 0
-    n = mask.grid_h * mask.grid_w
     for r in range(batch.n_req):
         l = batch.seq_lens[r]
         mm = po.mask_matrix(mp, l, batch.n_prefix[r], batch.n_frames[r])
+        tril = np.tril(np.ones((l, l), dtype=bool))
         pairs += int(mm.sum())
-        # per-token coordinates
-        for i in range(l):
-            mx, my = p["meta"][cu[r] + i]
-            v = i - batch.n_prefix[r]
-            if v < 0:
-                assert mx & 3 == 0
-            elif v >= batch.n_frames[r] * n:
-                assert mx & 3 == 2
-            else:
-                f, c = divmod(v, n)
-                assert mx & 3 == 1 and (mx >> 2) & 0x7FFF == f and (mx >> 17) & 0x7FFF == f % mask.temporal_stride
-                assert my & 0xFFFF == c // mask.grid_w and (my >> 16) & 0xFFFF == c % mask.grid_w
         for q0 in range(0, l, tq):
             q1 = min(l, q0 + tq)
             row = p["qt"][qi]
             qi += 1
             assert row[0] == cu[r] + q0 and row[1] == q1 - q0 and row[2] == cu[r] and row[3] == l
             ents = p["entries"][row[4]:row[4] + row[5]]
-            listed = {int(e) >> 2: int(e) & 3 for e in ents}
+            listed = {int(e[0]) >> 2: (int(e[0]) & 3, int(e[1])) for e in ents}
             assert len(listed) == len(ents) and list(listed) == sorted(listed)
             nkt = (q1 - 1) // tk + 1
             causal_tiles += nkt
@@ -89,17 +77,21 @@ def check_plan(batch: inputs.Batch, mask: inputs.STMask, dtype, head_dim):
                     assert kt not in listed
                     continue
                 kept += 1
-                cls = listed[kt]
-                causal_cnt = int(np.tril(np.ones((l, l), dtype=bool))[q0:q1, j0:j1].sum())
+                cls, at = listed[kt]
                 if cnt == (q1 - q0) * tk:
-                    assert cls == 0
+                    assert cls == 0 and at == -1
                     full += 1
-                elif cnt == causal_cnt:
-                    assert cls == 1
+                elif cnt == int(tril[q0:q1, j0:j1].sum()):
+                    assert cls == 1 and at == -1
                     diag += 1
                 else:
-                    assert cls == 2
+                    assert cls == 2 and at >= 0
                     gen += 1
+                    words = p["masks"][at:at + tq * wpr].reshape(tq, wpr)
+                    bits = ((words[:, :, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(tq, wpr * 32)[:, :tk].astype(bool)
+                    want = np.zeros((tq, tk), dtype=bool)
+                    want[:q1 - q0, :j1 - j0] = sub
+                    assert np.array_equal(bits, want)           # the mask of Sec. 3.2, bit for bit
     assert qi == p["nq"] == info.n_qtiles
     assert (info.pairs_kept, info.tiles_kept, info.tiles_causal) == (pairs, kept, causal_tiles)
     assert (info.tiles_full, info.tiles_diag, info.tiles_general) == (full, diag, gen)
