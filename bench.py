@@ -45,46 +45,106 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    """Samples SM clock and clock-event reasons of one GPU while the timed region runs: NVML read-only queries
+    from a thread every few milliseconds, or `nvidia-smi -lms` when the NVML binding is missing."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, index: int):
-        self.index, self.rows, self.proc = index, [], None
+    def __init__(self, index: int, period_s: float = 0.005):
+        self.index, self.period = index, period_s
+        self.sm, self.smax, self.reasons = [], [], set()
+        self.proc = self.thread = self.nvml = None
+        self._stop = threading.Event()
+
+    def _physical_index(self) -> int:
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+        if vis:
+            ids = [v.strip() for v in vis.split(",") if v.strip()]
+            if self.index < len(ids) and ids[self.index].isdigit():
+                return int(ids[self.index])
+        return self.index
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+            import pynvml
+            pynvml.nvmlInit()
+            self.nvml = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(self._physical_index())
+            self.smax.append(float(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM)))
+            self.thread = threading.Thread(target=self._poll_nvml, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self._physical_index()}", f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread = threading.Thread(target=self._read_smi, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
-
-    def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        self.thread.join(timeout=2)
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+    def _poll_nvml(self):
+        n = self.nvml
+        bits = {"hw_slowdown": n.nvmlClocksEventReasonHwSlowdown, "hw_thermal_slowdown": n.nvmlClocksEventReasonHwThermalSlowdown,
+                "sw_thermal_slowdown": n.nvmlClocksEventReasonSwThermalSlowdown, "sw_power_cap": n.nvmlClocksEventReasonSwPowerCap}
+        while not self._stop.is_set():
             try:
-                sm.append(float(r[0]))
-                smax.append(float(r[1]))
+                self.sm.append(float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)))
+                r = n.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                for name, bit in bits.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def _read_smi(self):
+        for line in self.proc.stdout:
+            r = [c.strip() for c in line.split(",")]
+            try:
+                self.sm.append(float(r[0]))
+                self.smax.append(float(r[1]))
             except (ValueError, IndexError):
                 continue
-            for n, v in zip(names, r[3:7]):
+            for name, v in zip(self.NAMES, r[3:7]):
                 if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                    self.reasons.add(name)
+
+    def stop(self):
+        self._stop.set()
+        if self.proc is not None:
+            self.proc.terminate()
+        if self.thread is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["clock query unavailable"]}
+        self.thread.join(timeout=2)
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": max(self.smax) if self.smax else None,
+                "samples": len(self.sm), "reasons": sorted(self.reasons),
+                "source": "nvml" if self.nvml is not None else "nvidia-smi"}
+
+
+# ---- multi-process plumbing: one process per GPU, replicas only (the path has no exchange step) -----------
+def rank_env():
+    return (int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def max_over_ranks(x: float, device="cpu") -> float:
+    """Max of a host scalar over all ranks (the slowest rank sets the job's time)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(tokens_per_rank: int, world: int, seconds_per_step_max: float) -> float:
+    """Whole-job tokens/s of `world` independent replicas that each process tokens_per_rank per step."""
+    return world * tokens_per_rank / seconds_per_step_max
 
 
 def oracle_sample(wl, layers_x, budget_s: float = 20.0):
@@ -129,8 +189,7 @@ def oracle_sample(wl, layers_x, budget_s: float = 20.0):
 
 def run_reference(args, wl):
     """--impl reference: the oracle as it stands, on host cores, bounded sample per step."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    if rank_env()[1] != 0:
         return
     from oracle import purekv_oracle as po
     from paper_2510_25600_b200 import inputs
@@ -177,9 +236,7 @@ def main():
     from paper_2510_25600_b200 import binding as P
     from paper_2510_25600_b200.pipeline import PureKVPipeline
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local = rank_env()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -231,12 +288,9 @@ def main():
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop()
     pipe.check_status()
-    t_max = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t_max, op=dist.ReduceOp.MAX)
-    ms_step = float(t_max.item()) / args.steps
+    ms_step = max_over_ranks(ms_total, "cuda") / args.steps
     tokens = b.total_tokens
-    value = world * tokens / (ms_step * 1e-3)
+    value = job_throughput(tokens, world, ms_step * 1e-3)
 
     # ---- roofline of the dominant kernel (tensor-core prefill), from events around each launch -------------
     info_d, info_s = pipe.plan_dense.info, pipe.plan_st.info
@@ -309,13 +363,11 @@ def main():
             pipe.run_host((hq, hk, hv), h_out, d_in)
         sync_all()
         dt = time.perf_counter() - t0
-        t_e = torch.tensor([dt], dtype=torch.float64, device="cuda")
-        if world > 1:
-            dist.all_reduce(t_e, op=dist.ReduceOp.MAX)
+        dt = max_over_ranks(dt, "cuda")
         h2d = sum(t.numel() * t.element_size() for t in (hq, hk, hv))
         d2h = sum(t.numel() * t.element_size() for t in h_out)
-        e2e = {"value": world * tokens / (float(t_e.item()) / n_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": 1e3 * float(t_e.item()) / n_e2e}
+        e2e = {"value": job_throughput(tokens, world, dt / n_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": 1e3 * dt / n_e2e}
     pipe.check_status()
 
     # ---- the oracle on this machine's host cores (rank 0, N = 1 only) ---------------------------------------------
