@@ -140,6 +140,30 @@ purekv_status purekv_lowlayer_score(const void *q, const void *k, float *c_out, 
                                     int32_t head_dim, purekv_dtype dtype, float softmax_scale,
                                     void *ws, size_t ws_bytes, void *stream);
 
+/* ---- the same scores for callers that cannot hand over a workspace ---------------------------
+ * (The paper has no counterpart: this is a packaging variant of purekv_lowlayer_score.)
+ * Some callers cannot obtain device memory at the moment they need the scores: a serving engine that
+ * gave all of HBM to its KV-cache pool at start-up has nothing left to cudaMalloc from, and code that
+ * runs where an allocation would stall the device (cudaMalloc and cudaFree synchronise) must not
+ * allocate at all.  For them this entry point keeps its scratch (the window rows' log-sum-exp values)
+ * in an array inside the library's device image instead of a caller-provided workspace.  It calls no
+ * cudaMalloc / cudaFree and no allocating library routine; inputs and c_out are still the caller's.
+ *  - Limit: n_req * n_q_heads * window <= PUREKV_NOALLOC_SCORE_MAX_ROWS (65536 values, 256 KiB that
+ *    every GPU loading the library holds until the process exits).  Larger problems return
+ *    PUREKV_ERR_WORKSPACE and leave c_out untouched; use purekv_lowlayer_score for those.
+ *  - The first call on each device looks up the array's device address (with that device current).
+ *    Make that first call before any stream capture on that device.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents.  Nothing in
+ *    it has to start at zero (each call overwrites every entry it later reads), but two calls whose
+ *    kernels overlap on the GPU -- different streams, or different host threads -- race on it.
+ *    Serialise them, e.g. by issuing them on one stream.
+ * Results are those of purekv_lowlayer_score. */
+#define PUREKV_NOALLOC_SCORE_MAX_ROWS 65536
+purekv_status purekv_lowlayer_score_noalloc(const void *q, const void *k, float *c_out,
+                                            const purekv_batch *batch, int32_t window, int32_t n_q_heads,
+                                            int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                            float softmax_scale, void *stream);
+
 /* ---- V-norm weighting and top-h selection, n_layers layers per call (Eq. 3-4) ----------
  * S[L, g, j] = C[g, j] * ||V_L[j, g, :]||_2 for non-recent j; idx[L, g, cu_kept[r] + t] lists,
  * for request r, the h_keep[r] positions with the largest S (ties: lower position), in

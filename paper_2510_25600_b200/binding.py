@@ -26,7 +26,8 @@ FLAG_DENSE_CAUSAL = 1
 
 EXPORTS = ("purekv_version", "purekv_last_error", "purekv_budget", "purekv_plan_bytes", "purekv_plan_build",
            "purekv_plan_build_host",
-           "purekv_st_sparse_prefill", "purekv_score_ws_bytes", "purekv_lowlayer_score", "purekv_select_ws_bytes",
+           "purekv_st_sparse_prefill", "purekv_score_ws_bytes", "purekv_lowlayer_score", "purekv_lowlayer_score_noalloc",
+           "purekv_select_ws_bytes",
            "purekv_select_topk", "purekv_compact_kv", "purekv_poll_status")
 
 _i32p = C.POINTER(C.c_int32)
@@ -65,6 +66,8 @@ _lib.purekv_st_sparse_prefill.argtypes = [C.c_void_p] * 5 + [C.POINTER(CBatch), 
 _lib.purekv_score_ws_bytes.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_int32]
 _lib.purekv_lowlayer_score.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32, C.c_int32,
                                        C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.purekv_lowlayer_score_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32,
+                                               C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p]
 _lib.purekv_select_ws_bytes.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_int32]
 _lib.purekv_select_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.POINTER(CBatch), C.c_int32,
                                     C.c_void_p, _i32p, C.c_void_p, _i32p, C.c_int32, C.c_int32, C.c_int, C.c_void_p,
@@ -225,6 +228,23 @@ def purekv_lowlayer_score(q: torch.Tensor, k: torch.Tensor, batch: Batch, window
     _check(_lib.purekv_lowlayer_score(q.data_ptr(), k.data_ptr(), c_out.data_ptr(), C.byref(batch.c), window, h, hkv,
                                       d, _dtype_code(q), softmax_scale, ws.data_ptr(), ws.numel(), _stream()),
            "purekv_lowlayer_score")
+    return c_out
+
+
+NOALLOC_SCORE_MAX_ROWS = 65536
+
+
+def purekv_lowlayer_score_noalloc(q: torch.Tensor, k: torch.Tensor, batch: Batch, window: int, c_out: torch.Tensor,
+                                  softmax_scale: float = 0.0) -> torch.Tensor:
+    """purekv_lowlayer_score for callers that cannot allocate: the scratch is an array inside the library, so
+    this wrapper allocates nothing either -- `c_out` [H_kv, T] fp32 must be passed in.  Problems with
+    n_req * H * window > NOALLOC_SCORE_MAX_ROWS raise PureKVError(ERR_WORKSPACE).  Calls share the scratch:
+    keep them on one stream."""
+    assert q.is_contiguous() and k.is_contiguous() and c_out.is_contiguous() and c_out.dtype == torch.float32
+    t, h, d = q.shape
+    _check(_lib.purekv_lowlayer_score_noalloc(q.data_ptr(), k.data_ptr(), c_out.data_ptr(), C.byref(batch.c), window,
+                                              h, k.shape[1], d, _dtype_code(q), softmax_scale, _stream()),
+           "purekv_lowlayer_score_noalloc")
     return c_out
 
 

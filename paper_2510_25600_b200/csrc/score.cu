@@ -9,10 +9,19 @@
 // (Eq. 2), so the attention matrix never leaves the SM and no atomics are needed.
 // Logits are fp32 FMA chains over exact products; exponentials use exp2f.
 #include <algorithm>
+#include <mutex>
 
 #include "common.cuh"
 
 namespace purekv {
+
+// Scratch of purekv_lowlayer_score_noalloc: the window rows' log-sum-exp values, one float per
+// (request, query head, window position).  It lives in the library's device image, so every GPU that
+// loads the library holds these 256 KiB until the process exits.  Host code may not pass this name to
+// a kernel (on the host it is only a stand-in for the symbol); the device address comes from
+// cudaGetSymbolAddress, looked up once per device.
+constexpr size_t kNoallocScoreFloats = PUREKV_NOALLOC_SCORE_MAX_ROWS;
+static __device__ __align__(256) float g_noalloc_score_scratch[kNoallocScoreFloats + 64];  // + the 256 bytes of alignment slack the workspace rule asks for
 
 constexpr int kRB = 32;        // stacked rows per block
 constexpr int kKB = 64;        // keys per block
@@ -271,4 +280,42 @@ extern "C" purekv_status purekv_lowlayer_score(const void* q, const void* k, flo
   if (dtype == PUREKV_BF16)
     return launch_score<__nv_bfloat16>(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
   return launch_score<float>(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
+}
+
+// Device address of the static scratch array on the current device; resolved on the first call per device.
+static purekv_status noalloc_scratch(float** out) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static float* ptrs[kMaxDevices] = {};
+  int dev = -1;
+  PK_CUDA(cudaGetDevice(&dev));
+  PK_REQUIRE(dev >= 0 && dev < kMaxDevices, PUREKV_ERR_UNSUPPORTED, "device ordinal %d is beyond %d", dev, kMaxDevices);
+  std::lock_guard<std::mutex> lock(mu);
+  if (!ptrs[dev]) {
+    float* p = nullptr;
+    PK_CUDA(cudaGetSymbolAddress((void**)&p, g_noalloc_score_scratch));
+    PK_REQUIRE(p != nullptr, PUREKV_ERR_CUDA, "cudaGetSymbolAddress returned a null scratch address");
+    ptrs[dev] = p;
+  }
+  *out = ptrs[dev];
+  return PUREKV_OK;
+}
+
+extern "C" purekv_status purekv_lowlayer_score_noalloc(const void* q, const void* k, float* c_out,
+                                                       const purekv_batch* batch, int32_t window, int32_t n_q_heads,
+                                                       int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                                       float softmax_scale, void* stream) {
+  purekv_status st = check_batch(batch, true);
+  if (st != PUREKV_OK) return st;
+  PK_REQUIRE(window >= 1 && n_q_heads >= 1, PUREKV_ERR_INVALID_ARG, "window and n_q_heads must be >= 1");
+  const size_t need = (size_t)batch->n_req * (size_t)n_q_heads * (size_t)window;
+  PK_REQUIRE(need <= kNoallocScoreFloats, PUREKV_ERR_WORKSPACE,
+             "purekv_lowlayer_score_noalloc: n_req * n_q_heads * window = %zu exceeds the built-in scratch of %zu "
+             "values; use purekv_lowlayer_score with a caller-provided workspace",
+             need, kNoallocScoreFloats);
+  float* scratch = nullptr;
+  if ((st = noalloc_scratch(&scratch)) != PUREKV_OK) return st;
+  // The scratch needs no clearing: pass 1 writes every (request, head, window position) entry that pass 2 reads.
+  return purekv_lowlayer_score(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, dtype, softmax_scale,
+                               scratch, (kNoallocScoreFloats + 64) * sizeof(float), stream);
 }
