@@ -85,6 +85,10 @@ typedef struct {
   int64_t tiles_full, tiles_diag, tiles_general; /* kept tiles by predicate class          */
   int64_t bytes_used;       /* bytes of the plan buffer actually written                   */
   int32_t dtype, head_dim;  /* what the plan was built for                                 */
+  int32_t n_q_heads, n_kv_heads;
+  int32_t n_ctas, n_units;  /* tensor-core kernel: persistent CTAs and their work units    */
+  int32_t max_chunks;       /* most chunks a kept-key list was split into                  */
+  int64_t ws_bytes;         /* workspace purekv_st_sparse_prefill needs with this plan     */
 } purekv_plan_info;
 
 const char *purekv_version(void);
@@ -97,36 +101,49 @@ void purekv_last_error(char *buf, size_t buf_bytes);
 purekv_status purekv_budget(int32_t len, int32_t window, double keep_ratio, int32_t *h_out, int32_t *k_out);
 
 /* ---- planning (host work + one host-to-device copy) --------------------------------- */
-/* Upper bound of the plan buffer size in bytes for this batch and mask; 0 on invalid input. */
+/* Size of the plan buffer in bytes for this batch, mask and head layout; 0 on invalid input.
+ * n_ctas = number of persistent CTAs the tensor-core kernel is scheduled for (0: 148, one per
+ * SM of a B200). */
 size_t purekv_plan_bytes(const purekv_batch *batch, const purekv_st_params *params,
-                         purekv_dtype dtype, int32_t head_dim);
+                         purekv_dtype dtype, int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads,
+                         int32_t n_ctas);
 /* Builds, on the host, the per-query-tile lists of key tiles the mask keeps (each tagged
- * full / causal-only / general), a longest-first work order and per-token grid coordinates,
- * then copies them into `plan` (device, plan_bytes >= purekv_plan_bytes) on `stream` and
- * waits for that copy.  A plan depends only on the batch shape and mask, not on Q/K/V, and
- * serves every layer and head. */
+ * full / causal-only / general, the latter with a bit mask), and for the tensor-core kernel a
+ * static schedule: lists longer than about half a CTA's share are split into chunks, and the
+ * (query tile, head pair, chunk) units are spread over n_ctas CTAs, longest first.  The result
+ * is copied into `plan` (device, plan_bytes >= purekv_plan_bytes) on `stream`, and the call
+ * waits for that copy.  A plan depends only on the batch shape, the mask and the head layout,
+ * not on Q/K/V, and serves every layer.  It holds a few counters the kernel uses to combine
+ * split lists (they return to zero when a launch ends), so one plan serves one launch at a
+ * time: launches that share a plan must be ordered, e.g. on one stream, and a plan whose launch
+ * reported PUREKV_ERR_TIMEOUT must be rebuilt. */
 purekv_status purekv_plan_build(const purekv_batch *batch, const purekv_st_params *params,
-                                purekv_dtype dtype, int32_t head_dim, void *plan, size_t plan_bytes,
+                                purekv_dtype dtype, int32_t head_dim, int32_t n_q_heads,
+                                int32_t n_kv_heads, int32_t n_ctas, void *plan, size_t plan_bytes,
                                 purekv_plan_info *h_info, void *stream);
 
 /* Same planning, written to a HOST buffer h_plan (plan_bytes >= purekv_plan_bytes); makes no
  * CUDA call.  The bytes may be copied to the device by the caller and used as `plan`. */
 purekv_status purekv_plan_build_host(const purekv_batch *batch, const purekv_st_params *params,
-                                     purekv_dtype dtype, int32_t head_dim, void *h_plan, size_t plan_bytes,
-                                     purekv_plan_info *h_info);
+                                     purekv_dtype dtype, int32_t head_dim, int32_t n_q_heads,
+                                     int32_t n_kv_heads, int32_t n_ctas, void *h_plan,
+                                     size_t plan_bytes, purekv_plan_info *h_info);
 
 /* ---- ST-SpAttn prefill, one layer (Sec. 3.2; softmax of Eq. 1 over the kept keys) ------
  * O[i,hq,:] = sum_{j<=i, M(i,j)} softmax_j(scale * q_i.k_j) v_j.   lse (nullable) [H, T] fp32
  * receives log-sum-exp (natural log) of each row's kept logits.  softmax_scale 0 means
  * 1/sqrt(head_dim).  bf16 with head_dim 128 and tile 64/128 runs on the tcgen05 tensor
  * cores; other supported shapes (head_dim 32, 64, 128 or 256) run on CUDA cores.
+ * `ws` is a device workspace of at least h_info->ws_bytes bytes (it holds the partial results
+ * of split key lists; may be null when ws_bytes is 0); it need not be initialised.
  * `status` (nullable) is a device int32 the kernel sets to PUREKV_ERR_TIMEOUT if a bounded
  * wait expires; the caller zeroes it and reads it (purekv_poll_status). */
 purekv_status purekv_st_sparse_prefill(const void *q, const void *k, const void *v, void *o, float *lse,
-                                       const purekv_batch *batch, const void *plan,
+                                       const purekv_batch *batch, void *plan,
                                        const purekv_plan_info *h_info, int32_t n_q_heads,
                                        int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
-                                       float softmax_scale, int32_t *status, void *stream);
+                                       float softmax_scale, void *ws, size_t ws_bytes, int32_t *status,
+                                       void *stream);
 
 /* ---- low-layer window scores (Eq. 1-2) -------------------------------------------------
  * For request r of length l, w = min(window, l), KV head g, key j < l-w:

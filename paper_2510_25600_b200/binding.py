@@ -48,21 +48,24 @@ class PlanInfo(C.Structure):
     _fields_ = [("tile_q", C.c_int32), ("tile_k", C.c_int32), ("n_qtiles", C.c_int32), ("max_list", C.c_int32),
                 ("tiles_kept", C.c_int64), ("tiles_causal", C.c_int64), ("pairs_kept", C.c_int64),
                 ("tiles_full", C.c_int64), ("tiles_diag", C.c_int64), ("tiles_general", C.c_int64),
-                ("bytes_used", C.c_int64), ("dtype", C.c_int32), ("head_dim", C.c_int32)]
+                ("bytes_used", C.c_int64), ("dtype", C.c_int32), ("head_dim", C.c_int32),
+                ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("n_ctas", C.c_int32), ("n_units", C.c_int32),
+                ("max_chunks", C.c_int32), ("ws_bytes", C.c_int64)]
 
 
 _lib.purekv_version.restype = C.c_char_p
 _lib.purekv_plan_bytes.restype = C.c_size_t
 _lib.purekv_score_ws_bytes.restype = C.c_size_t
 _lib.purekv_select_ws_bytes.restype = C.c_size_t
-_lib.purekv_plan_bytes.argtypes = [C.POINTER(CBatch), C.POINTER(StParams), C.c_int, C.c_int32]
-_lib.purekv_plan_build.argtypes = [C.POINTER(CBatch), C.POINTER(StParams), C.c_int, C.c_int32, C.c_void_p, C.c_size_t,
-                                   C.POINTER(PlanInfo), C.c_void_p]
-_lib.purekv_plan_build_host.argtypes = [C.POINTER(CBatch), C.POINTER(StParams), C.c_int, C.c_int32, C.c_void_p,
-                                        C.c_size_t, C.POINTER(PlanInfo)]
+_lib.purekv_plan_bytes.argtypes = [C.POINTER(CBatch), C.POINTER(StParams), C.c_int, C.c_int32, C.c_int32, C.c_int32,
+                                   C.c_int32]
+_lib.purekv_plan_build.argtypes = [C.POINTER(CBatch), C.POINTER(StParams), C.c_int, C.c_int32, C.c_int32, C.c_int32,
+                                   C.c_int32, C.c_void_p, C.c_size_t, C.POINTER(PlanInfo), C.c_void_p]
+_lib.purekv_plan_build_host.argtypes = [C.POINTER(CBatch), C.POINTER(StParams), C.c_int, C.c_int32, C.c_int32,
+                                        C.c_int32, C.c_int32, C.c_void_p, C.c_size_t, C.POINTER(PlanInfo)]
 _lib.purekv_st_sparse_prefill.argtypes = [C.c_void_p] * 5 + [C.POINTER(CBatch), C.c_void_p, C.POINTER(PlanInfo),
                                                              C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_float,
-                                                             C.c_void_p, C.c_void_p]
+                                                             C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p]
 _lib.purekv_score_ws_bytes.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_int32]
 _lib.purekv_lowlayer_score.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32, C.c_int32,
                                        C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -167,45 +170,52 @@ class Plan:
         self.buf, self.info = buf, info
 
 
-def purekv_plan_bytes(batch: Batch, params: StParams, dtype: int, head_dim: int) -> int:
-    return int(_lib.purekv_plan_bytes(C.byref(batch.c), C.byref(params), dtype, head_dim))
+def purekv_plan_bytes(batch: Batch, params: StParams, dtype: int, head_dim: int, n_q_heads: int, n_kv_heads: int,
+                      n_ctas: int = 0) -> int:
+    return int(_lib.purekv_plan_bytes(C.byref(batch.c), C.byref(params), dtype, head_dim, n_q_heads, n_kv_heads, n_ctas))
 
 
-def purekv_plan_build(batch: Batch, params: StParams, dtype: int, head_dim: int,
-                      buf: Optional[torch.Tensor] = None) -> Plan:
-    n = purekv_plan_bytes(batch, params, dtype, head_dim)
+def purekv_plan_build(batch: Batch, params: StParams, dtype: int, head_dim: int, n_q_heads: int, n_kv_heads: int,
+                      buf: Optional[torch.Tensor] = None, n_ctas: int = 0) -> Plan:
+    n = purekv_plan_bytes(batch, params, dtype, head_dim, n_q_heads, n_kv_heads, n_ctas)
     if n == 0:
-        _check(_lib.purekv_plan_build(C.byref(batch.c), C.byref(params), dtype, head_dim, None, 0,
-                                      C.byref(PlanInfo()), None), "purekv_plan_build")
+        _check(_lib.purekv_plan_build(C.byref(batch.c), C.byref(params), dtype, head_dim, n_q_heads, n_kv_heads,
+                                      n_ctas, None, 0, C.byref(PlanInfo()), None), "purekv_plan_build")
     if buf is None:
         buf = torch.empty(n, dtype=torch.uint8, device="cuda")
     info = PlanInfo()
-    _check(_lib.purekv_plan_build(C.byref(batch.c), C.byref(params), dtype, head_dim, buf.data_ptr(), buf.numel(),
-                                  C.byref(info), _stream()), "purekv_plan_build")
+    _check(_lib.purekv_plan_build(C.byref(batch.c), C.byref(params), dtype, head_dim, n_q_heads, n_kv_heads, n_ctas,
+                                  buf.data_ptr(), buf.numel(), C.byref(info), _stream()), "purekv_plan_build")
     return Plan(buf, info)
 
 
-def purekv_plan_build_host(batch: Batch, params: StParams, dtype: int, head_dim: int):
+def purekv_plan_build_host(batch: Batch, params: StParams, dtype: int, head_dim: int, n_q_heads: int, n_kv_heads: int,
+                           n_ctas: int = 0):
     """Plan bytes in host memory (numpy uint8) + PlanInfo; makes no CUDA call."""
-    n = purekv_plan_bytes(batch, params, dtype, head_dim)
+    n = purekv_plan_bytes(batch, params, dtype, head_dim, n_q_heads, n_kv_heads, n_ctas)
     buf = np.zeros(max(n, 1), dtype=np.uint8)
     info = PlanInfo()
-    _check(_lib.purekv_plan_build_host(C.byref(batch.c), C.byref(params), dtype, head_dim, buf.ctypes.data, n,
-                                       C.byref(info)), "purekv_plan_build_host")
+    _check(_lib.purekv_plan_build_host(C.byref(batch.c), C.byref(params), dtype, head_dim, n_q_heads, n_kv_heads,
+                                       n_ctas, buf.ctypes.data, n, C.byref(info)), "purekv_plan_build_host")
     return buf[:info.bytes_used], info
 
 
 def purekv_st_sparse_prefill(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, batch: Batch, plan: Plan,
                              out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
-                             softmax_scale: float = 0.0, status: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """q [T,H,d], k,v [T,H_kv,d] contiguous on the GPU; returns O [T,H,d]."""
+                             softmax_scale: float = 0.0, status: Optional[torch.Tensor] = None,
+                             ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q [T,H,d], k,v [T,H_kv,d] contiguous on the GPU; returns O [T,H,d].  `ws`: workspace of
+    plan.info.ws_bytes bytes (allocated here when not given)."""
     assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous()
     t, h, d = q.shape
     if out is None:
         out = torch.empty_like(q)
+    if ws is None and plan.info.ws_bytes > 0:
+        ws = torch.empty(plan.info.ws_bytes, dtype=torch.uint8, device=q.device)
     _check(_lib.purekv_st_sparse_prefill(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), _ptr(lse),
                                          C.byref(batch.c), plan.buf.data_ptr(), C.byref(plan.info), h, k.shape[1], d,
-                                         _dtype_code(q), softmax_scale, _ptr(status), _stream()),
+                                         _dtype_code(q), softmax_scale, _ptr(ws), 0 if ws is None else ws.numel(),
+                                         _ptr(status), _stream()),
            "purekv_st_sparse_prefill")
     return out
 

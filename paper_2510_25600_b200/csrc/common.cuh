@@ -40,8 +40,9 @@ __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162flo
 
 // ---- plan buffer layout (device memory, written by purekv_plan_build) -------------------
 // [PlanHeader][QTile x n_qtiles][order int32 x n_qtiles][entries int2 x n_entries][masks uint32 x n_mask_words]
-// all sections 16-byte aligned.
-constexpr uint32_t kPlanMagic = 0x504B5632u;  // "PKV2"
+// [cta_off int32 x (n_ctas+1)][Unit x n_units][merge counters int32 x n_counters]
+// all sections 16-byte aligned.  The last three sections exist only in plans for the tensor-core kernel.
+constexpr uint32_t kPlanMagic = 0x504B5633u;  // "PKV3"
 
 enum TileClass : int32_t { kTileFull = 0, kTileDiag = 1, kTileGeneral = 2 };
 
@@ -54,7 +55,10 @@ struct PlanHeader {
   int64_t n_mask_words;
   int64_t off_qtiles, off_order, off_entries, off_masks;  // byte offsets from the plan base
   int32_t words_per_row;                                  // max(1, tile_k / 32)
-  int32_t pad[3];
+  int32_t n_ctas, n_units, n_counters;
+  int64_t off_cta, off_units, off_counters;
+  int32_t n_q_heads, n_kv_heads;
+  int64_t part_slots;  // partial-result slots of the workspace (split chunks x query heads)
 };
 
 struct QTile {
@@ -71,5 +75,23 @@ struct QTile {
 // entry.y = for a general tile, the index of its first mask word: row r of the query tile owns
 // words [entry.y + r*words_per_row, +words_per_row), bit c of word w = key 32*w + c of the tile
 // (causality already applied; rows past q_rows are zero); -1 otherwise.
+
+// One unit of work of the tensor-core kernel: a query tile x a pair of query heads x a contiguous
+// chunk of the tile's kept-key list.  CTA c runs units cta_off[c] .. cta_off[c+1]-1 in order.
+// A list split into n_chunks > 1 chunks leaves one partial result per chunk and head in the
+// workspace; the chunk that arrives last (merge counter) combines them.
+struct __align__(16) Unit {
+  int32_t q_start, q_rows, req_start;
+  int32_t ent_begin, ent_count;  // into entries[]
+  int32_t pair;                  // KV head g = pair / ppg, first query head g*G + 2*(pair % ppg), ppg = (G+1)/2
+  int32_t chunk, n_chunks;
+  int32_t part_base;             // workspace slot of (chunk 0, head 0) = part_base; slot(chunk, hq) = (part_base + chunk) * H + hq
+  int32_t counter_base;          // merge counter of head hq = counters[counter_base + hq]
+  int32_t pad[2];
+};
+
+// Partial result of one (chunk, head): 128 x 128 fp32 unnormalised output laid out [col/4][row][col%4],
+// then 128 reference maxima (log2 domain) and 128 row sums.
+constexpr int64_t kPartFloats = 128 * 128 + 2 * 128;
 
 }  // namespace purekv

@@ -101,12 +101,78 @@ purekv_status purekv_budget(int32_t len, int32_t window, double keep_ratio, int3
   return PUREKV_OK;
 }
 
+// Splits long kept-key lists into chunks and assigns (query tile, head pair, chunk) units to n_ctas persistent
+// CTAs, longest first onto the least loaded CTA.  The cost of a unit is its tile count plus a fixed overhead
+// (query load, pipeline fill, epilogue), in tiles.
+static void schedule_units(const std::vector<QTile>& qtiles, int32_t H, int32_t Hkv, int32_t n_ctas, int32_t tk,
+                           std::vector<Unit>& units, std::vector<int32_t>& cta_off, int32_t* n_counters,
+                           int64_t* part_slots, int32_t* max_chunks) {
+  const int32_t G = H / Hkv, ppg = (G + 1) / 2, n_pairs = Hkv * ppg;
+  const int32_t overhead = tk >= 128 ? 2 : 3;
+  int64_t total = 0;
+  for (const QTile& q : qtiles) total += (int64_t)n_pairs * (q.entry_count + overhead);
+  const int64_t target = std::max<int64_t>(1, total / n_ctas);
+  const int32_t l_max = (int32_t)std::min<int64_t>(64, std::max<int64_t>(4, target / 2));
+  struct Item { Unit u; int32_t cost; };
+  std::vector<Item> items;
+  int32_t counters = 0, mc = 1;
+  int64_t slots = 0;
+  for (const QTile& q : qtiles) {
+    const int32_t nch = std::max(1, (q.entry_count + l_max - 1) / l_max);
+    mc = std::max(mc, nch);
+    const int32_t part_base = nch > 1 ? (int32_t)slots : -1, counter_base = nch > 1 ? counters : -1;
+    if (nch > 1) { slots += nch; counters += H; }
+    for (int32_t c = 0; c < nch; ++c) {
+      const int32_t a = (int32_t)((int64_t)q.entry_count * c / nch), e = (int32_t)((int64_t)q.entry_count * (c + 1) / nch);
+      for (int32_t pr = 0; pr < n_pairs; ++pr) {
+        Unit u;
+        u.q_start = q.q_start; u.q_rows = q.q_rows; u.req_start = q.req_start;
+        u.ent_begin = q.entry_begin + a; u.ent_count = e - a;
+        u.pair = pr; u.chunk = c; u.n_chunks = nch;
+        u.part_base = part_base; u.counter_base = counter_base;
+        u.pad[0] = u.pad[1] = 0;
+        items.push_back({u, e - a + overhead});
+      }
+    }
+  }
+  std::stable_sort(items.begin(), items.end(), [](const Item& x, const Item& y) { return x.cost > y.cost; });
+  std::vector<std::vector<int32_t>> bins((size_t)n_ctas);
+  std::vector<int64_t> load((size_t)n_ctas, 0);
+  // min-heap of (load, cta)
+  std::vector<std::pair<int64_t, int32_t>> heap;
+  for (int32_t c = 0; c < n_ctas; ++c) heap.push_back({0, c});
+  auto cmp = [](const std::pair<int64_t, int32_t>& x, const std::pair<int64_t, int32_t>& y) { return x > y; };
+  std::make_heap(heap.begin(), heap.end(), cmp);
+  for (size_t i = 0; i < items.size(); ++i) {
+    std::pop_heap(heap.begin(), heap.end(), cmp);
+    auto& top = heap.back();
+    bins[top.second].push_back((int32_t)i);
+    top.first += items[i].cost;
+    std::push_heap(heap.begin(), heap.end(), cmp);
+  }
+  units.clear();
+  cta_off.assign(1, 0);
+  for (int32_t c = 0; c < n_ctas; ++c) {
+    for (int32_t i : bins[c]) units.push_back(items[i].u);
+    cta_off.push_back((int32_t)units.size());
+  }
+  *n_counters = counters;
+  *part_slots = slots * H;
+  *max_chunks = mc;
+}
+
 static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
-                                int32_t head_dim, purekv_plan_info* info, std::vector<uint8_t>& host) {
+                                int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, int32_t n_ctas,
+                                purekv_plan_info* info, std::vector<uint8_t>& host) {
   int tq, tk;
   purekv_status st = check_params(b, p, dtype, head_dim, &tq, &tk);
   if (st != PUREKV_OK) return st;
   PK_REQUIRE(info, PUREKV_ERR_INVALID_ARG, "info is null");
+  PK_REQUIRE(n_q_heads >= 1 && n_kv_heads >= 1 && n_q_heads % n_kv_heads == 0 && n_q_heads <= 65535,
+             PUREKV_ERR_INVALID_ARG, "n_q_heads %d must be a positive multiple of n_kv_heads %d", n_q_heads,
+             n_kv_heads);
+  PK_REQUIRE(n_ctas >= 0 && n_ctas <= 4096, PUREKV_ERR_INVALID_ARG, "n_ctas %d outside [0, 4096]", n_ctas);
+  if (n_ctas == 0) n_ctas = 148;  // one persistent CTA per SM of a B200
   const bool dense = (p->flags & PUREKV_FLAG_DENSE_CAUSAL) != 0;
   const int32_t gw = p->grid_w, gh = p->grid_h, n = gw * gh;
   const int64_t T = b->total_tokens;
@@ -244,6 +310,17 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   std::stable_sort(order.begin(), order.end(),
                    [&](int32_t u, int32_t v) { return qtiles[u].entry_count > qtiles[v].entry_count; });
 
+  // tensor-core plans carry the persistent kernel's schedule
+  std::vector<Unit> units;
+  std::vector<int32_t> cta_off;
+  int32_t n_counters = 0, max_chunks = 1;
+  int64_t part_slots = 0;
+  if (tq == 128 && nq > 0) {
+    schedule_units(qtiles, n_q_heads, n_kv_heads, n_ctas, tk, units, cta_off, &n_counters, &part_slots, &max_chunks);
+  } else {
+    n_ctas = 0;
+  }
+
   PlanHeader h;
   memset(&h, 0, sizeof(h));
   h.magic = kPlanMagic;
@@ -258,7 +335,16 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   h.off_order = h.off_qtiles + align16((int64_t)nq * sizeof(QTile));
   h.off_entries = h.off_order + align16((int64_t)nq * 4);
   h.off_masks = h.off_entries + align16(h.n_entries * 8);
-  const int64_t total = h.off_masks + align16(h.n_mask_words * 4);
+  h.n_ctas = units.empty() ? 0 : n_ctas;
+  h.n_units = (int32_t)units.size();
+  h.n_counters = n_counters;
+  h.n_q_heads = n_q_heads;
+  h.n_kv_heads = n_kv_heads;
+  h.part_slots = part_slots;
+  h.off_cta = h.off_masks + align16(h.n_mask_words * 4);
+  h.off_units = h.off_cta + align16(((int64_t)h.n_ctas + 1) * 4);
+  h.off_counters = h.off_units + align16((int64_t)h.n_units * sizeof(Unit));
+  const int64_t total = h.off_counters + align16((int64_t)n_counters * 4);
 
   host.assign((size_t)total, 0);
   memcpy(host.data(), &h, sizeof(h));
@@ -266,6 +352,10 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   if (nq) memcpy(host.data() + h.off_order, order.data(), (size_t)nq * 4);
   if (!entries.empty()) memcpy(host.data() + h.off_entries, entries.data(), entries.size() * 8);
   if (!masks.empty()) memcpy(host.data() + h.off_masks, masks.data(), masks.size() * 4);
+  if (!units.empty()) {
+    memcpy(host.data() + h.off_cta, cta_off.data(), cta_off.size() * 4);
+    memcpy(host.data() + h.off_units, units.data(), units.size() * sizeof(Unit));
+  }
 
   info->tile_q = tq;
   info->tile_k = tk;
@@ -273,21 +363,29 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   info->bytes_used = total;
   info->dtype = (int32_t)dtype;
   info->head_dim = head_dim;
+  info->n_q_heads = n_q_heads;
+  info->n_kv_heads = n_kv_heads;
+  info->n_ctas = h.n_ctas;
+  info->n_units = h.n_units;
+  info->max_chunks = max_chunks;
+  info->ws_bytes = part_slots * kPartFloats * (int64_t)sizeof(float);
   return PUREKV_OK;
 }
 
-size_t purekv_plan_bytes(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype, int32_t head_dim) {
+size_t purekv_plan_bytes(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype, int32_t head_dim,
+                         int32_t n_q_heads, int32_t n_kv_heads, int32_t n_ctas) {
   purekv_plan_info info;
   std::vector<uint8_t> host;
-  if (build_plan(b, p, dtype, head_dim, &info, host) != PUREKV_OK) return 0;
+  if (build_plan(b, p, dtype, head_dim, n_q_heads, n_kv_heads, n_ctas, &info, host) != PUREKV_OK) return 0;
   return host.size();
 }
 
 purekv_status purekv_plan_build_host(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
-                                     int32_t head_dim, void* h_plan, size_t plan_bytes, purekv_plan_info* info) {
+                                     int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, int32_t n_ctas,
+                                     void* h_plan, size_t plan_bytes, purekv_plan_info* info) {
   PK_REQUIRE(h_plan, PUREKV_ERR_INVALID_ARG, "h_plan is null");
   std::vector<uint8_t> host;
-  purekv_status st = build_plan(b, p, dtype, head_dim, info, host);
+  purekv_status st = build_plan(b, p, dtype, head_dim, n_q_heads, n_kv_heads, n_ctas, info, host);
   if (st != PUREKV_OK) return st;
   PK_REQUIRE(host.size() <= plan_bytes, PUREKV_ERR_WORKSPACE, "plan needs %zu bytes, buffer has %zu", host.size(),
              plan_bytes);
@@ -296,11 +394,11 @@ purekv_status purekv_plan_build_host(const purekv_batch* b, const purekv_st_para
 }
 
 purekv_status purekv_plan_build(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
-                                int32_t head_dim, void* plan, size_t plan_bytes, purekv_plan_info* info,
-                                void* stream) {
+                                int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, int32_t n_ctas, void* plan,
+                                size_t plan_bytes, purekv_plan_info* info, void* stream) {
   PK_REQUIRE(plan, PUREKV_ERR_INVALID_ARG, "plan is null");
   std::vector<uint8_t> host;
-  purekv_status st = build_plan(b, p, dtype, head_dim, info, host);
+  purekv_status st = build_plan(b, p, dtype, head_dim, n_q_heads, n_kv_heads, n_ctas, info, host);
   if (st != PUREKV_OK) return st;
   PK_REQUIRE(host.size() <= plan_bytes, PUREKV_ERR_WORKSPACE, "plan needs %zu bytes, buffer has %zu", host.size(),
              plan_bytes);

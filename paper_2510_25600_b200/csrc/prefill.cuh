@@ -9,11 +9,13 @@ struct PrefillArgs {
   void* o;
   float* lse;
   const purekv_batch* batch;
-  const void* plan;
+  void* plan;
   const purekv_plan_info* info;
   int32_t n_q_heads, n_kv_heads, head_dim;
   purekv_dtype dtype;
   float scale;
+  void* ws;
+  size_t ws_bytes;
   int32_t* status;
   cudaStream_t stream;
 };

@@ -1,18 +1,23 @@
 // Tensor-core ST-SpAttn prefill (Sec. 3.2) for bf16, head_dim 128, on sm_100a.
 //
-// One CTA = one 128-row query tile of a PAIR of query heads that share a KV head ("slots"), so
-// every K/V tile staged in shared memory feeds two heads.  It walks the plan's list of kept key
-// tiles: key blocks the mask removes are never read.  Roles:
-//   warp 0      TMA producer: Q of both slots once, then K and V tiles (128B-swizzled, two
-//               64-column panels each) into a ring of stages.
-//   warp 1      owns the 512 TMEM columns; one lane issues tcgen05.mma, alternating slots:
+// Persistent kernel: one CTA per SM walks the list of work units the plan assigned to it.  A unit is a
+// 128-row query tile of a PAIR of query heads that share a KV head ("slots") and a chunk of that tile's
+// list of kept key tiles, so every K/V tile staged in shared memory feeds two heads and key blocks the
+// mask removes are never read.  Roles:
+//   warp 8      producer: per unit Q of both slots, then per key tile the tile's class word and, for
+//               general tiles, its bit mask (bulk copy) into a small ring, and K and V (TMA, 128-byte
+//               swizzle, two 64-column panels each) into a ring of stages.  It runs ahead across units.
+//   warp 9      owns the 512 TMEM columns; one lane issues tcgen05.mma, alternating slots:
 //               S = Q K^T (K-major A and B from shared memory) and
 //               O += P V (A = bf16 P from TMEM, B = V as MN-major shared-memory operand),
 //               so the tensor pipe works on one slot while the other slot's rows are in softmax.
-//   warps 2-9   one thread per query row of a slot: the row of S from TMEM into registers, the
-//               tile's predicate class (full / causal / bit mask from the plan), online softmax in
-//               the log2 domain with lazy rescaling of O, bf16 P written over S, final normalise
-//               and store.
+//   warps 0-7   one thread per query row of a slot (registers raised with setmaxnreg at the expense of
+//               warps 8-11): the row of S from TMEM into registers, the
+//               tile's predicate (none / causal / bit mask), online softmax in the log2 domain with lazy
+//               rescaling of O, bf16 P written over S; at the end of a unit either the normalised output
+//               (whole list in one unit) or an unnormalised fp32 partial result plus (max, sum) per row
+//               into the workspace.  The chunk of a split list that finishes last (a counter in the plan)
+//               combines the partial results in chunk order, so the result does not depend on timing.
 // Every wait on an mbarrier is bounded in time; on expiry the CTA raises a shared abort flag,
 // sets the device status word, drains, frees TMEM and exits.
 #include <cuda.h>
@@ -24,7 +29,9 @@ namespace tc {
 
 constexpr int kD = 128;
 constexpr int kBQ = 128;
-constexpr int kThreads = 320;  // warp 0 TMA, warp 1 MMA, warps 2-5 softmax of slot 0, warps 6-9 of slot 1
+constexpr int kThreads = 384;  // warps 0-3 softmax of slot 0, warps 4-7 of slot 1, warp 8 producer, warp 9 MMA, 10-11 idle
+constexpr int kWarpProducer = 8, kWarpMma = 9;
+constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // per-thread registers after the warpgroups trade them
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 256;
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
@@ -183,21 +190,36 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
          ((uint32_t)(128 >> 4) << 24);
 }
 
+// 1-D bulk copy global -> shared, completing on an mbarrier (addresses and size multiples of 16 bytes).
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
 template <int BK>
 struct Cfg {
   static constexpr int kStages = BK == 64 ? 4 : 2;  // K/V ring depth (32 KB resp. 64 KB per stage)
   static constexpr int kSBuf = BK == 64 ? 2 : 1;    // S buffers per slot: kSBuf * BK = 128 TMEM columns
+  static constexpr int kMeta = 2 * kStages;         // ring of per-tile class words and bit masks
+  static constexpr uint32_t kMaskBytes = kBQ * BK / 8;
 };
 
 template <int BK>
 struct __align__(8) Barriers {
-  static constexpr int ST = Cfg<BK>::kStages, SB = Cfg<BK>::kSBuf;
-  uint64_t q_full;
+  static constexpr int ST = Cfg<BK>::kStages, SB = Cfg<BK>::kSBuf, MR = Cfg<BK>::kMeta;
+  uint64_t q_full, q_empty;
   uint64_t k_full[ST], k_empty[ST], v_full[ST], v_empty[ST];
+  uint64_t m_full[MR];     // producer -> softmax: class word (and bit mask) of a tile are in place
   uint64_t s_full[2][SB];  // MMA -> softmax: S of (slot, buffer) is complete
   uint64_t p_full[2][SB];  // softmax -> MMA: P written (and O rescaled) by all 128 row threads
   uint64_t o_done[2];      // one completion per P.V product of the slot
-  uint64_t o_final[2];     // completes once, after the slot's last P.V product
+  uint64_t o_final[2];     // one completion per unit, after the slot's last P.V product
+  uint64_t rows_sync[2];   // the 128 row threads of a slot meet here around the merge-counter update
   uint64_t drain;
 };
 
@@ -206,50 +228,49 @@ template <int BK>
 __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
     const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, float* __restrict__ lse,
-    const uint8_t* __restrict__ plan, int32_t n_q_heads, int32_t n_kv_heads, float scale_log2,
+    uint8_t* __restrict__ plan, float* __restrict__ ws, int32_t n_q_heads, int32_t n_kv_heads, float scale_log2,
     int32_t* __restrict__ status) {
-  constexpr int ST = Cfg<BK>::kStages, SB = Cfg<BK>::kSBuf;
+  constexpr int ST = Cfg<BK>::kStages, SB = Cfg<BK>::kSBuf, MR = Cfg<BK>::kMeta;
   constexpr uint32_t kPanelQ = kBQ * 128;  // bytes of one 64-column panel of a Q tile
   constexpr uint32_t kTileQ = 2 * kPanelQ;
   constexpr uint32_t kPanelKV = BK * 128;  // bytes of one 64-column panel of a K or V tile
   constexpr uint32_t kTileKV = 2 * kPanelKV;
+  constexpr uint32_t kMaskBytes = Cfg<BK>::kMaskBytes;
   extern __shared__ uint8_t smem_raw[];
   __shared__ Barriers<BK> bars;
+  __shared__ int2 meta_s[MR];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
+  __shared__ int merge_s[2];
 
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sQ = smem0;                 // [2 slots][2 panels][128 rows x 128 B]
   const uint32_t sK = sQ + 2 * kTileQ;       // [ST][2 panels][BK rows x 128 B]
   const uint32_t sV = sK + ST * kTileKV;
+  const uint32_t sM = sV + ST * kTileKV;     // [MR][128 rows x BK/8 B]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(plan);
-  const QTile* qtiles = reinterpret_cast<const QTile*>(plan + hdr->off_qtiles);
-  const int32_t* order = reinterpret_cast<const int32_t*>(plan + hdr->off_order);
   const int2* entries = reinterpret_cast<const int2*>(plan + hdr->off_entries);
   const uint32_t* masks = reinterpret_cast<const uint32_t*>(plan + hdr->off_masks);
-  // blockIdx.x = rank of the query tile in the longest-first order * n_pairs + pair, so the long lists of
-  // every head start first.  A pair = (KV head, two of its query heads); the last pair of an odd group is single.
-  const int32_t G = n_q_heads / n_kv_heads, ppg = (G + 1) >> 1, n_pairs = n_kv_heads * ppg;
-  const QTile qt = qtiles[order[blockIdx.x / n_pairs]];
-  const int32_t pair = blockIdx.x % n_pairs;
-  const int32_t g = pair / ppg, pr = pair % ppg;
-  const int32_t hq0 = g * G + 2 * pr;
-  const int32_t n_slots = (2 * pr + 1 < G) ? 2 : 1;
-  const int32_t nt = qt.entry_count;
-  const int2* ent = entries + qt.entry_begin;
+  const int32_t* cta_off = reinterpret_cast<const int32_t*>(plan + hdr->off_cta);
+  const Unit* units = reinterpret_cast<const Unit*>(plan + hdr->off_units);
+  int32_t* counters = reinterpret_cast<int32_t*>(plan + hdr->off_counters);
+  const int32_t G = n_q_heads / n_kv_heads, ppg = (G + 1) >> 1;
+  const int32_t u_begin = cta_off[blockIdx.x], u_end = cta_off[blockIdx.x + 1];
   volatile int* abort_flag = &abort_s;
 
   if (tid == 0) {
-    abort_s = *reinterpret_cast<volatile int32_t*>(status) != 0;  // an earlier CTA already failed
+    abort_s = *reinterpret_cast<volatile int32_t*>(status) != 0;  // an earlier CTA or launch already failed
     mbar_init(smem_u32(&bars.q_full), 1);
+    mbar_init(smem_u32(&bars.q_empty), 1);
     for (int s = 0; s < ST; ++s) {
       mbar_init(smem_u32(&bars.k_full[s]), 1);
       mbar_init(smem_u32(&bars.k_empty[s]), 1);
       mbar_init(smem_u32(&bars.v_full[s]), 1);
       mbar_init(smem_u32(&bars.v_empty[s]), 1);
     }
+    for (int s = 0; s < MR; ++s) mbar_init(smem_u32(&bars.m_full[s]), 1);
     for (int sl = 0; sl < 2; ++sl) {
       for (int b = 0; b < SB; ++b) {
         mbar_init(smem_u32(&bars.s_full[sl][b]), 1);
@@ -257,12 +278,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       }
       mbar_init(smem_u32(&bars.o_done[sl]), 1);
       mbar_init(smem_u32(&bars.o_final[sl]), 1);
+      mbar_init(smem_u32(&bars.rows_sync[sl]), 128);
     }
     mbar_init(smem_u32(&bars.drain), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == kWarpMma) {
     tmem_alloc(smem_u32(&tmem_base_s), kTmemCols);
     tmem_relinquish();
   }
@@ -270,51 +292,97 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
-  const bool start_ok = abort_s == 0;
+  const bool start_ok = abort_s == 0 && u_begin < u_end;
+  // the two softmax warpgroups take registers from the warpgroup of the producer and MMA warps
 
-  if (start_ok && warp == 0) {
-    // ---------------- TMA producer ----------------
-    if (lane == 0) {
-      mbar_expect_tx(smem_u32(&bars.q_full), n_slots * kTileQ);
-      for (int sl = 0; sl < n_slots; ++sl) {
-        tma_load_3d(sQ + sl * kTileQ, &tm_q, smem_u32(&bars.q_full), 0, hq0 + sl, qt.q_start);
-        tma_load_3d(sQ + sl * kTileQ + kPanelQ, &tm_q, smem_u32(&bars.q_full), 64, hq0 + sl, qt.q_start);
+  if (warp >= 8) {
+    setmaxnreg_dec<kRegsOther>();
+  if (start_ok && warp == kWarpProducer) {
+    // ---------------- producer (whole warp; lane 0 issues) ----------------
+    uint32_t it = 0;  // key tiles issued so far by this CTA, over all units
+    int32_t issued_k = 0, issued_v = 0;
+    bool ok = true;
+    Unit u = units[u_begin];
+    for (int32_t k = u_begin; ok && k < u_end; ++k) {
+      const Unit nxt = units[min(k + 1, u_end - 1)];
+      const int32_t nt = u.ent_count;
+      const int32_t g = u.pair / ppg, hq0 = g * G + 2 * (u.pair % ppg);
+      const int32_t n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
+      if (lane == 0) {
+        if (k > u_begin) ok = mbar_wait(smem_u32(&bars.q_empty), (uint32_t)(k - u_begin - 1) & 1u, abort_flag);
+        if (ok) {
+          mbar_expect_tx(smem_u32(&bars.q_full), n_slots * kTileQ);
+          for (int sl = 0; sl < n_slots; ++sl) {
+            tma_load_3d(sQ + sl * kTileQ, &tm_q, smem_u32(&bars.q_full), 0, hq0 + sl, u.q_start);
+            tma_load_3d(sQ + sl * kTileQ + kPanelQ, &tm_q, smem_u32(&bars.q_full), 64, hq0 + sl, u.q_start);
+          }
+        }
       }
-      int32_t issued_k = 0, issued_v = 0;
-      for (int32_t n = 0; n < nt; ++n) {
-        const int32_t s = n % ST;
-        const uint32_t par = ((n / ST) - 1) & 1;
-        const int32_t tok = qt.req_start + (ent[n].x >> 2) * BK;
-        if (n >= ST && !mbar_wait(smem_u32(&bars.k_empty[s]), par, abort_flag)) break;
-        mbar_expect_tx(smem_u32(&bars.k_full[s]), kTileKV);
-        tma_load_3d(sK + s * kTileKV, &tm_k, smem_u32(&bars.k_full[s]), 0, g, tok);
-        tma_load_3d(sK + s * kTileKV + kPanelKV, &tm_k, smem_u32(&bars.k_full[s]), 64, g, tok);
-        issued_k = n + 1;
-        if (n >= ST && !mbar_wait(smem_u32(&bars.v_empty[s]), par, abort_flag)) break;
-        mbar_expect_tx(smem_u32(&bars.v_full[s]), kTileKV);
-        tma_load_3d(sV + s * kTileKV, &tm_v, smem_u32(&bars.v_full[s]), 0, g, tok);
-        tma_load_3d(sV + s * kTileKV + kPanelKV, &tm_v, smem_u32(&bars.v_full[s]), 64, g, tok);
-        issued_v = n + 1;
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      for (int32_t n0 = 0; ok && n0 < nt; n0 += 32) {
+        int2 e_l = make_int2(0, -1);
+        if (n0 + lane < nt) e_l = __ldg(entries + u.ent_begin + n0 + lane);
+        const int32_t n1 = min(nt, n0 + 32);
+        for (int32_t n = n0; ok && n < n1; ++n) {
+          int2 e;
+          e.x = __shfl_sync(0xffffffffu, e_l.x, n - n0);
+          e.y = __shfl_sync(0xffffffffu, e_l.y, n - n0);
+          if (lane == 0) {
+            const uint32_t s = it % ST, par = ((it / ST) - 1u) & 1u, ms = it % MR;
+            const int32_t tok = u.req_start + (e.x >> 2) * BK;
+            if (it >= (uint32_t)ST) ok = mbar_wait(smem_u32(&bars.k_empty[s]), par, abort_flag);
+            if (ok) {
+              meta_s[ms] = e;
+              if ((e.x & 3) == kTileGeneral) {
+                mbar_expect_tx(smem_u32(&bars.m_full[ms]), kMaskBytes);
+                bulk_load(sM + ms * kMaskBytes, masks + e.y, kMaskBytes, smem_u32(&bars.m_full[ms]));
+              } else {
+                mbar_arrive(smem_u32(&bars.m_full[ms]));
+              }
+              mbar_expect_tx(smem_u32(&bars.k_full[s]), kTileKV);
+              tma_load_3d(sK + s * kTileKV, &tm_k, smem_u32(&bars.k_full[s]), 0, g, tok);
+              tma_load_3d(sK + s * kTileKV + kPanelKV, &tm_k, smem_u32(&bars.k_full[s]), 64, g, tok);
+              issued_k = (int32_t)it + 1;
+              if (it >= (uint32_t)ST) ok = mbar_wait(smem_u32(&bars.v_empty[s]), par, abort_flag);
+            }
+            if (ok) {
+              mbar_expect_tx(smem_u32(&bars.v_full[s]), kTileKV);
+              tma_load_3d(sV + s * kTileKV, &tm_v, smem_u32(&bars.v_full[s]), 0, g, tok);
+              tma_load_3d(sV + s * kTileKV + kPanelKV, &tm_v, smem_u32(&bars.v_full[s]), 64, g, tok);
+              issued_v = (int32_t)it + 1;
+            }
+          }
+          ++it;
+          ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        }
       }
-      if (*abort_flag) {
-        // drain: every issued copy must have landed before shared memory is released
-        const uint64_t t0 = global_ns();
-        for (int32_t n = max(0, issued_k - ST); n < issued_k; ++n)
-          while (!mbar_try_wait(smem_u32(&bars.k_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < kWaitLimitNs) {}
-        for (int32_t n = max(0, issued_v - ST); n < issued_v; ++n)
-          while (!mbar_try_wait(smem_u32(&bars.v_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < kWaitLimitNs) {}
-        while (!mbar_try_wait(smem_u32(&bars.q_full), 0) && global_ns() - t0 < kWaitLimitNs) {}
-      }
+      u = nxt;
     }
-  } else if (start_ok && warp == 1) {
+    if (lane == 0 && *abort_flag) {
+      // drain: every issued copy must have landed before shared memory is released
+      const uint64_t t0 = global_ns();
+      for (int32_t n = max(0, issued_k - ST); n < issued_k; ++n)
+        while (!mbar_try_wait(smem_u32(&bars.k_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+      for (int32_t n = max(0, issued_v - ST); n < issued_v; ++n)
+        while (!mbar_try_wait(smem_u32(&bars.v_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+      for (int32_t n = max(0, issued_k - MR); n < issued_k; ++n)
+        while (!mbar_try_wait(smem_u32(&bars.m_full[n % MR]), (n / MR) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+      __nanosleep(20000);  // a Q tile possibly still in flight (its barrier's phase is not known here)
+    }
+  } else if (start_ok && warp == kWarpMma) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(BK, false);
       constexpr uint32_t idesc_pv = instr_desc(kD, true);
+      uint32_t it_base = 0;            // key tiles of earlier units
+      uint32_t tq[2] = {0, 0};         // S products issued per slot, over all units
+      uint32_t tp[2] = {0, 0};         // P.V products issued per slot, over all units
+      int32_t nt = 0, n_slots = 0;
       // S(slot, n) = Q_slot K_n^T; the last slot to read K_n releases its stage
       auto issue_qk = [&](int32_t sl, int32_t n) -> bool {
-        const int32_t s = n % ST, b = n % SB;
-        if (!mbar_wait(smem_u32(&bars.k_full[s]), (n / ST) & 1, abort_flag)) return false;
+        const uint32_t it = it_base + (uint32_t)n;
+        const uint32_t s = it % ST, b = tq[sl] % SB;
+        if (!mbar_wait(smem_u32(&bars.k_full[s]), (it / ST) & 1u, abort_flag)) return false;
         tc_fence_after();
         const uint32_t d_addr = tmem + sl * 128 + b * BK;
 #pragma unroll
@@ -323,15 +391,21 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
           const uint32_t koff = s * kTileKV + (ks >> 2) * kPanelKV + (ks & 3) * 32;
           mma_ss(d_addr, smem_desc(sQ + qoff, 16, 1024), smem_desc(sK + koff, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
         }
-        if (sl == n_slots - 1) tc_commit(smem_u32(&bars.k_empty[s]));
+        if (sl == n_slots - 1) {
+          tc_commit(smem_u32(&bars.k_empty[s]));
+          if (n == nt - 1) tc_commit(smem_u32(&bars.q_empty));  // the unit's last read of Q
+        }
         tc_commit(smem_u32(&bars.s_full[sl][b]));
+        ++tq[sl];
         return true;
       };
       // O(slot) += P(slot, n) V_n; the last slot to read V_n releases its stage
       auto issue_pv = [&](int32_t sl, int32_t n) -> bool {
-        const int32_t s = n % ST, b = n % SB;
-        if (!mbar_wait(smem_u32(&bars.v_full[s]), (n / ST) & 1, abort_flag)) return false;
-        if (!mbar_wait(smem_u32(&bars.p_full[sl][b]), (n / SB) & 1, abort_flag)) return false;
+        const uint32_t it = it_base + (uint32_t)n;
+        const uint32_t s = it % ST, b = tp[sl] % SB;
+        if (!mbar_wait(smem_u32(&bars.v_full[s]), (it / ST) & 1u, abort_flag)) return false;
+        // P of the unit's first tile also implies that the previous unit's output has left TMEM
+        if (!mbar_wait(smem_u32(&bars.p_full[sl][b]), (tp[sl] / SB) & 1u, abort_flag)) return false;
         tc_fence_after();
         const uint32_t p_addr = tmem + sl * 128 + b * BK;
 #pragma unroll
@@ -343,16 +417,26 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         if (sl == n_slots - 1) tc_commit(smem_u32(&bars.v_empty[s]));
         tc_commit(smem_u32(&bars.o_done[sl]));
         if (n == nt - 1) tc_commit(smem_u32(&bars.o_final[sl]));
+        ++tp[sl];
         return true;
       };
-      bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort_flag);
-      for (int32_t n = 0; ok && n < SB && n < nt; ++n)
-        for (int32_t sl = 0; ok && sl < n_slots; ++sl) ok = issue_qk(sl, n);
-      for (int32_t n = 0; ok && n < nt; ++n)
-        for (int32_t sl = 0; ok && sl < n_slots; ++sl) {
-          ok = issue_pv(sl, n);
-          if (ok && n + SB < nt) ok = issue_qk(sl, n + SB);  // in order behind P.V of tile n, which frees S(slot, n % SB)
-        }
+      bool ok = true;
+      Unit u = units[u_begin];
+      for (int32_t k = u_begin; ok && k < u_end; ++k) {
+        const Unit nxt = units[min(k + 1, u_end - 1)];
+        nt = u.ent_count;
+        n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
+        ok = mbar_wait(smem_u32(&bars.q_full), (uint32_t)(k - u_begin) & 1u, abort_flag);
+        for (int32_t n = 0; ok && n < SB && n < nt; ++n)
+          for (int32_t sl = 0; ok && sl < n_slots; ++sl) ok = issue_qk(sl, n);
+        for (int32_t n = 0; ok && n < nt; ++n)
+          for (int32_t sl = 0; ok && sl < n_slots; ++sl) {
+            ok = issue_pv(sl, n);
+            if (ok && n + SB < nt) ok = issue_qk(sl, n + SB);  // in order behind P.V of tile n, which frees S(slot, n % SB)
+          }
+        it_base += (uint32_t)nt;
+        u = nxt;
+      }
       if (!ok) {
         // leaving early: let every issued MMA finish before TMEM is released
         tc_commit(smem_u32(&bars.drain));
@@ -360,157 +444,266 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         while (!mbar_try_wait(smem_u32(&bars.drain), 0) && global_ns() - t0 < kWaitLimitNs) {}
       }
     }
-  } else if (start_ok && (warp - 2) / 4 < n_slots) {
+  }
+  } else {
+    setmaxnreg_inc<kRegsSoftmax>();
+  if (start_ok) {
     // ---------------- softmax / epilogue: one thread per query row of one slot ----------------
-    const int sl = (warp - 2) >> 2;
+    const int sl = warp >> 2;
     const int quad = warp & 3;  // TMEM lane quadrant this warp may access
     const int row = quad * 32 + lane;
-    const int32_t hq = hq0 + sl;
     const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
-    const bool row_valid = row < qt.q_rows;
-    const int32_t i_rel = qt.q_start - qt.req_start + row;
-    const int32_t wpr = BK / 32;
     // waits are made warp-uniform: the TMEM loads/stores below need the whole warp
     auto wait_w = [&](uint32_t bar, uint32_t parity) -> bool {
       return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
     };
-    float m_ref = -INFINITY, l_sum = 0.f;
+    uint32_t it_base = 0;     // key tiles of earlier units (both slots)
+    uint32_t t = 0;           // tiles this slot has processed, over all units
+    uint32_t slot_units = 0;  // units this slot took part in
+    uint32_t row_syncs = 0;   // completed phases of rows_sync[sl]
     bool ok = true;
-    for (int32_t n = 0; n < nt; ++n) {
-      const int32_t b = n % SB;
-      const int2 e = ent[n];
-      const int32_t cls = e.x & 3, j0 = (e.x >> 2) * BK;
-      uint32_t keep[BK / 32];
-      if (cls == kTileGeneral) {  // this row's bits of the tile's mask (read before the wait to hide the latency)
-        const uint32_t* mrow = masks + e.y + row * wpr;
-#pragma unroll
-        for (int c = 0; c < BK / 32; ++c) keep[c] = __ldg(mrow + c);
-      } else if (cls == kTileDiag) {
-        const int32_t n_ok = min(BK, max(0, i_rel - j0 + 1));  // causal: columns 0 .. n_ok-1
-#pragma unroll
-        for (int c = 0; c < BK / 32; ++c) {
-          const int32_t k_in = min(32, max(0, n_ok - 32 * c));
-          keep[c] = k_in >= 32 ? 0xFFFFFFFFu : ((1u << k_in) - 1u);
+    // bounded meeting of the slot's 128 row threads (a plain barrier could not be left on a failure)
+    auto sync_rows = [&]() -> bool {
+      mbar_arrive(smem_u32(&bars.rows_sync[sl]));
+      const bool r = wait_w(smem_u32(&bars.rows_sync[sl]), row_syncs & 1u);
+      ++row_syncs;
+      return r;
+    };
+    Unit u = units[u_begin];
+    for (int32_t k = u_begin; ok && k < u_end; ++k) {
+      const Unit nxt = units[min(k + 1, u_end - 1)];
+      const int32_t nt = u.ent_count;
+      const int32_t pr = u.pair % ppg, g = u.pair / ppg;
+      const int32_t n_slots = (2 * pr + 1 < G) ? 2 : 1;
+      if (sl >= n_slots) {
+        // A single-head unit: this slot sits it out, but still follows the tile ring step by step.  A parity wait
+        // only tells the current phase from the one before, so a waiter must never get a whole ring ahead.
+        for (int32_t n = 0; ok && n < nt; ++n) {
+          const uint32_t it = it_base + (uint32_t)n;
+          ok = wait_w(smem_u32(&bars.m_full[it % MR]), (it / MR) & 1u);
         }
+        it_base += (uint32_t)nt;
+        u = nxt;
+        continue;
       }
-      if (!wait_w(smem_u32(&bars.s_full[sl][b]), (n / SB) & 1)) { ok = false; break; }
-      tc_fence_after();
-      const uint32_t s_addr = t_lane + sl * 128 + b * BK;
-      // Row maximum.  BK = 64: the whole row of S stays in registers; BK = 128: the register file cannot hold
-      // 128 values beside the rest (168 registers per thread at this CTA size), so the row is read twice.
-      constexpr int NR = BK == 64 ? 64 : 32;
-      uint32_t r[NR];
-      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      if constexpr (BK == 64) {
+      const int32_t hq = g * G + 2 * pr + sl;
+      const bool row_valid = row < u.q_rows;
+      const int32_t i_rel = u.q_start - u.req_start + row;
+      float m_ref = -INFINITY, l_sum = 0.f;
+      for (int32_t n = 0; n < nt; ++n) {
+        const uint32_t it = it_base + (uint32_t)n, ms = it % MR, b = t % SB;
+        if (!wait_w(smem_u32(&bars.m_full[ms]), (it / MR) & 1u)) { ok = false; break; }
+        const int2 e = meta_s[ms];
+        const int32_t cls = e.x & 3, j0 = (e.x >> 2) * BK;
+        uint32_t keep[BK / 32];
+        if (cls == kTileGeneral) {  // this row's bits of the tile's mask
+          const uint32_t* mrow = reinterpret_cast<const uint32_t*>(smem_raw + (sM - smem_u32(smem_raw)) + ms * kMaskBytes) +
+                                 row * (BK / 32);
+          if constexpr (BK == 128) {
+            const uint4 w4 = *reinterpret_cast<const uint4*>(mrow);
+            keep[0] = w4.x; keep[1] = w4.y; keep[BK / 32 - 2] = w4.z; keep[BK / 32 - 1] = w4.w;
+          } else {
+            const uint2 w2 = *reinterpret_cast<const uint2*>(mrow);
+            keep[0] = w2.x; keep[1] = w2.y;
+          }
+        } else if (cls == kTileDiag) {
+          const int32_t n_ok = min(BK, max(0, i_rel - j0 + 1));  // causal: columns 0 .. n_ok-1
+#pragma unroll
+          for (int c = 0; c < BK / 32; ++c) {
+            const int32_t k_in = min(32, max(0, n_ok - 32 * c));
+            keep[c] = k_in >= 32 ? 0xFFFFFFFFu : ((1u << k_in) - 1u);
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < BK / 32; ++c) keep[c] = 0xFFFFFFFFu;
+        }
+        if (!wait_w(smem_u32(&bars.s_full[sl][b]), (t / SB) & 1u)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t s_addr = t_lane + sl * 128 + b * BK;
+        // the whole row of S into registers
+        uint32_t r[BK];
         tmem_ld32_at<0>(s_addr, r);
         tmem_ld32_at<32>(s_addr + 32, r);
+        if constexpr (BK == 128) {
+          tmem_ld32_at<64>(s_addr + 64, r);
+          tmem_ld32_at<96>(s_addr + 96, r);
+        }
         tc_wait_ld();
         if (cls != kTileFull) {
 #pragma unroll
-          for (int x = 0; x < 64; ++x)
-            if (!((keep[x >> 5] >> (x & 31)) & 1u)) r[x] = 0xFF800000u;  // -inf: drops out of max and exp
-        }
+          for (int c = 0; c < BK / 32; ++c) {
+            if (__any_sync(0xffffffffu, keep[c] != 0xFFFFFFFFu)) {  // warp-uniform: skip chunks every row keeps
 #pragma unroll
-        for (int x = 0; x < 64; ++x) mx[x & 3] = fmaxf(mx[x & 3], __uint_as_float(r[x]));
-      } else {
+              for (int x = 0; x < 32; ++x)
+                if (!((keep[c] >> x) & 1u)) r[32 * c + x] = 0xFF800000u;  // -inf: drops out of max and exp
+            }
+          }
+        }
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int x = 0; x < BK; ++x) mx[x & 3] = fmaxf(mx[x & 3], __uint_as_float(r[x]));
+        const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
+        // lazy rescale: move the reference only when the maximum grew by more than the threshold
+        float m_use = m_ref;
+        const bool grow = m_tile > m_ref + kRescaleThreshold || (m_ref == -INFINITY && m_tile > -INFINITY);
+        if (grow) m_use = m_tile;
+        const float m_sub = m_use == -INFINITY ? 0.f : m_use;
+        // rescale O and the running sum where the reference moved (warp-uniform decision)
+        const float alpha = grow ? (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_use)) : 1.f;
+        if (n > 0 && __any_sync(0xffffffffu, grow)) {
+          // O must be quiescent: with one S buffer, S of tile n was issued behind P.V of tile n-1, so it is;
+          // with two, S of tile n only implies P.V of tile n-2 (o_done is then in phase t-1 or t).
+          if (SB > 1 && !wait_w(smem_u32(&bars.o_done[sl]), (t - 1u) & 1u)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < kD / 32; ++c) {
+            uint32_t tt[32];
+            tmem_ld32(t_lane + kColO + sl * 128 + 32 * c, tt);
+            tc_wait_ld();
+#pragma unroll
+            for (int x = 0; x < 32; ++x) tt[x] = __float_as_uint(__uint_as_float(tt[x]) * alpha);
+            tmem_st32(t_lane + kColO + sl * 128 + 32 * c, tt);
+          }
+        }
+        // probabilities -> bf16 P over the S columns, row sum in fp32
+        float2 ls2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        const float2 sc2 = make_float2(scale_log2, scale_log2), mm2 = make_float2(-m_sub, -m_sub);
 #pragma unroll
         for (int c = 0; c < BK / 32; ++c) {
-          tmem_ld32_at<0>(s_addr + 32 * c, r);
-          tc_wait_ld();
-          if (cls != kTileFull) {
+          uint32_t pk[16];
 #pragma unroll
-            for (int x = 0; x < 32; ++x)
-              if (!((keep[c] >> x) & 1u)) r[x] = 0xFF800000u;
+          for (int x = 0; x < 32; x += 2) {
+            const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[32 * c + x]), __uint_as_float(r[32 * c + x + 1])), sc2, mm2);
+            const float2 p = make_float2(ex2(a.x), ex2(a.y));
+            ls2[(x >> 1) & 1] = __fadd2_rn(ls2[(x >> 1) & 1], p);
+            pk[x >> 1] = pack_bf16(p.x, p.y);
           }
-#pragma unroll
-          for (int x = 0; x < 32; ++x) mx[x & 3] = fmaxf(mx[x & 3], __uint_as_float(r[x]));
+          // P chunk c lands on S columns 16c..16c+15, which this thread has already consumed
+          tmem_st16(s_addr + 16 * c, pk);
         }
+        l_sum = l_sum * alpha + ((ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y));
+        m_ref = m_use;
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars.p_full[sl][b]));
+        ++t;
       }
-      const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
-      // lazy rescale: move the reference only when the maximum grew by more than the threshold
-      float m_use = m_ref;
-      const bool grow = m_tile > m_ref + kRescaleThreshold || (m_ref == -INFINITY && m_tile > -INFINITY);
-      if (grow) m_use = m_tile;
-      const float m_sub = m_use == -INFINITY ? 0.f : m_use;
-      // rescale O and the running sum where the reference moved (warp-uniform decision)
-      const float alpha = grow ? (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_use)) : 1.f;
-      if (n > 0 && __any_sync(0xffffffffu, grow)) {
-        // O must be quiescent: with one S buffer, S of tile n was issued behind P.V of tile n-1, so it is;
-        // with two, S of tile n only implies P.V of tile n-2 (o_done is then in phase n-1 or n).
-        if (SB > 1 && !wait_w(smem_u32(&bars.o_done[sl]), (n - 1) & 1)) { ok = false; break; }
-        tc_fence_after();
+      if (!ok) break;
+      it_base += (uint32_t)nt;
+      // o_done may be two phases behind here, which a parity wait cannot tell apart; o_final moves once per unit.
+      if (!wait_w(smem_u32(&bars.o_final[sl]), slot_units & 1u)) { ok = false; break; }
+      ++slot_units;
+      tc_fence_after();
+      if (u.n_chunks == 1) {
+        const float inv = 1.f / l_sum;
+        __nv_bfloat16* dst = o + ((int64_t)(u.q_start + row) * n_q_heads + hq) * kD;
 #pragma unroll
         for (int c = 0; c < kD / 32; ++c) {
-          uint32_t t[32];
-          tmem_ld32(t_lane + kColO + sl * 128 + 32 * c, t);
+          uint32_t tt[32];
+          tmem_ld32(t_lane + kColO + sl * 128 + 32 * c, tt);
           tc_wait_ld();
+          if (row_valid) {
 #pragma unroll
-          for (int x = 0; x < 32; ++x) t[x] = __float_as_uint(__uint_as_float(t[x]) * alpha);
-          tmem_st32(t_lane + kColO + sl * 128 + 32 * c, t);
-        }
-      }
-      // probabilities -> bf16 P over the S columns, row sum in fp32
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int c = 0; c < BK / 32; ++c) {
-        constexpr int kOff = BK == 64 ? 32 : 0;
-        if constexpr (BK == 128) {
-          tmem_ld32_at<0>(s_addr + 32 * c, r);
-          tc_wait_ld();
-          if (cls != kTileFull) {
-#pragma unroll
-            for (int x = 0; x < 32; ++x)
-              if (!((keep[c] >> x) & 1u)) r[x] = 0xFF800000u;
+            for (int x = 0; x < 32; x += 8) {
+              uint4 w;
+              w.x = pack_bf16(__uint_as_float(tt[x + 0]) * inv, __uint_as_float(tt[x + 1]) * inv);
+              w.y = pack_bf16(__uint_as_float(tt[x + 2]) * inv, __uint_as_float(tt[x + 3]) * inv);
+              w.z = pack_bf16(__uint_as_float(tt[x + 4]) * inv, __uint_as_float(tt[x + 5]) * inv);
+              w.w = pack_bf16(__uint_as_float(tt[x + 6]) * inv, __uint_as_float(tt[x + 7]) * inv);
+              *reinterpret_cast<uint4*>(dst + 32 * c + x) = w;
+            }
           }
         }
-        uint32_t pk[16];
+        if (lse && row_valid)
+          lse[(int64_t)hq * hdr->total_tokens + u.q_start + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+      } else {
+        // one chunk of a split list: leave the unnormalised result for whoever arrives last
+        float* part = ws + ((int64_t)(u.part_base + u.chunk) * n_q_heads + hq) * kPartFloats;
 #pragma unroll
-        for (int x = 0; x < 32; x += 2) {
-          const float p0 = ex2(fmaf(__uint_as_float(r[kOff * c + x]), scale_log2, -m_sub));
-          const float p1 = ex2(fmaf(__uint_as_float(r[kOff * c + x + 1]), scale_log2, -m_sub));
-          ls[(x >> 1) & 3] += p0 + p1;
-          pk[x >> 1] = pack_bf16(p0, p1);
+        for (int c = 0; c < kD / 32; ++c) {
+          uint32_t tt[32];
+          tmem_ld32(t_lane + kColO + sl * 128 + 32 * c, tt);
+          tc_wait_ld();
+#pragma unroll
+          for (int x = 0; x < 32; x += 4)
+            *reinterpret_cast<uint4*>(part + ((c * 8 + (x >> 2)) * 128 + row) * 4) =
+                make_uint4(tt[x], tt[x + 1], tt[x + 2], tt[x + 3]);
         }
-        // P chunk c lands on S columns 16c..16c+15, which this thread has already consumed
-        tmem_st16(s_addr + 16 * c, pk);
-      }
-      l_sum = l_sum * alpha + ((ls[0] + ls[1]) + (ls[2] + ls[3]));
-      m_ref = m_use;
-      tc_wait_st();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&bars.p_full[sl][b]));
-    }
-    // o_done may be two phases behind here, which a parity wait cannot tell apart; o_final has one phase.
-    if (ok) ok = wait_w(smem_u32(&bars.o_final[sl]), 0);
-    if (ok) {
-      tc_fence_after();
-      const float inv = 1.f / l_sum;
-      __nv_bfloat16* dst = o + ((int64_t)(qt.q_start + row) * n_q_heads + hq) * kD;
-#pragma unroll
-      for (int c = 0; c < kD / 32; ++c) {
-        uint32_t t[32];
-        tmem_ld32(t_lane + kColO + sl * 128 + 32 * c, t);
-        tc_wait_ld();
-        if (row_valid) {
-#pragma unroll
-          for (int x = 0; x < 32; x += 8) {
-            uint4 u;
-            u.x = pack_bf16(__uint_as_float(t[x + 0]) * inv, __uint_as_float(t[x + 1]) * inv);
-            u.y = pack_bf16(__uint_as_float(t[x + 2]) * inv, __uint_as_float(t[x + 3]) * inv);
-            u.z = pack_bf16(__uint_as_float(t[x + 4]) * inv, __uint_as_float(t[x + 5]) * inv);
-            u.w = pack_bf16(__uint_as_float(t[x + 6]) * inv, __uint_as_float(t[x + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + 32 * c + x) = u;
+        part[128 * 128 + row] = m_ref;
+        part[128 * 128 + 128 + row] = l_sum;
+        __threadfence();
+        if (!sync_rows()) { ok = false; break; }
+        if (row == 0) {
+          __threadfence();
+          int32_t* cnt = counters + u.counter_base + hq;
+          const int32_t old = atomicAdd(cnt, 1);
+          const int last = old == u.n_chunks - 1;
+          if (last) atomicExch(cnt, 0);  // every chunk has arrived: ready for the next launch
+          __threadfence();
+          merge_s[sl] = last;
+        }
+        if (!sync_rows()) { ok = false; break; }
+        if (merge_s[sl]) {
+          __threadfence();
+          const float* p0 = ws + ((int64_t)u.part_base * n_q_heads + hq) * kPartFloats;
+          const int64_t cstride = (int64_t)n_q_heads * kPartFloats;
+          float m_all = -INFINITY;
+          for (int32_t c = 0; c < u.n_chunks; ++c) {
+            const float lc = __ldcg(p0 + c * cstride + 128 * 128 + 128 + row);
+            const float mc = __ldcg(p0 + c * cstride + 128 * 128 + row);
+            if (lc > 0.f) m_all = fmaxf(m_all, mc);
           }
+          float l_all = 0.f;
+          for (int32_t c = 0; c < u.n_chunks; ++c) {
+            const float lc = __ldcg(p0 + c * cstride + 128 * 128 + 128 + row);
+            const float mc = __ldcg(p0 + c * cstride + 128 * 128 + row);
+            if (lc > 0.f) l_all += lc * ex2(mc - m_all);
+          }
+          const float inv = 1.f / l_all;
+          __nv_bfloat16* dst = o + ((int64_t)(u.q_start + row) * n_q_heads + hq) * kD;
+#pragma unroll 1
+          for (int cc = 0; cc < kD / 32; ++cc) {
+            float acc[32];
+#pragma unroll
+            for (int x = 0; x < 32; ++x) acc[x] = 0.f;
+            for (int32_t c = 0; c < u.n_chunks; ++c) {
+              const float lc = __ldcg(p0 + c * cstride + 128 * 128 + 128 + row);
+              const float mc = __ldcg(p0 + c * cstride + 128 * 128 + row);
+              const float wgt = lc > 0.f ? ex2(mc - m_all) : 0.f;
+              const float* pc = p0 + c * cstride;
+#pragma unroll
+              for (int x = 0; x < 32; x += 4) {
+                const float4 v4 = __ldcg(reinterpret_cast<const float4*>(pc + ((cc * 8 + (x >> 2)) * 128 + row) * 4));
+                acc[x] = fmaf(wgt, v4.x, acc[x]);
+                acc[x + 1] = fmaf(wgt, v4.y, acc[x + 1]);
+                acc[x + 2] = fmaf(wgt, v4.z, acc[x + 2]);
+                acc[x + 3] = fmaf(wgt, v4.w, acc[x + 3]);
+              }
+            }
+            if (row_valid) {
+#pragma unroll
+              for (int x = 0; x < 32; x += 8) {
+                uint4 w;
+                w.x = pack_bf16(acc[x + 0] * inv, acc[x + 1] * inv);
+                w.y = pack_bf16(acc[x + 2] * inv, acc[x + 3] * inv);
+                w.z = pack_bf16(acc[x + 4] * inv, acc[x + 5] * inv);
+                w.w = pack_bf16(acc[x + 6] * inv, acc[x + 7] * inv);
+                *reinterpret_cast<uint4*>(dst + 32 * cc + x) = w;
+              }
+            }
+          }
+          if (lse && row_valid)
+            lse[(int64_t)hq * hdr->total_tokens + u.q_start + row] = (m_all + log2f(l_all)) * 0.6931471805599453f;
         }
       }
-      if (lse && row_valid)
-        lse[(int64_t)hq * hdr->total_tokens + qt.q_start + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+      u = nxt;
     }
+  }
   }
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) {
+  if (warp == kWarpMma) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
@@ -554,12 +747,12 @@ __device__ int32_t g_default_status;
 template <int BK>
 static purekv_status launch(const PrefillArgs& a, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             int32_t* status) {
-  const size_t smem = 1024 + 2 * 2 * (size_t)kBQ * 128 + 2 * (size_t)Cfg<BK>::kStages * 2 * BK * 128;
+  const size_t smem = 1024 + 2 * 2 * (size_t)kBQ * 128 + 2 * (size_t)Cfg<BK>::kStages * 2 * BK * 128 +
+                      (size_t)Cfg<BK>::kMeta * Cfg<BK>::kMaskBytes;
   PK_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  const int32_t G = a.n_q_heads / a.n_kv_heads;
-  dim3 grid((unsigned)((int64_t)a.info->n_qtiles * a.n_kv_heads * ((G + 1) / 2)));
-  prefill_tc_kernel<BK><<<grid, kThreads, smem, a.stream>>>(mq, mk, mv, (__nv_bfloat16*)a.o, a.lse,
-                                                            (const uint8_t*)a.plan, a.n_q_heads, a.n_kv_heads,
+  dim3 grid((unsigned)a.info->n_ctas);
+  prefill_tc_kernel<BK><<<grid, kThreads, smem, a.stream>>>(mq, mk, mv, (__nv_bfloat16*)a.o, a.lse, (uint8_t*)a.plan,
+                                                            (float*)a.ws, a.n_q_heads, a.n_kv_heads,
                                                             a.scale * 1.4426950408889634f, status);
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
@@ -571,6 +764,7 @@ purekv_status launch_prefill_tc(const PrefillArgs& a) {
   using namespace tc;
   PK_REQUIRE(a.info->tile_q == kBQ && (a.info->tile_k == 64 || a.info->tile_k == 128) && a.head_dim == kD,
              PUREKV_ERR_UNSUPPORTED, "tensor-core prefill needs tile_q 128, tile_k 64/128, head_dim 128");
+  PK_REQUIRE(a.info->n_ctas >= 1 && a.info->n_units >= 1, PUREKV_ERR_INVALID_ARG, "plan holds no schedule");
   const int64_t T = a.batch->total_tokens;
   CUtensorMap mq, mk, mv;
   purekv_status st;

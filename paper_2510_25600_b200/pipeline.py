@@ -41,10 +41,12 @@ class PureKVPipeline:
         params_dense = P.st_params(mask)
         params_dense.flags |= P.FLAG_DENSE_CAUSAL
         self.params_dense, self.params_st = params_dense, P.st_params(mask)
-        self.plan_buf_dense = torch.empty(max(1, P.purekv_plan_bytes(self.batch, params_dense, self.code, head_dim)),
+        hh = (n_q_heads, n_kv_heads)
+        self.plan_buf_dense = torch.empty(max(1, P.purekv_plan_bytes(self.batch, params_dense, self.code, head_dim, *hh)),
                                           dtype=torch.uint8, device=dev)
-        self.plan_buf_st = torch.empty(max(1, P.purekv_plan_bytes(self.batch, self.params_st, self.code, head_dim)),
+        self.plan_buf_st = torch.empty(max(1, P.purekv_plan_bytes(self.batch, self.params_st, self.code, head_dim, *hh)),
                                        dtype=torch.uint8, device=dev)
+        self.prefill_ws = None
         self.o = torch.empty((n_layers, t, n_q_heads, head_dim), dtype=dtype, device=dev)
         self.c = torch.empty((len(self.scored), n_kv_heads, t), dtype=torch.float32, device=dev)
         self.score_ws = torch.empty(P.purekv_score_ws_bytes(self.batch, window, n_q_heads), dtype=torch.uint8, device=dev)
@@ -58,12 +60,17 @@ class PureKVPipeline:
         self.launches_per_step = n_layers + 2 * len(self.scored) + 2 + 1   # prefill, score (2 kernels), select (2), compact
 
     def build_plans(self) -> None:
-        self.plan_dense = P.purekv_plan_build(self.batch, self.params_dense, self.code, self.d, self.plan_buf_dense)
-        self.plan_st = P.purekv_plan_build(self.batch, self.params_st, self.code, self.d, self.plan_buf_st)
+        self.plan_dense = P.purekv_plan_build(self.batch, self.params_dense, self.code, self.d, self.h, self.hkv,
+                                              self.plan_buf_dense)
+        self.plan_st = P.purekv_plan_build(self.batch, self.params_st, self.code, self.d, self.h, self.hkv,
+                                           self.plan_buf_st)
+        need = max(16, self.plan_dense.info.ws_bytes, self.plan_st.info.ws_bytes)
+        if self.prefill_ws is None or self.prefill_ws.numel() < need:
+            self.prefill_ws = torch.empty(need, dtype=torch.uint8, device="cuda")
 
     def prefill_layer(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor) -> None:
         plan = self.plan_dense if layer <= self.clie else self.plan_st
-        P.purekv_st_sparse_prefill(q, k, v, self.batch, plan, out=self.o[layer], status=self.status)
+        P.purekv_st_sparse_prefill(q, k, v, self.batch, plan, out=self.o[layer], status=self.status, ws=self.prefill_ws)
 
     def run_device(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, events=None) -> None:
         """q [n_layers,T,H,d], k,v [kv_layers,T,H_kv,d] on the GPU.  Results in self.o / idx / k_c / v_c.

@@ -34,12 +34,13 @@ def device_batch(wl: inputs.Workload):
     return pk().Batch(b.seq_lens, b.n_prefix, b.n_frames)
 
 
-def gpu_prefill(wl: inputs.Workload, x: dict, want_lse: bool = True, mask=None):
+def gpu_prefill(wl: inputs.Workload, x: dict, want_lse: bool = True, mask=None, n_ctas: int = 0):
     P = pk()
     db = device_batch(wl)
     q, k, v = (upload(x, n, wl.dtype) for n in "qkv")
     code = P.BF16 if wl.dtype == "bf16" else P.FP32
-    plan = P.purekv_plan_build(db, P.st_params(mask or wl.mask), code, wl.head_dim)
+    plan = P.purekv_plan_build(db, P.st_params(mask or wl.mask), code, wl.head_dim, wl.n_q_heads, wl.n_kv_heads,
+                               n_ctas=n_ctas)
     lse = torch.full((wl.n_q_heads, db.total_tokens), float("nan"), dtype=torch.float32, device="cuda") if want_lse else None
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     out = torch.full_like(q, float("nan"))
@@ -48,8 +49,8 @@ def gpu_prefill(wl: inputs.Workload, x: dict, want_lse: bool = True, mask=None):
     return out, lse, plan
 
 
-def check_prefill(wl: inputs.Workload, x: dict, rows=None, heads=None, mask=None):
-    out, lse, plan = gpu_prefill(wl, x, mask=mask)
+def check_prefill(wl: inputs.Workload, x: dict, rows=None, heads=None, mask=None, n_ctas: int = 0):
+    out, lse, plan = gpu_prefill(wl, x, mask=mask, n_ctas=n_ctas)
     b = wl.batch
     ref, ref_lse = po.prefill(x["q"], x["k"], x["v"], b.cu_seqlens, b.n_prefix, b.n_frames,
                               po.mask_params(mask or wl.mask), rows=rows, heads=heads)

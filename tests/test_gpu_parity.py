@@ -37,6 +37,34 @@ def test_prefill_tensor_core_kernel(tile, mask_kw):
     gc.check_prefill(wl, inputs.make_qkv(wl, 0))
 
 
+@pytest.mark.parametrize("tile", [64, 128])
+@pytest.mark.parametrize("H,Hkv,n_ctas", [(3, 1, 0), (7, 1, 5), (4, 2, 600), (5, 1, 300), (2, 2, 1)])
+def test_prefill_tensor_core_schedules(tile, H, Hkv, n_ctas):
+    # odd groups (a single-head unit per group), key lists split into chunks that are merged through the
+    # workspace (many CTAs, little work each), everything on one CTA
+    wl = make_wl("bf16", H, Hkv, 128, [37, 0, 5], [5, 3, 1], [29, 300, 0], 9, 11, tile)
+    x = inputs.make_qkv(wl, 0)
+    for mask in (wl.mask, inputs.STMask(9, 11, tile=tile, dense_causal=True)):
+        err, plan = gc.check_prefill(wl, x, mask=mask, n_ctas=n_ctas)
+        if n_ctas >= 300:
+            assert plan.info.max_chunks > 1 and plan.info.ws_bytes > 0
+
+
+def test_prefill_plan_is_reusable_after_split_merges():
+    # the merge counters in the plan return to zero: the same plan gives the same bits launch after launch
+    P = gc.pk()
+    wl = make_wl("bf16", 4, 2, 128, [10], [6], [200], 8, 8, 64)
+    x = inputs.make_qkv(wl, 0)
+    db = gc.device_batch(wl)
+    q, k, v = (gc.upload(x, n, "bf16") for n in "qkv")
+    plan = P.purekv_plan_build(db, P.st_params(wl.mask), P.BF16, 128, 4, 2, n_ctas=500)
+    assert plan.info.max_chunks > 1
+    outs = [P.purekv_st_sparse_prefill(q, k, v, db, plan).clone() for _ in range(3)]
+    torch.cuda.synchronize()
+    assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+    assert torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
+
+
 def test_prefill_tensor_core_single_token_and_tiny_requests():
     wl = make_wl("bf16", 2, 1, 128, [1, 0, 3], [0, 1, 0], [0, 0, 126], 1, 1, 128)
     gc.check_prefill(wl, inputs.make_qkv(wl, 0))
@@ -158,7 +186,7 @@ def test_empty_inputs_and_bad_arguments():
     db = P.Batch([], [], [])
     bud = P.Budget(db, 4, 0.5)
     z = torch.empty((0, 2, 128), dtype=torch.bfloat16, device="cuda")
-    plan = P.purekv_plan_build(db, P.st_params(inputs.STMask(4, 4, tile=64)), P.BF16, 128)
+    plan = P.purekv_plan_build(db, P.st_params(inputs.STMask(4, 4, tile=64)), P.BF16, 128, 2, 2)
     P.purekv_st_sparse_prefill(z, z, z, db, plan)
     c = P.purekv_lowlayer_score(z, z, db, 4)
     idx = P.purekv_select_topk(c, z[None], db, bud)
@@ -167,7 +195,7 @@ def test_empty_inputs_and_bad_arguments():
     db = P.Batch([40], [0], [0])
     q = torch.zeros((40, 3, 128), dtype=torch.bfloat16, device="cuda")
     kv = torch.zeros((40, 2, 128), dtype=torch.bfloat16, device="cuda")
-    plan = P.purekv_plan_build(db, P.st_params(inputs.STMask(4, 4, tile=64)), P.BF16, 128)
+    plan = P.purekv_plan_build(db, P.st_params(inputs.STMask(4, 4, tile=64)), P.BF16, 128, 2, 2)
     with pytest.raises(P.PureKVError) as e:
         P.purekv_st_sparse_prefill(q, kv, kv, db, plan)          # 3 query heads, 2 KV heads
     assert e.value.status == P.ERR_INVALID_ARG

@@ -34,20 +34,82 @@ def test_budget_matches_oracle_rule():
 
 def parse_plan(buf: np.ndarray):
     raw = buf.tobytes()
-    magic, tq, tk, nq, T, ne, nm, oq, oo, oe, om, wpr = struct.unpack_from("<Iiiiqqqqqqqi", raw, 0)
-    assert magic == 0x504B5632
+    (magic, tq, tk, nq, T, ne, nm, oq, oo, oe, om, wpr, n_ctas, n_units, n_counters, o_cta, o_units, o_counters, H, Hkv,
+     part_slots) = struct.unpack_from("<Iiiiqqqqqqqiiiiqqqiiq", raw, 0)
+    assert magic == 0x504B5633
     qt = np.frombuffer(raw, dtype=np.int32, count=nq * 8, offset=oq).reshape(nq, 8)
     order = np.frombuffer(raw, dtype=np.int32, count=nq, offset=oo)
     entries = np.frombuffer(raw, dtype=np.int32, count=2 * ne, offset=oe).reshape(ne, 2)
     masks = np.frombuffer(raw, dtype=np.uint32, count=nm, offset=om)
-    return dict(tq=tq, tk=tk, nq=nq, T=T, qt=qt, order=order, entries=entries, masks=masks, wpr=wpr)
+    cta_off = np.frombuffer(raw, dtype=np.int32, count=n_ctas + 1 if n_units else 0, offset=o_cta)
+    units = np.frombuffer(raw, dtype=np.int32, count=12 * n_units, offset=o_units).reshape(n_units, 12)
+    counters = np.frombuffer(raw, dtype=np.int32, count=n_counters, offset=o_counters)
+    return dict(tq=tq, tk=tk, nq=nq, T=T, qt=qt, order=order, entries=entries, masks=masks, wpr=wpr, n_ctas=n_ctas,
+                cta_off=cta_off, units=units, counters=counters, H=H, Hkv=Hkv, part_slots=part_slots)
 
 
-def check_plan(batch: inputs.Batch, mask: inputs.STMask, dtype, head_dim):
+def check_schedule(p, info, H, Hkv, n_ctas):
+    """The persistent kernel's schedule: every (query tile, head pair, list entry) is covered exactly once, chunks
+    of a split list are contiguous and complete, workspace slots and merge counters do not collide, and no CTA
+    carries much more than its share."""
+    G = H // Hkv
+    n_pairs = Hkv * ((G + 1) // 2)
+    units, cta_off = p["units"], p["cta_off"]
+    assert p["n_ctas"] == n_ctas == info.n_ctas and len(units) == info.n_units == cta_off[-1] and cta_off[0] == 0
+    assert (np.diff(cta_off) >= 0).all() and (p["counters"] == 0).all()
+    by_start = {int(r[0]): r for r in p["qt"]}
+    covered = {}
+    chunks = {}
+    for u in units:
+        q_start, q_rows, req_start, eb, ec, pair, chunk, nch, part_base, counter_base = (int(x) for x in u[:10])
+        qt = by_start[q_start]
+        assert q_rows == qt[1] and req_start == qt[2] and 0 <= pair < n_pairs and 0 <= chunk < nch and ec >= 1
+        assert qt[4] <= eb and eb + ec <= qt[4] + qt[5]
+        for e in range(eb, eb + ec):
+            assert (q_start, pair, e) not in covered
+            covered[(q_start, pair, e)] = chunk
+        chunks.setdefault((q_start, pair), []).append((chunk, eb, ec, nch, part_base, counter_base))
+    assert len(covered) == n_pairs * int(p["qt"][:, 5].sum())
+    slots_used, counters_used = set(), set()
+    for (q_start, pair), lst in chunks.items():
+        lst.sort()
+        qt = by_start[q_start]
+        nch = lst[0][3]
+        assert [c[0] for c in lst] == list(range(nch)) and all(c[3] == nch for c in lst)
+        assert lst[0][1] == qt[4] and lst[-1][1] + lst[-1][2] == qt[4] + qt[5]
+        assert all(a[1] + a[2] == b[1] for a, b in zip(lst, lst[1:]))          # contiguous, in order
+        if nch == 1:
+            assert lst[0][4] == -1 and lst[0][5] == -1
+        else:
+            assert len({c[4] for c in lst}) == 1 and len({c[5] for c in lst}) == 1
+            if pair == 0:
+                for c in range(nch):
+                    for hq in range(H):
+                        slot = (lst[0][4] + c) * H + hq
+                        assert slot not in slots_used and 0 <= slot < p["part_slots"]
+                        slots_used.add(slot)
+                for hq in range(H):
+                    cnt = lst[0][5] + hq
+                    assert cnt not in counters_used and 0 <= cnt < len(p["counters"])
+                    counters_used.add(cnt)
+    assert len(slots_used) == p["part_slots"] and len(counters_used) == len(p["counters"])
+    assert info.ws_bytes == p["part_slots"] * (128 * 128 + 256) * 4
+    overhead = 2 if p["tk"] >= 128 else 3
+    load = np.array([sum(int(u[4]) + overhead for u in units[a:b]) for a, b in zip(cta_off[:-1], cta_off[1:])])
+    if len(units) >= 4 * n_ctas:
+        assert load.max() <= 1.25 * load.mean() + 4
+    return load
+
+
+def check_plan(batch: inputs.Batch, mask: inputs.STMask, dtype, head_dim, H=4, Hkv=2, n_ctas=0):
     b = pk.Batch(batch.seq_lens, batch.n_prefix, batch.n_frames, device=None)
-    buf, info = pk.purekv_plan_build_host(b, pk.st_params(mask), dtype, head_dim)
-    assert pk.purekv_plan_bytes(b, pk.st_params(mask), dtype, head_dim) == info.bytes_used == len(buf)
+    buf, info = pk.purekv_plan_build_host(b, pk.st_params(mask), dtype, head_dim, H, Hkv, n_ctas)
+    assert pk.purekv_plan_bytes(b, pk.st_params(mask), dtype, head_dim, H, Hkv, n_ctas) == info.bytes_used == len(buf)
     p = parse_plan(buf)
+    if info.tile_q == 128:
+        check_schedule(p, info, H, Hkv, n_ctas or 148)
+    else:
+        assert info.n_ctas == 0 and info.n_units == 0 and info.ws_bytes == 0
     tq, tk, wpr = p["tq"], p["tk"], p["wpr"]
     assert (tq, tk) == (info.tile_q, info.tile_k) and wpr == max(1, tk // 32)
     mp = po.mask_params(mask)
@@ -115,8 +177,10 @@ def test_plan_matches_oracle_mask(tile, mask_kw):
 def test_plan_for_tensor_core_shapes_and_workload_counts():
     batch = inputs.make_batch([64, 3], [5, 2], [64, 130], 12, 12)
     for tile in (64, 128):
-        info = check_plan(batch, inputs.STMask(12, 12, tile=tile), pk.BF16, 128)
-        assert info.tile_q == 128 and info.tile_k == tile
+        for H, Hkv, n_ctas in ((4, 2, 0), (7, 1, 5), (6, 2, 3), (2, 2, 400)):
+            info = check_plan(batch, inputs.STMask(12, 12, tile=tile), pk.BF16, 128, H, Hkv, n_ctas)
+            assert info.tile_q == 128 and info.tile_k == tile
+        assert info.max_chunks > 1                       # many CTAs, little work each: the long text lists are split
     # cfg 0: pair count of the paper's mask (closed form) and the block density quoted for 16-tiles
     wl = inputs.workload(0)
     info = check_plan(wl.batch, wl.mask, pk.FP32, 64)
@@ -128,19 +192,21 @@ def test_plan_pair_counts_on_the_large_workloads():
     for cfg, pairs in [(1, 783264), (2, 4148800), (3, 41042944)]:
         wl = inputs.workload(cfg)
         b = pk.Batch(wl.batch.seq_lens, wl.batch.n_prefix, wl.batch.n_frames, device=None)
-        _, info = pk.purekv_plan_build_host(b, pk.st_params(wl.mask), pk.BF16, 128)
+        buf, info = pk.purekv_plan_build_host(b, pk.st_params(wl.mask), pk.BF16, 128, wl.n_q_heads, wl.n_kv_heads)
         assert info.pairs_kept == pairs
         assert info.tile_q == 128 and 0 < info.tiles_kept < info.tiles_causal
+        load = check_schedule(parse_plan(buf), info, wl.n_q_heads, wl.n_kv_heads, 148)
+        assert load.max() <= 1.2 * load.mean() + 4
 
 
 def test_argument_errors():
     b = pk.Batch([10], [2], [1], device=None)
     with pytest.raises(pk.PureKVError) as e:
-        pk.purekv_plan_build_host(b, pk.st_params(inputs.STMask(4, 4)), pk.FP32, 64)     # 2 + 16 > 10
+        pk.purekv_plan_build_host(b, pk.st_params(inputs.STMask(4, 4)), pk.FP32, 64, 2, 1)     # 2 + 16 > 10
     assert e.value.status == pk.ERR_INVALID_ARG
     b = pk.Batch([30], [2], [1], device=None)
     with pytest.raises(pk.PureKVError) as e:
-        pk.purekv_plan_build_host(b, pk.st_params(inputs.STMask(4, 4, tile=48)), pk.FP32, 64)
+        pk.purekv_plan_build_host(b, pk.st_params(inputs.STMask(4, 4, tile=48)), pk.FP32, 64, 2, 1)
     assert e.value.status == pk.ERR_UNSUPPORTED
     with pytest.raises(pk.PureKVError):
         pk.purekv_budget(-1, 4, 0.5)
