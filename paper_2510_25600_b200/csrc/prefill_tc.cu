@@ -13,8 +13,9 @@
 //               so the tensor pipe works on one slot while the other slot's rows are in softmax.
 //   warps 0-7   one thread per query row of a slot (registers raised with setmaxnreg at the expense of
 //               warps 8-11): the row of S from TMEM into registers, the
-//               tile's predicate (none / causal / bit mask), online softmax in the log2 domain with lazy
-//               rescaling of O, bf16 P written over S; at the end of a unit either the normalised output
+//               tile's predicate (none / causal / bit mask), online softmax in the log2 domain against a
+//               reference that moves only when exp2 would overflow (then O is rescaled), a share of the
+//               exponentials on the FMA pipe, bf16 P written over S; at the end of a unit either the normalised output
 //               (whole list in one unit) or an unnormalised fp32 partial result plus (max, sum) per row
 //               into the workspace.  The chunk of a split list that finishes last (a counter in the plan)
 //               combines the partial results in chunk order, so the result does not depend on timing.
@@ -35,7 +36,7 @@ constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // per-thread registers afte
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 256;
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
-constexpr float kRescaleThreshold = 8.0f;                        // log2 units
+constexpr int kPolyOf8 = 2;  // of every 8 pairs of exponentials, how many are computed on the FMA pipe
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -128,6 +129,25 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
       : "memory");
 }
 
+// The same with the 64-bit shared-memory descriptors given as (low, high) words: only the low word (start
+// address) changes from one K step to the next, so the issuing thread spends one add per operand.
+__device__ __forceinline__ void mma_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n .reg .b64 da, db;\n setp.ne.b32 p, %6, 0;\n mov.b64 da, {%1, %2};\n mov.b64 db, {%3, %4};\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n}\n" ::"r"(d_tmem),
+      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n .reg .pred p;\n .reg .b64 db;\n setp.ne.b32 p, %5, 0;\n mov.b64 db, {%2, %3};\n"
+      " tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 #define PK_R8(r, o) "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]), "=r"(r[o + 6]), "=r"(r[o + 7])
 #define PK_W8(r, o) "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), "r"(r[o + 6]), "r"(r[o + 7])
 
@@ -173,6 +193,30 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// 2^x for a pair of values on the FMA pipe (the MUFU unit is the scarce one): round to the nearest integer n with
+// the 1.5 * 2^23 trick, a cubic for 2^f on f = x - n in [-0.5, 0.5] (relative error 7.5e-5, below bf16 rounding),
+// then n is added into the exponent field.  x <= 0 here; inputs below -126 (and -inf) give 2^-126, which is
+// nothing beside the row's largest term (2^0 .. 2^-8 after lazy rescaling).
+__device__ __forceinline__ float2 exp2_poly2(float2 x) {
+  const float kMagic = 12582912.f;  // 1.5 * 2^23
+  x.x = fmaxf(x.x, -126.f);
+  x.y = fmaxf(x.y, -126.f);
+  const float2 r = __fadd2_rn(x, make_float2(kMagic, kMagic));
+  const float2 f = __ffma2_rn(__fadd2_rn(r, make_float2(-kMagic, -kMagic)), make_float2(-1.f, -1.f), x);  // x - n
+  float2 p = __ffma2_rn(make_float2(0.05517115443944931f, 0.05517115443944931f), f,
+                        make_float2(0.2426101416349411f, 0.2426101416349411f));
+  p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
+  p = __ffma2_rn(p, f, make_float2(0.9999281167984009f, 0.9999281167984009f));
+  // 2^n: the integer sits in the low mantissa bits of r; shifted into the exponent field it adds to p's exponent
+  p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(r.x) << 23));
+  p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(r.y) << 23));
+  return p;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
@@ -216,7 +260,7 @@ struct __align__(8) Barriers {
   uint64_t k_full[ST], k_empty[ST], v_full[ST], v_empty[ST];
   uint64_t m_full[MR];     // producer -> softmax: class word (and bit mask) of a tile are in place
   uint64_t s_full[2][SB];  // MMA -> softmax: S of (slot, buffer) is complete
-  uint64_t p_full[2][SB];  // softmax -> MMA: P written (and O rescaled) by all 128 row threads
+  uint64_t p_full[2][SB];  // softmax -> MMA: P written (and O rescaled) by the slot's four row warps
   uint64_t o_done[2];      // one completion per P.V product of the slot
   uint64_t o_final[2];     // one completion per unit, after the slot's last P.V product
   uint64_t rows_sync[2];   // the 128 row threads of a slot meet here around the merge-counter update
@@ -274,7 +318,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     for (int sl = 0; sl < 2; ++sl) {
       for (int b = 0; b < SB; ++b) {
         mbar_init(smem_u32(&bars.s_full[sl][b]), 1);
-        mbar_init(smem_u32(&bars.p_full[sl][b]), 128);
+        mbar_init(smem_u32(&bars.p_full[sl][b]), 4);
       }
       mbar_init(smem_u32(&bars.o_done[sl]), 1);
       mbar_init(smem_u32(&bars.o_final[sl]), 1);
@@ -378,19 +422,25 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       uint32_t tq[2] = {0, 0};         // S products issued per slot, over all units
       uint32_t tp[2] = {0, 0};         // P.V products issued per slot, over all units
       int32_t nt = 0, n_slots = 0;
+      // Descriptor words.  High word: stride between 8-row groups 1024 B, descriptor version 1, 128-byte swizzle.
+      // Low word: start address / 16 and the leading-dimension offset / 16 (used by the MN-major V operand only).
+      constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t q_lo0 = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
+      const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
+      const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((kPanelKV >> 4) << 16);
       // S(slot, n) = Q_slot K_n^T; the last slot to read K_n releases its stage
       auto issue_qk = [&](int32_t sl, int32_t n) -> bool {
         const uint32_t it = it_base + (uint32_t)n;
         const uint32_t s = it % ST, b = tq[sl] % SB;
-        if (!mbar_wait(smem_u32(&bars.k_full[s]), (it / ST) & 1u, abort_flag)) return false;
+        // the stage was already awaited for slot 0 of the same tile
+        if (sl == 0 && !mbar_wait(smem_u32(&bars.k_full[s]), (it / ST) & 1u, abort_flag)) return false;
         tc_fence_after();
         const uint32_t d_addr = tmem + sl * 128 + b * BK;
+        const uint32_t q_lo = q_lo0 + (uint32_t)sl * (kTileQ >> 4), k_lo = k_lo0 + s * (kTileKV >> 4);
 #pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks) {
-          const uint32_t qoff = sl * kTileQ + (ks >> 2) * kPanelQ + (ks & 3) * 32;
-          const uint32_t koff = s * kTileKV + (ks >> 2) * kPanelKV + (ks & 3) * 32;
-          mma_ss(d_addr, smem_desc(sQ + qoff, 16, 1024), smem_desc(sK + koff, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
-        }
+        for (int ks = 0; ks < kD / 16; ++ks)
+          mma_ss_lh(d_addr, q_lo + (ks >> 2) * (kPanelQ >> 4) + (ks & 3) * 2, kDescHi,
+                    k_lo + (ks >> 2) * (kPanelKV >> 4) + (ks & 3) * 2, kDescHi, idesc_qk, ks > 0 ? 1u : 0u);
         if (sl == n_slots - 1) {
           tc_commit(smem_u32(&bars.k_empty[s]));
           if (n == nt - 1) tc_commit(smem_u32(&bars.q_empty));  // the unit's last read of Q
@@ -403,19 +453,23 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       auto issue_pv = [&](int32_t sl, int32_t n) -> bool {
         const uint32_t it = it_base + (uint32_t)n;
         const uint32_t s = it % ST, b = tp[sl] % SB;
-        if (!mbar_wait(smem_u32(&bars.v_full[s]), (it / ST) & 1u, abort_flag)) return false;
+        if (sl == 0 && !mbar_wait(smem_u32(&bars.v_full[s]), (it / ST) & 1u, abort_flag)) return false;
         // P of the unit's first tile also implies that the previous unit's output has left TMEM
         if (!mbar_wait(smem_u32(&bars.p_full[sl][b]), (tp[sl] / SB) & 1u, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t p_addr = tmem + sl * 128 + b * BK;
+        const uint32_t p_addr = tmem + sl * 128 + b * BK, o_addr = tmem + kColO + sl * 128;
+        // B = V tile, MN-major: per K step 16 key rows (2 groups of 8, 1024 B apart) x 128 dims (2 panels)
+        const uint32_t v_lo = v_lo0 + s * (kTileKV >> 4);
+        if (n > 0) {
 #pragma unroll
-        for (int ks = 0; ks < BK / 16; ++ks) {
-          // B = V tile, MN-major: 16 key rows (2 groups of 8, SBO 1024) x 128 dims (2 panels, LBO)
-          const uint64_t bdesc = smem_desc(sV + s * kTileKV + ks * 2048, kPanelKV, 1024);
-          mma_ts(tmem + kColO + sl * 128, p_addr + ks * 8, bdesc, idesc_pv, (n > 0 || ks > 0) ? 1u : 0u);
+          for (int ks = 0; ks < BK / 16; ++ks) mma_ts_lh(o_addr, p_addr + ks * 8, v_lo + ks * (2048 >> 4), kDescHi, idesc_pv, 1u);
+        } else {
+#pragma unroll
+          for (int ks = 0; ks < BK / 16; ++ks)
+            mma_ts_lh(o_addr, p_addr + ks * 8, v_lo + ks * (2048 >> 4), kDescHi, idesc_pv, ks > 0 ? 1u : 0u);
         }
         if (sl == n_slots - 1) tc_commit(smem_u32(&bars.v_empty[s]));
-        tc_commit(smem_u32(&bars.o_done[sl]));
+        if (SB > 1) tc_commit(smem_u32(&bars.o_done[sl]));
         if (n == nt - 1) tc_commit(smem_u32(&bars.o_final[sl]));
         ++tp[sl];
         return true;
@@ -489,7 +543,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       const int32_t hq = g * G + 2 * pr + sl;
       const bool row_valid = row < u.q_rows;
       const int32_t i_rel = u.q_start - u.req_start + row;
-      float m_ref = -INFINITY, l_sum = 0.f;
+      float m_ref = 0.f, l_sum = 0.f;
       for (int32_t n = 0; n < nt; ++n) {
         const uint32_t it = it_base + (uint32_t)n, ms = it % MR, b = t % SB;
         if (!wait_w(smem_u32(&bars.m_full[ms]), (it / MR) & 1u)) { ok = false; break; }
@@ -520,72 +574,108 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         if (!wait_w(smem_u32(&bars.s_full[sl][b]), (t / SB) & 1u)) { ok = false; break; }
         tc_fence_after();
         const uint32_t s_addr = t_lane + sl * 128 + b * BK;
-        // the whole row of S into registers
-        uint32_t r[BK];
-        tmem_ld32_at<0>(s_addr, r);
-        tmem_ld32_at<32>(s_addr + 32, r);
-        if constexpr (BK == 128) {
-          tmem_ld32_at<64>(s_addr + 64, r);
-          tmem_ld32_at<96>(s_addr + 96, r);
-        }
-        tc_wait_ld();
-        if (cls != kTileFull) {
+        // Fast path: exponentials against the row's standing reference m_ref, no maximum taken.  Softmax does not depend
+        // on the reference, and fp32 / bf16 carry 8 exponent bits, so the reference (0 at the start of a unit) only has
+        // to keep exp2 in range: it moves when a tile overflows, or when everything kept so far has underflowed; those
+        // tiles take the exact path below.
+        uint32_t pk[BK / 2];
+        float l_tile = 0.f;
+        bool exact = false;
+        {
+          uint32_t r[BK];
+          tmem_ld32_at<0>(s_addr, r);
+          tmem_ld32_at<32>(s_addr + 32, r);
+          if constexpr (BK == 128) {
+            tmem_ld32_at<64>(s_addr + 64, r);
+            tmem_ld32_at<96>(s_addr + 96, r);
+          }
+          tc_wait_ld();
+          float2 ls2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+          const float2 sc2 = make_float2(scale_log2, scale_log2), mm2 = make_float2(-m_ref, -m_ref);
 #pragma unroll
           for (int c = 0; c < BK / 32; ++c) {
-            if (__any_sync(0xffffffffu, keep[c] != 0xFFFFFFFFu)) {  // warp-uniform: skip chunks every row keeps
+            if (cls != kTileFull && __any_sync(0xffffffffu, keep[c] != 0xFFFFFFFFu)) {  // warp-uniform
 #pragma unroll
               for (int x = 0; x < 32; ++x)
-                if (!((keep[c] >> x) & 1u)) r[32 * c + x] = 0xFF800000u;  // -inf: drops out of max and exp
+                if (!((keep[c] >> x) & 1u)) r[32 * c + x] = 0xFF800000u;  // -inf: exp2 gives 0
+            }
+#pragma unroll
+            for (int x = 0; x < 32; x += 2) {
+              const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[32 * c + x]), __uint_as_float(r[32 * c + x + 1])), sc2, mm2);
+              // kPolyOf8 of every 8 column pairs take the polynomial on the FMA pipe, the rest the MUFU unit
+              const float2 pp = ((x >> 1) & 7) < kPolyOf8 ? exp2_poly2(a) : make_float2(ex2(a.x), ex2(a.y));
+              ls2[(x >> 1) & 1] = __fadd2_rn(ls2[(x >> 1) & 1], pp);
+              pk[16 * c + (x >> 1)] = pack_bf16(pp.x, pp.y);
             }
           }
+          l_tile = (ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y);
+          bool has_kept = cls == kTileFull;
+#pragma unroll
+          for (int c = 0; c < BK / 32; ++c) has_kept |= keep[c] != 0u;
+          // overflow (inf or NaN), or kept keys and still nothing representable: redo against the true maximum
+          exact = __any_sync(0xffffffffu, !(l_tile <= 1.0e30f) || (has_kept && l_sum + l_tile < 1.0e-30f));
         }
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        if (exact) {
+          // Exact path (rare): re-reference the row; O and the running sum are rescaled.  S is still intact in TMEM
+          // (P has not been stored yet).
+          float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int x = 0; x < BK; ++x) mx[x & 3] = fmaxf(mx[x & 3], __uint_as_float(r[x]));
-        const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
-        // lazy rescale: move the reference only when the maximum grew by more than the threshold
-        float m_use = m_ref;
-        const bool grow = m_tile > m_ref + kRescaleThreshold || (m_ref == -INFINITY && m_tile > -INFINITY);
-        if (grow) m_use = m_tile;
-        const float m_sub = m_use == -INFINITY ? 0.f : m_use;
-        // rescale O and the running sum where the reference moved (warp-uniform decision)
-        const float alpha = grow ? (m_ref == -INFINITY ? 0.f : ex2(m_ref - m_use)) : 1.f;
-        if (n > 0 && __any_sync(0xffffffffu, grow)) {
-          // O must be quiescent: with one S buffer, S of tile n was issued behind P.V of tile n-1, so it is;
-          // with two, S of tile n only implies P.V of tile n-2 (o_done is then in phase t-1 or t).
-          if (SB > 1 && !wait_w(smem_u32(&bars.o_done[sl]), (t - 1u) & 1u)) { ok = false; break; }
-          tc_fence_after();
-#pragma unroll
-          for (int c = 0; c < kD / 32; ++c) {
-            uint32_t tt[32];
-            tmem_ld32(t_lane + kColO + sl * 128 + 32 * c, tt);
+          for (int c = 0; c < BK / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld32(s_addr + 32 * c, r);
             tc_wait_ld();
 #pragma unroll
-            for (int x = 0; x < 32; ++x) tt[x] = __float_as_uint(__uint_as_float(tt[x]) * alpha);
-            tmem_st32(t_lane + kColO + sl * 128 + 32 * c, tt);
+            for (int x = 0; x < 32; ++x)
+              if ((keep[c] >> x) & 1u) mx[x & 3] = fmaxf(mx[x & 3], __uint_as_float(r[x]));
           }
-        }
-        // probabilities -> bf16 P over the S columns, row sum in fp32
-        float2 ls2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-        const float2 sc2 = make_float2(scale_log2, scale_log2), mm2 = make_float2(-m_sub, -m_sub);
+          const float m_tile = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;  // scale > 0
+          // the new reference: the larger of this tile's maximum and the log-sum of what has been accumulated
+          const float m_eff = l_sum > 0.f ? m_ref + log2f(l_sum) : -INFINITY;
+          const float m_max = fmaxf(m_eff, m_tile);
+          const float m_new = m_max == -INFINITY ? m_ref : m_max;  // nothing kept yet and nothing accumulated: stay
+          const float alpha = l_sum > 0.f ? ex2(m_ref - m_new) : 1.f;  // with l_sum == 0 every earlier P was 0, so O is 0
+          const float m_sub = m_new;
+          if (n > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+            // O must be quiescent: with one S buffer, S of tile n was issued behind P.V of tile n-1, so it is;
+            // with two, S of tile n only implies P.V of tile n-2 (o_done is then in phase t-1 or t).
+            if (SB > 1 && !wait_w(smem_u32(&bars.o_done[sl]), (t - 1u) & 1u)) { ok = false; break; }
+            tc_fence_after();
 #pragma unroll
-        for (int c = 0; c < BK / 32; ++c) {
-          uint32_t pk[16];
+            for (int c = 0; c < kD / 32; ++c) {
+              uint32_t tt[32];
+              tmem_ld32(t_lane + kColO + sl * 128 + 32 * c, tt);
+              tc_wait_ld();
 #pragma unroll
-          for (int x = 0; x < 32; x += 2) {
-            const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[32 * c + x]), __uint_as_float(r[32 * c + x + 1])), sc2, mm2);
-            const float2 p = make_float2(ex2(a.x), ex2(a.y));
-            ls2[(x >> 1) & 1] = __fadd2_rn(ls2[(x >> 1) & 1], p);
-            pk[x >> 1] = pack_bf16(p.x, p.y);
+              for (int x = 0; x < 32; ++x) tt[x] = __float_as_uint(__uint_as_float(tt[x]) * alpha);
+              tmem_st32(t_lane + kColO + sl * 128 + 32 * c, tt);
+            }
           }
-          // P chunk c lands on S columns 16c..16c+15, which this thread has already consumed
-          tmem_st16(s_addr + 16 * c, pk);
+          float ls[2] = {0.f, 0.f};
+#pragma unroll
+          for (int c = 0; c < BK / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld32(s_addr + 32 * c, r);
+            tc_wait_ld();
+#pragma unroll
+            for (int x = 0; x < 32; x += 2) {
+              const float p0 = ((keep[c] >> x) & 1u) ? ex2(fmaf(__uint_as_float(r[x]), scale_log2, -m_sub)) : 0.f;
+              const float p1 = ((keep[c] >> (x + 1)) & 1u) ? ex2(fmaf(__uint_as_float(r[x + 1]), scale_log2, -m_sub)) : 0.f;
+              ls[(x >> 1) & 1] += p0 + p1;
+              pk[16 * c + (x >> 1)] = pack_bf16(p0, p1);
+            }
+          }
+          l_tile = ls[0] + ls[1];
+          l_sum *= alpha;
+          m_ref = m_new;
         }
-        l_sum = l_sum * alpha + ((ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y));
-        m_ref = m_use;
+        l_sum += l_tile;
+        // bf16 P over the first BK/2 columns of S, which this thread has consumed
+#pragma unroll
+        for (int c = 0; c < BK / 32; ++c) tmem_st16(s_addr + 16 * c, reinterpret_cast<const uint32_t(&)[16]>(pk[16 * c]));
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(smem_u32(&bars.p_full[sl][b]));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[sl][b]));  // one arrival per warp: 4 per slot
         ++t;
       }
       if (!ok) break;

@@ -65,6 +65,35 @@ def test_prefill_plan_is_reusable_after_split_merges():
     assert torch.equal(outs[0].view(torch.int16), outs[2].view(torch.int16))
 
 
+@pytest.mark.parametrize("tile", [64, 128])
+@pytest.mark.parametrize("kind", ["huge", "very_negative", "rising", "falling"])
+def test_prefill_tensor_core_extreme_logits(tile, kind):
+    # The kernel takes exponentials against a reference that only moves when a tile would overflow exp2 or when all
+    # kept terms have underflowed; these inputs force both moves (and the rescaling of O that goes with them).
+    wl = make_wl("bf16", 4, 2, 128, [20, 3], [4, 2], [150, 40], 6, 7, tile)
+    x = inputs.make_qkv(wl, 0)
+    T = wl.batch.total_tokens
+    u = np.zeros(128, dtype=np.float32)
+    u[:4] = 0.5                                              # unit vector, exactly representable
+    ramp = np.linspace(0.0, 1.0, T, dtype=np.float32)[:, None, None]
+    if kind == "huge":                                       # logits of several hundred either way
+        x["q"] = x["q"] * 40.0
+    elif kind == "very_negative":                            # every logit near -115 (log2 units)
+        x["k"] = x["k"] * 0.25 + 30.0 * u
+        x["q"] = x["q"] * 0.25 - 30.0 * u
+    elif kind == "rising":                                   # later keys score ever higher: the reference must move up often
+        x["k"] = x["k"] + 60.0 * ramp * u
+        x["q"] = x["q"] + 40.0 * u
+    else:                                                    # later keys score ever lower
+        x["k"] = x["k"] - 60.0 * ramp * u
+        x["q"] = x["q"] + 40.0 * u
+    for n in "qk":
+        bits = inputs.f32_to_bf16_bits(x[n])
+        x[n + "_bits"], x[n] = bits, inputs.bf16_bits_to_f32(bits)
+    gc.check_prefill(wl, x)
+    gc.check_prefill(wl, x, mask=inputs.STMask(6, 7, tile=tile, dense_causal=True), n_ctas=300)
+
+
 def test_prefill_tensor_core_single_token_and_tiny_requests():
     wl = make_wl("bf16", 2, 1, 128, [1, 0, 3], [0, 1, 0], [0, 0, 126], 1, 1, 128)
     gc.check_prefill(wl, inputs.make_qkv(wl, 0))
