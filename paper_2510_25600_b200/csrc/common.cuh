@@ -70,8 +70,10 @@ struct QTile {
   int32_t entry_count;
   int32_t pad[2];
 };
-// entry.x = (key tile index inside the request << 2) | TileClass;  key tile kt covers request
-// positions kt*tile_k .. kt*tile_k + tile_k - 1.
+// entry.x = (key tile index inside the request << 4) | (half mask << 2) | TileClass;  key tile kt covers
+// request positions kt*tile_k .. kt*tile_k + tile_k - 1.  In tensor-core plans tile_k is 128 and, when the mask
+// was built with a 64-key skip granularity, bit h of the half mask says whether keys 64h .. 64h+63 of the tile
+// hold any kept pair (an absent half is neither loaded nor computed); otherwise the half mask is 3.
 // entry.y = for a general tile, the index of its first mask word: row r of the query tile owns
 // words [entry.y + r*words_per_row, +words_per_row), bit c of word w = key 32*w + c of the tile
 // (causality already applied; rows past q_rows are zero); -1 otherwise.

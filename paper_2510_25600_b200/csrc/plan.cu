@@ -164,9 +164,13 @@ static void schedule_units(const std::vector<QTile>& qtiles, int32_t H, int32_t 
 static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p, purekv_dtype dtype,
                                 int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, int32_t n_ctas,
                                 purekv_plan_info* info, std::vector<uint8_t>& host) {
-  int tq, tk;
-  purekv_status st = check_params(b, p, dtype, head_dim, &tq, &tk);
+  int tq, gk;  // rows per query tile; skip granularity in keys (the mask parameter `tile`)
+  purekv_status st = check_params(b, p, dtype, head_dim, &tq, &gk);
   if (st != PUREKV_OK) return st;
+  // The tensor-core kernel always works on 128-key entries; with a 64-key skip granularity an entry carries a
+  // 2-bit mask of the halves that hold kept pairs, and an absent half is neither loaded nor computed.
+  const int32_t tk = tq == 128 ? 128 : gk;  // keys per list entry
+  const int32_t hpe = tk / gk;              // key blocks of the skip granularity per entry (1 or 2)
   PK_REQUIRE(info, PUREKV_ERR_INVALID_ARG, "info is null");
   PK_REQUIRE(n_q_heads >= 1 && n_kv_heads >= 1 && n_q_heads % n_kv_heads == 0 && n_q_heads <= 65535,
              PUREKV_ERR_INVALID_ARG, "n_q_heads %d must be a positive multiple of n_kv_heads %d", n_q_heads,
@@ -183,7 +187,7 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   std::vector<uint32_t> masks;
   memset(info, 0, sizeof(*info));
 
-  std::vector<int64_t> cnt, diff;
+  std::vector<int64_t> cnt, diff, cg;  // kept pairs per gk-key block of the current query tile
   std::vector<Span> spans, row_spans;
   std::vector<int32_t> row_off;
   for (int r = 0; r < b->n_req; ++r) {
@@ -191,25 +195,27 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
     const int32_t len = b->h_cu_seqlens[r + 1] - base;
     const int32_t npre = b->h_n_prefix[r], nfr = b->h_n_frames[r];
     const int32_t vis_end = npre + nfr * n;
-    const int32_t nkt = (len + tk - 1) / tk;
-    cnt.assign((size_t)nkt + 1, 0);
-    diff.assign((size_t)nkt + 2, 0);
+    const int32_t nkt = (len + gk - 1) / gk + 2;
+    cnt.assign((size_t)nkt + 2, 0);
+    diff.assign((size_t)nkt + 3, 0);
+    cg.assign((size_t)nkt + 3, 0);
     const int32_t anchor_end = (int32_t)std::min<int64_t>(vis_end, npre + (int64_t)p->anchor_frames * n);  // exclusive
     for (int32_t q0 = 0; q0 < len; q0 += tq) {
       const int32_t q1 = std::min(len, q0 + tq);  // exclusive
-      const int32_t kt_hi = (q1 - 1) / tk;        // last key tile a causal mask reaches
-      std::fill(cnt.begin(), cnt.begin() + kt_hi + 1, 0);
-      std::fill(diff.begin(), diff.begin() + kt_hi + 2, 0);
+      const int32_t kt_hi = (q1 - 1) / tk;        // last list entry a causal mask reaches
+      const int32_t kg_hi = (q1 - 1) / gk;        // last gk-key block a causal mask reaches
+      std::fill(cnt.begin(), cnt.begin() + kg_hi + 3, 0);
+      std::fill(diff.begin(), diff.begin() + kg_hi + 4, 0);
       row_spans.clear();
       row_off.assign(1, 0);
       auto add_span = [&](int32_t a, int32_t bb) {  // inclusive, a <= bb
         row_spans.push_back({a, bb});
-        const int32_t ta = a / tk, tb = bb / tk;
+        const int32_t ta = a / gk, tb = bb / gk;
         if (ta == tb) { cnt[ta] += bb - a + 1; return; }
-        cnt[ta] += (ta + 1) * tk - a;
-        cnt[tb] += bb - tb * tk + 1;
-        diff[ta + 1] += tk;
-        diff[tb] -= tk;
+        cnt[ta] += (ta + 1) * gk - a;
+        cnt[tb] += bb - tb * gk + 1;
+        diff[ta + 1] += gk;
+        diff[tb] -= gk;
       };
       // each row's kept keys as disjoint ascending spans (Sec. 3.2)
       for (int32_t i = q0; i < q1; ++i) {
@@ -260,11 +266,20 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
       qt.entry_begin = (int32_t)entries.size();
       qt.pad[0] = qt.pad[1] = 0;
       int64_t run = 0;
+      for (int32_t kg = 0; kg <= kg_hi + 1; ++kg) {
+        run += diff[kg];
+        cg[kg] = cnt[kg] + run;
+      }
+      info->tiles_causal += kg_hi + 1;
       for (int32_t kt = 0; kt <= kt_hi; ++kt) {
-        run += diff[kt];
-        const int64_t c = cnt[kt] + run;
-        info->tiles_causal++;
+        int64_t c = 0;
+        int32_t half_mask = 0;
+        for (int32_t hh = 0; hh < hpe; ++hh) {
+          const int32_t kg = kt * hpe + hh;
+          if (kg <= kg_hi && cg[kg] > 0) { c += cg[kg]; half_mask |= 1 << hh; info->tiles_kept++; }
+        }
         if (c == 0) continue;
+        if (hpe == 1) half_mask = 3;  // one block per entry: both bits set by convention
         const int32_t j0 = kt * tk;
         const int64_t full = (int64_t)(q1 - q0) * tk;
         int64_t causal = full;  // pairs with j <= i inside this tile
@@ -294,9 +309,8 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
               }
             }
         }
-        entries.push_back(make_int2((kt << 2) | cls, mask_at));
+        entries.push_back(make_int2((kt << 4) | (half_mask << 2) | cls, mask_at));
         info->pairs_kept += c;
-        info->tiles_kept++;
         (cls == kTileFull ? info->tiles_full : cls == kTileDiag ? info->tiles_diag : info->tiles_general)++;
       }
       qt.entry_count = (int32_t)entries.size() - qt.entry_begin;
@@ -358,7 +372,7 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   }
 
   info->tile_q = tq;
-  info->tile_k = tk;
+  info->tile_k = gk;
   info->n_qtiles = nq;
   info->bytes_used = total;
   info->dtype = (int32_t)dtype;

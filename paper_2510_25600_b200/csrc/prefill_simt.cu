@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(kSimtThreads) prefill_simt_kernel(
 
   for (int32_t e = 0; e < qt.entry_count; ++e) {
     const int2 ent = entries[qt.entry_begin + e];
-    const int32_t cls = ent.x & 3, j0 = (ent.x >> 2) * tk;
+    const int32_t cls = ent.x & 3, j0 = (ent.x >> 4) * tk;
     __syncthreads();
     for (int x = tid; x < tk * D; x += kSimtThreads) {
       const int row = x / D, c = x % D;

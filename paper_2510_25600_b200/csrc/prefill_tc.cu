@@ -271,7 +271,8 @@ struct __align__(8) Barriers {
 template <int BK>
 __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-    const __grid_constant__ CUtensorMap tm_v, __nv_bfloat16* __restrict__ o, float* __restrict__ lse,
+    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k64,
+    const __grid_constant__ CUtensorMap tm_v64, __nv_bfloat16* __restrict__ o, float* __restrict__ lse,
     uint8_t* __restrict__ plan, float* __restrict__ ws, int32_t n_q_heads, int32_t n_kv_heads, float scale_log2,
     int32_t* __restrict__ status) {
   constexpr int ST = Cfg<BK>::kStages, SB = Cfg<BK>::kSBuf, MR = Cfg<BK>::kMeta;
@@ -373,7 +374,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
           e.y = __shfl_sync(0xffffffffu, e_l.y, n - n0);
           if (lane == 0) {
             const uint32_t s = it % ST, par = ((it / ST) - 1u) & 1u, ms = it % MR;
-            const int32_t tok = u.req_start + (e.x >> 2) * BK;
+            const int32_t tok = u.req_start + (e.x >> 4) * BK;
+            const uint32_t hm = (uint32_t)(e.x >> 2) & 3u;  // which 64-key halves of the tile are present
             if (it >= (uint32_t)ST) ok = mbar_wait(smem_u32(&bars.k_empty[s]), par, abort_flag);
             if (ok) {
               meta_s[ms] = e;
@@ -383,16 +385,32 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
               } else {
                 mbar_arrive(smem_u32(&bars.m_full[ms]));
               }
-              mbar_expect_tx(smem_u32(&bars.k_full[s]), kTileKV);
-              tma_load_3d(sK + s * kTileKV, &tm_k, smem_u32(&bars.k_full[s]), 0, g, tok);
-              tma_load_3d(sK + s * kTileKV + kPanelKV, &tm_k, smem_u32(&bars.k_full[s]), 64, g, tok);
+              if (hm == 3u) {
+                mbar_expect_tx(smem_u32(&bars.k_full[s]), kTileKV);
+                tma_load_3d(sK + s * kTileKV, &tm_k, smem_u32(&bars.k_full[s]), 0, g, tok);
+                tma_load_3d(sK + s * kTileKV + kPanelKV, &tm_k, smem_u32(&bars.k_full[s]), 64, g, tok);
+              } else {  // one half: 64 rows into their place inside each panel
+                const uint32_t hh = hm >> 1, off = hh * (kPanelKV / 2);
+                mbar_expect_tx(smem_u32(&bars.k_full[s]), kTileKV / 2);
+                tma_load_3d(sK + s * kTileKV + off, &tm_k64, smem_u32(&bars.k_full[s]), 0, g, tok + 64 * (int32_t)hh);
+                tma_load_3d(sK + s * kTileKV + kPanelKV + off, &tm_k64, smem_u32(&bars.k_full[s]), 64, g,
+                            tok + 64 * (int32_t)hh);
+              }
               issued_k = (int32_t)it + 1;
               if (it >= (uint32_t)ST) ok = mbar_wait(smem_u32(&bars.v_empty[s]), par, abort_flag);
             }
             if (ok) {
-              mbar_expect_tx(smem_u32(&bars.v_full[s]), kTileKV);
-              tma_load_3d(sV + s * kTileKV, &tm_v, smem_u32(&bars.v_full[s]), 0, g, tok);
-              tma_load_3d(sV + s * kTileKV + kPanelKV, &tm_v, smem_u32(&bars.v_full[s]), 64, g, tok);
+              if (hm == 3u) {
+                mbar_expect_tx(smem_u32(&bars.v_full[s]), kTileKV);
+                tma_load_3d(sV + s * kTileKV, &tm_v, smem_u32(&bars.v_full[s]), 0, g, tok);
+                tma_load_3d(sV + s * kTileKV + kPanelKV, &tm_v, smem_u32(&bars.v_full[s]), 64, g, tok);
+              } else {
+                const uint32_t hh = hm >> 1, off = hh * (kPanelKV / 2);
+                mbar_expect_tx(smem_u32(&bars.v_full[s]), kTileKV / 2);
+                tma_load_3d(sV + s * kTileKV + off, &tm_v64, smem_u32(&bars.v_full[s]), 0, g, tok + 64 * (int32_t)hh);
+                tma_load_3d(sV + s * kTileKV + kPanelKV + off, &tm_v64, smem_u32(&bars.v_full[s]), 64, g,
+                            tok + 64 * (int32_t)hh);
+              }
               issued_v = (int32_t)it + 1;
             }
           }
@@ -417,6 +435,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(BK, false);
+      constexpr uint32_t idesc_qk_half = instr_desc(BK / 2, false);
       constexpr uint32_t idesc_pv = instr_desc(kD, true);
       uint32_t it_base = 0;            // key tiles of earlier units
       uint32_t tq[2] = {0, 0};         // S products issued per slot, over all units
@@ -435,12 +454,23 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         // the stage was already awaited for slot 0 of the same tile
         if (sl == 0 && !mbar_wait(smem_u32(&bars.k_full[s]), (it / ST) & 1u, abort_flag)) return false;
         tc_fence_after();
-        const uint32_t d_addr = tmem + sl * 128 + b * BK;
-        const uint32_t q_lo = q_lo0 + (uint32_t)sl * (kTileQ >> 4), k_lo = k_lo0 + s * (kTileKV >> 4);
+        const uint32_t hm = (uint32_t)(meta_s[it % MR].x >> 2) & 3u;  // written before the stage's barrier was armed
+        const uint32_t q_lo = q_lo0 + (uint32_t)sl * (kTileQ >> 4);
+        if (hm == 3u) {
+          const uint32_t d_addr = tmem + sl * 128 + b * BK, k_lo = k_lo0 + s * (kTileKV >> 4);
 #pragma unroll
-        for (int ks = 0; ks < kD / 16; ++ks)
-          mma_ss_lh(d_addr, q_lo + (ks >> 2) * (kPanelQ >> 4) + (ks & 3) * 2, kDescHi,
-                    k_lo + (ks >> 2) * (kPanelKV >> 4) + (ks & 3) * 2, kDescHi, idesc_qk, ks > 0 ? 1u : 0u);
+          for (int ks = 0; ks < kD / 16; ++ks)
+            mma_ss_lh(d_addr, q_lo + (ks >> 2) * (kPanelQ >> 4) + (ks & 3) * 2, kDescHi,
+                      k_lo + (ks >> 2) * (kPanelKV >> 4) + (ks & 3) * 2, kDescHi, idesc_qk, ks > 0 ? 1u : 0u);
+        } else {  // one 64-key half: N = 64, into that half's columns of S
+          const uint32_t hh = hm >> 1;
+          const uint32_t d_addr = tmem + sl * 128 + b * BK + hh * 64;
+          const uint32_t k_lo = k_lo0 + s * (kTileKV >> 4) + hh * (kPanelKV >> 5);
+#pragma unroll
+          for (int ks = 0; ks < kD / 16; ++ks)
+            mma_ss_lh(d_addr, q_lo + (ks >> 2) * (kPanelQ >> 4) + (ks & 3) * 2, kDescHi,
+                      k_lo + (ks >> 2) * (kPanelKV >> 4) + (ks & 3) * 2, kDescHi, idesc_qk_half, ks > 0 ? 1u : 0u);
+        }
         if (sl == n_slots - 1) {
           tc_commit(smem_u32(&bars.k_empty[s]));
           if (n == nt - 1) tc_commit(smem_u32(&bars.q_empty));  // the unit's last read of Q
@@ -460,13 +490,17 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         const uint32_t p_addr = tmem + sl * 128 + b * BK, o_addr = tmem + kColO + sl * 128;
         // B = V tile, MN-major: per K step 16 key rows (2 groups of 8, 1024 B apart) x 128 dims (2 panels)
         const uint32_t v_lo = v_lo0 + s * (kTileKV >> 4);
-        if (n > 0) {
-#pragma unroll
-          for (int ks = 0; ks < BK / 16; ++ks) mma_ts_lh(o_addr, p_addr + ks * 8, v_lo + ks * (2048 >> 4), kDescHi, idesc_pv, 1u);
-        } else {
+        const uint32_t hm = (uint32_t)(meta_s[it % MR].x >> 2) & 3u;
+        const uint32_t acc0 = n > 0 ? 1u : 0u;  // the unit's first product overwrites O
+        if (hm == 3u) {
 #pragma unroll
           for (int ks = 0; ks < BK / 16; ++ks)
-            mma_ts_lh(o_addr, p_addr + ks * 8, v_lo + ks * (2048 >> 4), kDescHi, idesc_pv, ks > 0 ? 1u : 0u);
+            mma_ts_lh(o_addr, p_addr + ks * 8, v_lo + ks * (2048 >> 4), kDescHi, idesc_pv, ks > 0 ? 1u : acc0);
+        } else {  // the K steps of the present half only
+          const uint32_t k0 = (hm >> 1) * (BK / 32);
+#pragma unroll
+          for (int ks = 0; ks < BK / 32; ++ks)
+            mma_ts_lh(o_addr, p_addr + (k0 + ks) * 8, v_lo + (k0 + ks) * (2048 >> 4), kDescHi, idesc_pv, ks > 0 ? 1u : acc0);
         }
         if (sl == n_slots - 1) tc_commit(smem_u32(&bars.v_empty[s]));
         if (SB > 1) tc_commit(smem_u32(&bars.o_done[sl]));
@@ -548,7 +582,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         const uint32_t it = it_base + (uint32_t)n, ms = it % MR, b = t % SB;
         if (!wait_w(smem_u32(&bars.m_full[ms]), (it / MR) & 1u)) { ok = false; break; }
         const int2 e = meta_s[ms];
-        const int32_t cls = e.x & 3, j0 = (e.x >> 2) * BK;
+        const int32_t cls = e.x & 3, j0 = (e.x >> 4) * BK;
+        const uint32_t hm = (uint32_t)(e.x >> 2) & 3u;  // present 64-key halves; chunk c belongs to half c / 2
         uint32_t keep[BK / 32];
         if (cls == kTileGeneral) {  // this row's bits of the tile's mask
           const uint32_t* mrow = reinterpret_cast<const uint32_t*>(smem_raw + (sM - smem_u32(smem_raw)) + ms * kMaskBytes) +
@@ -571,6 +606,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
 #pragma unroll
           for (int c = 0; c < BK / 32; ++c) keep[c] = 0xFFFFFFFFu;
         }
+        if (hm != 3u) {  // columns of an absent half hold nothing: treat them as masked and leave them alone
+#pragma unroll
+          for (int c = 0; c < BK / 32; ++c)
+            if (!((hm >> (c >> 1)) & 1u)) keep[c] = 0u;
+        }
         if (!wait_w(smem_u32(&bars.s_full[sl][b]), (t / SB) & 1u)) { ok = false; break; }
         tc_fence_after();
         const uint32_t s_addr = t_lane + sl * 128 + b * BK;
@@ -582,30 +622,31 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         float l_tile = 0.f;
         bool exact = false;
         {
-          uint32_t r[BK];
-          tmem_ld32_at<0>(s_addr, r);
-          tmem_ld32_at<32>(s_addr + 32, r);
-          if constexpr (BK == 128) {
-            tmem_ld32_at<64>(s_addr + 64, r);
-            tmem_ld32_at<96>(s_addr + 96, r);
-          }
-          tc_wait_ld();
           float2 ls2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
           const float2 sc2 = make_float2(scale_log2, scale_log2), mm2 = make_float2(-m_ref, -m_ref);
 #pragma unroll
-          for (int c = 0; c < BK / 32; ++c) {
-            if (cls != kTileFull && __any_sync(0xffffffffu, keep[c] != 0xFFFFFFFFu)) {  // warp-uniform
+          for (int hh = 0; hh < 2; ++hh) {
+            if (!((hm >> hh) & 1u)) continue;  // absent half (uniform over the CTA)
+            uint32_t r[64];
+            tmem_ld32_at<0>(s_addr + 64 * hh, r);
+            tmem_ld32_at<32>(s_addr + 64 * hh + 32, r);
+            tc_wait_ld();
 #pragma unroll
-              for (int x = 0; x < 32; ++x)
-                if (!((keep[c] >> x) & 1u)) r[32 * c + x] = 0xFF800000u;  // -inf: exp2 gives 0
-            }
+            for (int cc = 0; cc < 2; ++cc) {
+              const int c = 2 * hh + cc;
+              if (cls != kTileFull && __any_sync(0xffffffffu, keep[c] != 0xFFFFFFFFu)) {  // warp-uniform
 #pragma unroll
-            for (int x = 0; x < 32; x += 2) {
-              const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[32 * c + x]), __uint_as_float(r[32 * c + x + 1])), sc2, mm2);
-              // kPolyOf8 of every 8 column pairs take the polynomial on the FMA pipe, the rest the MUFU unit
-              const float2 pp = ((x >> 1) & 7) < kPolyOf8 ? exp2_poly2(a) : make_float2(ex2(a.x), ex2(a.y));
-              ls2[(x >> 1) & 1] = __fadd2_rn(ls2[(x >> 1) & 1], pp);
-              pk[16 * c + (x >> 1)] = pack_bf16(pp.x, pp.y);
+                for (int x = 0; x < 32; ++x)
+                  if (!((keep[c] >> x) & 1u)) r[32 * cc + x] = 0xFF800000u;  // -inf: exp2 gives 0
+              }
+#pragma unroll
+              for (int x = 0; x < 32; x += 2) {
+                const float2 a = __ffma2_rn(make_float2(__uint_as_float(r[32 * cc + x]), __uint_as_float(r[32 * cc + x + 1])), sc2, mm2);
+                // kPolyOf8 of every 8 column pairs take the polynomial on the FMA pipe, the rest the MUFU unit
+                const float2 pp = ((x >> 1) & 7) < kPolyOf8 ? exp2_poly2(a) : make_float2(ex2(a.x), ex2(a.y));
+                ls2[(x >> 1) & 1] = __fadd2_rn(ls2[(x >> 1) & 1], pp);
+                pk[16 * c + (x >> 1)] = pack_bf16(pp.x, pp.y);
+              }
             }
           }
           l_tile = (ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y);
@@ -671,7 +712,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         l_sum += l_tile;
         // bf16 P over the first BK/2 columns of S, which this thread has consumed
 #pragma unroll
-        for (int c = 0; c < BK / 32; ++c) tmem_st16(s_addr + 16 * c, reinterpret_cast<const uint32_t(&)[16]>(pk[16 * c]));
+        for (int c = 0; c < BK / 32; ++c)
+          if ((hm >> (c >> 1)) & 1u) tmem_st16(s_addr + 16 * c, reinterpret_cast<const uint32_t(&)[16]>(pk[16 * c]));
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -834,15 +876,15 @@ static purekv_status make_map(CUtensorMap* map, const void* base, int64_t n_toke
 
 __device__ int32_t g_default_status;
 
-template <int BK>
 static purekv_status launch(const PrefillArgs& a, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
-                            int32_t* status) {
+                            const CUtensorMap& mk64, const CUtensorMap& mv64, int32_t* status) {
+  constexpr int BK = 128;
   const size_t smem = 1024 + 2 * 2 * (size_t)kBQ * 128 + 2 * (size_t)Cfg<BK>::kStages * 2 * BK * 128 +
                       (size_t)Cfg<BK>::kMeta * Cfg<BK>::kMaskBytes;
   PK_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid((unsigned)a.info->n_ctas);
-  prefill_tc_kernel<BK><<<grid, kThreads, smem, a.stream>>>(mq, mk, mv, (__nv_bfloat16*)a.o, a.lse, (uint8_t*)a.plan,
-                                                            (float*)a.ws, a.n_q_heads, a.n_kv_heads,
+  prefill_tc_kernel<BK><<<grid, kThreads, smem, a.stream>>>(mq, mk, mv, mk64, mv64, (__nv_bfloat16*)a.o, a.lse,
+                                                            (uint8_t*)a.plan, (float*)a.ws, a.n_q_heads, a.n_kv_heads,
                                                             a.scale * 1.4426950408889634f, status);
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
@@ -856,14 +898,16 @@ purekv_status launch_prefill_tc(const PrefillArgs& a) {
              PUREKV_ERR_UNSUPPORTED, "tensor-core prefill needs tile_q 128, tile_k 64/128, head_dim 128");
   PK_REQUIRE(a.info->n_ctas >= 1 && a.info->n_units >= 1, PUREKV_ERR_INVALID_ARG, "plan holds no schedule");
   const int64_t T = a.batch->total_tokens;
-  CUtensorMap mq, mk, mv;
+  CUtensorMap mq, mk, mv, mk64, mv64;
   purekv_status st;
   if ((st = make_map(&mq, a.q, T, a.n_q_heads, kBQ)) != PUREKV_OK) return st;
-  if ((st = make_map(&mk, a.k, T, a.n_kv_heads, a.info->tile_k)) != PUREKV_OK) return st;
-  if ((st = make_map(&mv, a.v, T, a.n_kv_heads, a.info->tile_k)) != PUREKV_OK) return st;
+  if ((st = make_map(&mk, a.k, T, a.n_kv_heads, 128)) != PUREKV_OK) return st;
+  if ((st = make_map(&mv, a.v, T, a.n_kv_heads, 128)) != PUREKV_OK) return st;
+  if ((st = make_map(&mk64, a.k, T, a.n_kv_heads, 64)) != PUREKV_OK) return st;
+  if ((st = make_map(&mv64, a.v, T, a.n_kv_heads, 64)) != PUREKV_OK) return st;
   int32_t* status = a.status;
   if (!status) PK_CUDA(cudaGetSymbolAddress((void**)&status, g_default_status));
-  return a.info->tile_k == 64 ? launch<64>(a, mq, mk, mv, status) : launch<128>(a, mq, mk, mv, status);
+  return launch(a, mq, mk, mv, mk64, mv64, status);
 }
 
 }  // namespace purekv

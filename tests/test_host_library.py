@@ -111,7 +111,9 @@ def check_plan(batch: inputs.Batch, mask: inputs.STMask, dtype, head_dim, H=4, H
     else:
         assert info.n_ctas == 0 and info.n_units == 0 and info.ws_bytes == 0
     tq, tk, wpr = p["tq"], p["tk"], p["wpr"]
-    assert (tq, tk) == (info.tile_q, info.tile_k) and wpr == max(1, tk // 32)
+    gk = info.tile_k                                  # skip granularity; tk = keys per list entry
+    assert tq == info.tile_q and gk == mask.tile and wpr == max(1, tk // 32)
+    assert tk == (128 if tq == 128 else gk)
     mp = po.mask_params(mask)
     cu = batch.cu_seqlens
     pairs = kept = full = diag = gen = causal_tiles = 0
@@ -127,19 +129,21 @@ def check_plan(batch: inputs.Batch, mask: inputs.STMask, dtype, head_dim, H=4, H
             qi += 1
             assert row[0] == cu[r] + q0 and row[1] == q1 - q0 and row[2] == cu[r] and row[3] == l
             ents = p["entries"][row[4]:row[4] + row[5]]
-            listed = {int(e[0]) >> 2: (int(e[0]) & 3, int(e[1])) for e in ents}
+            listed = {int(e[0]) >> 4: ((int(e[0]) >> 2) & 3, int(e[0]) & 3, int(e[1])) for e in ents}
             assert len(listed) == len(ents) and list(listed) == sorted(listed)
-            nkt = (q1 - 1) // tk + 1
-            causal_tiles += nkt
-            for kt in range(nkt):
+            causal_tiles += (q1 - 1) // gk + 1
+            for kt in range((q1 - 1) // tk + 1):
                 j0, j1 = kt * tk, min(l, kt * tk + tk)
                 sub = mm[q0:q1, j0:j1]
                 cnt = int(sub.sum())
+                # blocks of the skip granularity inside this entry that hold a kept pair
+                present = [int(mm[q0:q1, j0 + h * gk:min(l, j0 + (h + 1) * gk)].sum()) > 0 for h in range(tk // gk)]
+                kept += sum(present)
                 if cnt == 0:
                     assert kt not in listed
                     continue
-                kept += 1
-                cls, at = listed[kt]
+                hm, cls, at = listed[kt]
+                assert hm == (3 if tk == gk else sum(1 << h for h, pr in enumerate(present) if pr))
                 if cnt == (q1 - q0) * tk:
                     assert cls == 0 and at == -1
                     full += 1
