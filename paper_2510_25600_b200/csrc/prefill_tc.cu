@@ -23,6 +23,8 @@
 // sets the device status word, drains, frees TMEM and exits.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "prefill.cuh"
 
 namespace purekv {
@@ -216,6 +218,12 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x) {
   p.x = __uint_as_float(__float_as_uint(p.x) + (__float_as_uint(r.x) << 23));
   p.y = __uint_as_float(__float_as_uint(p.y) + (__float_as_uint(r.y) << 23));
   return p;
+}
+// 32 contiguous bytes in one store: half as many store instructions (and LSU passes) as 16-byte stores
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&w)[8]) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+               "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+               : "memory");
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
@@ -624,16 +632,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         {
           float2 ls2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
           const float2 sc2 = make_float2(scale_log2, scale_log2), mm2 = make_float2(-m_ref, -m_ref);
-#pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            if (!((hm >> hh) & 1u)) continue;  // absent half (uniform over the CTA)
-            uint32_t r[64];
-            tmem_ld32_at<0>(s_addr + 64 * hh, r);
-            tmem_ld32_at<32>(s_addr + 64 * hh + 32, r);
-            tc_wait_ld();
+          // exponentials of one 64-key half whose S values are in r
+          auto half_exp = [&](uint32_t (&r)[64], auto hh_c) {
+            constexpr int hh = decltype(hh_c)::value;
 #pragma unroll
             for (int cc = 0; cc < 2; ++cc) {
-              const int c = 2 * hh + cc;
+              constexpr int c0 = 2 * hh;
+              const int c = c0 + cc;
               if (cls != kTileFull && __any_sync(0xffffffffu, keep[c] != 0xFFFFFFFFu)) {  // warp-uniform
 #pragma unroll
                 for (int x = 0; x < 32; ++x)
@@ -648,6 +653,23 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
                 pk[16 * c + (x >> 1)] = pack_bf16(pp.x, pp.y);
               }
             }
+          };
+          if (hm == 3u) {  // both halves: all loads in flight before the one wait
+            uint32_t r0[64], r1[64];
+            tmem_ld32_at<0>(s_addr, r0);
+            tmem_ld32_at<32>(s_addr + 32, r0);
+            tmem_ld32_at<0>(s_addr + 64, r1);
+            tmem_ld32_at<32>(s_addr + 96, r1);
+            tc_wait_ld();
+            half_exp(r0, std::integral_constant<int, 0>{});
+            half_exp(r1, std::integral_constant<int, 1>{});
+          } else {
+            uint32_t r[64];
+            tmem_ld32_at<0>(s_addr + (hm >> 1) * 64, r);
+            tmem_ld32_at<32>(s_addr + (hm >> 1) * 64 + 32, r);
+            tc_wait_ld();
+            if (hm == 1u) half_exp(r, std::integral_constant<int, 0>{});
+            else half_exp(r, std::integral_constant<int, 1>{});
           }
           l_tile = (ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y);
           bool has_kept = cls == kTileFull;
@@ -736,13 +758,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
           tc_wait_ld();
           if (row_valid) {
 #pragma unroll
-            for (int x = 0; x < 32; x += 8) {
-              uint4 w;
-              w.x = pack_bf16(__uint_as_float(tt[x + 0]) * inv, __uint_as_float(tt[x + 1]) * inv);
-              w.y = pack_bf16(__uint_as_float(tt[x + 2]) * inv, __uint_as_float(tt[x + 3]) * inv);
-              w.z = pack_bf16(__uint_as_float(tt[x + 4]) * inv, __uint_as_float(tt[x + 5]) * inv);
-              w.w = pack_bf16(__uint_as_float(tt[x + 6]) * inv, __uint_as_float(tt[x + 7]) * inv);
-              *reinterpret_cast<uint4*>(dst + 32 * c + x) = w;
+            for (int x = 0; x < 32; x += 16) {
+              uint32_t w[8];
+#pragma unroll
+              for (int y = 0; y < 8; ++y)
+                w[y] = pack_bf16(__uint_as_float(tt[x + 2 * y]) * inv, __uint_as_float(tt[x + 2 * y + 1]) * inv);
+              st_global_v8(dst + 32 * c + x, w);
             }
           }
         }
@@ -897,6 +918,7 @@ purekv_status launch_prefill_tc(const PrefillArgs& a) {
   PK_REQUIRE(a.info->tile_q == kBQ && (a.info->tile_k == 64 || a.info->tile_k == 128) && a.head_dim == kD,
              PUREKV_ERR_UNSUPPORTED, "tensor-core prefill needs tile_q 128, tile_k 64/128, head_dim 128");
   PK_REQUIRE(a.info->n_ctas >= 1 && a.info->n_units >= 1, PUREKV_ERR_INVALID_ARG, "plan holds no schedule");
+  PK_REQUIRE((uintptr_t)a.o % 32 == 0, PUREKV_ERR_INVALID_ARG, "O must be 32-byte aligned for the tensor-core kernel");
   const int64_t T = a.batch->total_tokens;
   CUtensorMap mq, mk, mv, mk64, mv64;
   purekv_status st;
