@@ -150,7 +150,8 @@ purekv_status purekv_st_sparse_prefill(const void *q, const void *k, const void 
  *   C[g, j] = (1/G) sum_{hq in group g} sum_{i=l-w}^{l-1} A^{hq}[i, j],
  * A = dense causal softmax (each row normalised over all keys j' <= i).  c_out [H_kv, T]
  * fp32; the last w entries of each request are written as 0.  The attention matrix is never
- * stored.  ws: device workspace of purekv_score_ws_bytes. */
+ * stored.  ws: device workspace of purekv_score_ws_bytes (log-sum-exp of the window rows and, for the
+ * tensor-core path, their per-key-block parts); it need not be initialised. */
 size_t purekv_score_ws_bytes(const purekv_batch *batch, int32_t window, int32_t n_q_heads);
 purekv_status purekv_lowlayer_score(const void *q, const void *k, float *c_out, const purekv_batch *batch,
                                     int32_t window, int32_t n_q_heads, int32_t n_kv_heads,
@@ -165,9 +166,10 @@ purekv_status purekv_lowlayer_score(const void *q, const void *k, float *c_out, 
  * allocate at all.  For them this entry point keeps its scratch (the window rows' log-sum-exp values)
  * in an array inside the library's device image instead of a caller-provided workspace.  It calls no
  * cudaMalloc / cudaFree and no allocating library routine; inputs and c_out are still the caller's.
- *  - Limit: n_req * n_q_heads * window <= PUREKV_NOALLOC_SCORE_MAX_ROWS (65536 values, 256 KiB that
- *    every GPU loading the library holds until the process exits).  Larger problems return
- *    PUREKV_ERR_WORKSPACE and leave c_out untouched; use purekv_lowlayer_score for those.
+ *  - Limit: the problem's workspace need, purekv_score_ws_bytes(batch, window, n_q_heads), must not exceed
+ *    PUREKV_NOALLOC_SCORE_MAX_ROWS (65536) values, i.e. n_req * n_q_heads * window * (1 + 2 * ceil(longest
+ *    request / 64)) <= 65536 -- 256 KiB that every GPU loading the library holds until the process exits.
+ *    Larger problems return PUREKV_ERR_WORKSPACE and leave c_out untouched; use purekv_lowlayer_score.
  *  - The first call on each device looks up the array's device address (with that device current).
  *    Make that first call before any stream capture on that device.
  *  - All calls on a device share the one array, and it keeps the previous call's contents.  Nothing in

@@ -247,8 +247,8 @@ NOALLOC_SCORE_MAX_ROWS = 65536
 def purekv_lowlayer_score_noalloc(q: torch.Tensor, k: torch.Tensor, batch: Batch, window: int, c_out: torch.Tensor,
                                   softmax_scale: float = 0.0) -> torch.Tensor:
     """purekv_lowlayer_score for callers that cannot allocate: the scratch is an array inside the library, so
-    this wrapper allocates nothing either -- `c_out` [H_kv, T] fp32 must be passed in.  Problems with
-    n_req * H * window > NOALLOC_SCORE_MAX_ROWS raise PureKVError(ERR_WORKSPACE).  Calls share the scratch:
+    this wrapper allocates nothing either -- `c_out` [H_kv, T] fp32 must be passed in.  Problems whose
+    workspace need exceeds NOALLOC_SCORE_MAX_ROWS values raise PureKVError(ERR_WORKSPACE).  Calls share the scratch:
     keep them on one stream."""
     assert q.is_contiguous() and k.is_contiguous() and c_out.is_contiguous() and c_out.dtype == torch.float32
     t, h, d = q.shape

@@ -38,7 +38,7 @@ constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // per-thread registers afte
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 256;
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
-constexpr int kPolyOf8 = 2;  // of every 8 pairs of exponentials, how many are computed on the FMA pipe
+constexpr int kPolyOf8 = 1;  // of every 8 pairs of exponentials, how many are computed on the FMA pipe
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }

@@ -15,8 +15,8 @@
 
 namespace purekv {
 
-// Scratch of purekv_lowlayer_score_noalloc: the window rows' log-sum-exp values, one float per
-// (request, query head, window position).  It lives in the library's device image, so every GPU that
+// Scratch of purekv_lowlayer_score_noalloc: the window rows' log-sum-exp values and their per-key-block
+// parts, i.e. what purekv_lowlayer_score keeps in its workspace.  It lives in the library's device image, so every GPU that
 // loads the library holds these 256 KiB until the process exits.  Host code may not pass this name to
 // a kernel (on the host it is only a stand-in for the symbol); the device address comes from
 // cudaGetSymbolAddress, looked up once per device.
@@ -226,6 +226,244 @@ static int32_t max_len(const purekv_batch* b) {
   return m;
 }
 
+// ---- bf16 path on tensor cores ------------------------------------------------------------------
+// Both passes use the same tiling: a CTA owns one block of 64 keys of one (request, KV head) and walks the
+// G*w stacked window rows in blocks of 128; warp wi computes the 16 x 64 logits of rows 16*wi .. 16*wi+15 with
+// mma.sync m16n8k16 (bf16 x bf16 -> fp32: products exact, fp32 accumulation).  Pass 1 leaves, per key block and
+// row, the maximum and the sum of exponentials of the causal logits; a small kernel folds those into the row's
+// log-sum-exp; pass 2 forms exp(s - lse) and sums down the rows.  Every key block is an independent CTA, so the
+// grid is (key blocks) x (KV heads) x (requests) in both passes.
+constexpr int kMmaKeys = 64;
+constexpr int kMmaRows = 128;
+constexpr int kMmaThreads = 256;
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x2(uint32_t addr, uint32_t (&r)[2]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0, %1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16x8x16(float (&c)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
+// Copies `rows` rows of d bf16 (global row r at src + row_of(r)) into shared memory with a row stride of d + 8
+// elements (conflict-free for ldmatrix); rows for which row_of gives a negative offset are zero-filled.
+template <typename RowOf>
+__device__ __forceinline__ void stage_rows_bf16(__nv_bfloat16* dst, const __nv_bfloat16* src, int rows, int d, RowOf row_of) {
+  const int cpr = d / 8;  // 16-byte chunks per row
+  for (int x = threadIdx.x; x < rows * cpr; x += kMmaThreads) {
+    const int r = x / cpr, c = x % cpr;
+    const int64_t off = row_of(r);
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (off >= 0) v = __ldg(reinterpret_cast<const uint4*>(src + off) + c);
+    *reinterpret_cast<uint4*>(dst + r * (d + 8) + c * 8) = v;
+  }
+}
+
+// acc[nb][0..3] = logits of rows (16*warp + lane/4, +8) x keys (8*nb + 2*(lane%4), +1) of the staged tiles
+__device__ __forceinline__ void logits_16x64(const __nv_bfloat16* qs, const __nv_bfloat16* ks, int d, float (&acc)[8][4]) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, ld = d + 8;
+#pragma unroll
+  for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+    for (int x = 0; x < 4; ++x) acc[nb][x] = 0.f;
+  const uint32_t qa = (uint32_t)__cvta_generic_to_shared(qs + (16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1)) * ld + 8 * (lane >> 4));
+  const uint32_t ka = (uint32_t)__cvta_generic_to_shared(ks + (lane & 7) * ld + 8 * ((lane >> 3) & 1));
+  for (int k0 = 0; k0 < d; k0 += 16) {
+    uint32_t a[4];
+    ldmatrix_x4(qa + k0 * 2, a);
+#pragma unroll
+    for (int nb = 0; nb < 8; ++nb) {
+      uint32_t b[2];
+      ldmatrix_x2(ka + (nb * 8 * ld + k0) * 2, b);
+      mma_bf16_16x8x16(acc[nb], a, b);
+    }
+  }
+}
+
+// Pass 1.  partial[((r * Hkv + g) * n_kb + kb) * rows_max + row] = (max, sum of exp2) of the causal logits of the
+// stacked row against key block kb, in log2 units of the scaled logits.
+__global__ void __launch_bounds__(kMmaThreads) score_mma_partial_kernel(
+    const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k, const int32_t* __restrict__ cu_seqlens,
+    int32_t window, int32_t n_q_heads, int32_t n_kv_heads, int32_t d, float scale_log2, int32_t n_kb, int32_t rows_max,
+    float2* __restrict__ partial) {
+  extern __shared__ __align__(16) uint8_t smem_mma[];
+  __nv_bfloat16* ks = reinterpret_cast<__nv_bfloat16*>(smem_mma);
+  __nv_bfloat16* qs = ks + kMmaKeys * (d + 8);
+  const int32_t r = blockIdx.z, g = blockIdx.y, kb = blockIdx.x;
+  const int32_t G = n_q_heads / n_kv_heads;
+  const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
+  const int32_t w = min(window, len), n_rows = G * w, j0 = kb * kMmaKeys;
+  if (j0 >= len) return;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  stage_rows_bf16(ks, k, kMmaKeys, d, [&](int rr) -> int64_t {
+    return j0 + rr < len ? ((int64_t)(base + j0 + rr) * n_kv_heads + g) * d : -1;
+  });
+  float2* out = partial + ((int64_t)(r * n_kv_heads + g) * n_kb + kb) * rows_max;
+  for (int32_t row0 = 0; row0 < n_rows; row0 += kMmaRows) {
+    __syncthreads();
+    stage_rows_bf16(qs, q, kMmaRows, d, [&](int rr) -> int64_t {
+      const int32_t row = row0 + rr;
+      return row < n_rows ? ((int64_t)(base + len - w + row % w) * n_q_heads + g * G + row / w) * d : -1;
+    });
+    __syncthreads();
+    float acc[8][4];
+    logits_16x64(qs, ks, d, acc);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {  // the thread's two rows
+      const int32_t row = row0 + 16 * warp + (lane >> 2) + 8 * h;
+      const int32_t i = row < n_rows ? len - w + row % w : -1;  // causal limit of the row (-1: no row)
+      float m = -INFINITY;
+#pragma unroll
+      for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+        for (int x = 0; x < 2; ++x) {
+          const int32_t j = j0 + 8 * nb + 2 * (lane & 3) + x;
+          const float s = j <= i ? acc[nb][2 * h + x] * scale_log2 : -INFINITY;
+          acc[nb][2 * h + x] = s;
+          m = fmaxf(m, s);
+        }
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+      float l = 0.f;
+      if (m > -INFINITY) {
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) l += exp2f(acc[nb][2 * h] - m) + exp2f(acc[nb][2 * h + 1] - m);
+      }
+      l += __shfl_xor_sync(0xffffffffu, l, 1);
+      l += __shfl_xor_sync(0xffffffffu, l, 2);
+      if ((lane & 3) == 0 && row < n_rows) out[row] = make_float2(m, l);
+    }
+  }
+}
+
+// Folds the per-key-block (max, sum) pairs into each stacked row's log-sum-exp.  One thread per (request, query
+// head, window position).
+__global__ void __launch_bounds__(256) score_lse_merge_kernel(const float2* __restrict__ partial,
+                                                              const int32_t* __restrict__ cu_seqlens, int32_t window,
+                                                              int32_t n_q_heads, int32_t n_kv_heads, int32_t n_kb,
+                                                              int32_t rows_max, int32_t n_req, float* __restrict__ lse2) {
+  const int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (x >= (int64_t)n_req * n_q_heads * window) return;
+  const int32_t iw = (int32_t)(x % window), hq = (int32_t)((x / window) % n_q_heads), r = (int32_t)(x / ((int64_t)window * n_q_heads));
+  const int32_t G = n_q_heads / n_kv_heads, g = hq / G, hl = hq % G;
+  const int32_t len = cu_seqlens[r + 1] - cu_seqlens[r];
+  const int32_t w = min(window, len);
+  if (iw >= w) return;
+  const int32_t row = hl * w + iw, kbs = (len + kMmaKeys - 1) / kMmaKeys;
+  const float2* p = partial + ((int64_t)(r * n_kv_heads + g) * n_kb) * rows_max + row;
+  float m = -INFINITY;
+  for (int32_t kb = 0; kb < kbs; ++kb) m = fmaxf(m, p[(int64_t)kb * rows_max].x);
+  float l = 0.f;
+  for (int32_t kb = 0; kb < kbs; ++kb) {
+    const float2 v = p[(int64_t)kb * rows_max];
+    if (v.y > 0.f) l += v.y * exp2f(v.x - m);
+  }
+  lse2[((int64_t)r * n_q_heads + hq) * window + iw] = m + log2f(l);
+}
+
+// Pass 2 (Eq. 2).  C[g, j] = (1/G) * sum over the stacked rows of exp2(s - lse) for the non-recent keys of block kb.
+__global__ void __launch_bounds__(kMmaThreads) score_mma_colsum_kernel(
+    const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k, const int32_t* __restrict__ cu_seqlens,
+    int32_t window, int32_t n_q_heads, int32_t n_kv_heads, int32_t d, float scale_log2, const float* __restrict__ lse2,
+    int64_t n_tokens, float* __restrict__ c_out) {
+  extern __shared__ __align__(16) uint8_t smem_mma[];
+  __shared__ float red[kMmaThreads / 32][kMmaKeys];
+  __nv_bfloat16* ks = reinterpret_cast<__nv_bfloat16*>(smem_mma);
+  __nv_bfloat16* qs = ks + kMmaKeys * (d + 8);
+  const int32_t r = blockIdx.z, g = blockIdx.y, j0 = blockIdx.x * kMmaKeys;
+  const int32_t G = n_q_heads / n_kv_heads;
+  const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
+  const int32_t w = min(window, len), nr = len - w, n_rows = G * w;
+  if (j0 >= len) return;
+  float* cg = c_out + (int64_t)g * n_tokens + base;
+  if (j0 >= nr) {  // block inside the window: defined as 0
+    for (int c = threadIdx.x; c < kMmaKeys; c += kMmaThreads)
+      if (j0 + c < len) cg[j0 + c] = 0.f;
+    return;
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  stage_rows_bf16(ks, k, kMmaKeys, d, [&](int rr) -> int64_t {
+    return j0 + rr < len ? ((int64_t)(base + j0 + rr) * n_kv_heads + g) * d : -1;
+  });
+  float col[8][2];
+#pragma unroll
+  for (int nb = 0; nb < 8; ++nb) col[nb][0] = col[nb][1] = 0.f;
+  for (int32_t row0 = 0; row0 < n_rows; row0 += kMmaRows) {
+    __syncthreads();
+    stage_rows_bf16(qs, q, kMmaRows, d, [&](int rr) -> int64_t {
+      const int32_t row = row0 + rr;
+      return row < n_rows ? ((int64_t)(base + len - w + row % w) * n_q_heads + g * G + row / w) * d : -1;
+    });
+    __syncthreads();
+    float acc[8][4];
+    logits_16x64(qs, ks, d, acc);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int32_t row = row0 + 16 * warp + (lane >> 2) + 8 * h;
+      if (row < n_rows) {
+        // every non-recent key precedes every window row, so causality holds for all of them
+        const float lse = __ldg(lse2 + ((int64_t)r * n_q_heads + g * G + row / w) * window + row % w);
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb) {
+          col[nb][0] += exp2f(fmaf(acc[nb][2 * h], scale_log2, -lse));
+          col[nb][1] += exp2f(fmaf(acc[nb][2 * h + 1], scale_log2, -lse));
+        }
+      }
+    }
+  }
+  // sum over the 8 row groups of the warp (lanes with equal lane % 4 hold the same columns), then over the warps
+#pragma unroll
+  for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+    for (int x = 0; x < 2; ++x) {
+      float v = col[nb][x];
+      v += __shfl_xor_sync(0xffffffffu, v, 4);
+      v += __shfl_xor_sync(0xffffffffu, v, 8);
+      v += __shfl_xor_sync(0xffffffffu, v, 16);
+      if (lane < 4) red[warp][8 * nb + 2 * lane + x] = v;
+    }
+  __syncthreads();
+  if (threadIdx.x < kMmaKeys) {
+    float sum = 0.f;
+#pragma unroll
+    for (int t = 0; t < kMmaThreads / 32; ++t) sum += red[t][threadIdx.x];
+    const int32_t j = j0 + threadIdx.x;
+    if (j < len) cg[j] = j < nr ? sum / (float)G : 0.f;
+  }
+}
+
+static purekv_status launch_score_mma(const void* q, const void* k, float* c_out, const purekv_batch* b, int32_t window,
+                                      int32_t H, int32_t Hkv, int32_t d, float scale, float* ws_f, cudaStream_t sm) {
+  const int32_t ml = max_len(b);
+  const int32_t n_kb = (ml + kMmaKeys - 1) / kMmaKeys, rows_max = (H / Hkv) * window;
+  float* lse2 = ws_f;                                                             // [n_req][H][window]
+  // the pairs start on a 256-byte boundary behind the log-sum-exp values
+  float2* partial = reinterpret_cast<float2*>(ws_f + (((int64_t)b->n_req * H * window + 63) & ~(int64_t)63));  // [n_req][Hkv][n_kb][rows_max]
+  const size_t smem = (size_t)(kMmaKeys + kMmaRows) * (d + 8) * sizeof(__nv_bfloat16);
+  PK_CUDA(cudaFuncSetAttribute(score_mma_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  PK_CUDA(cudaFuncSetAttribute(score_mma_colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const float scale_log2 = scale * 1.4426950408889634f;
+  dim3 grid((unsigned)n_kb, (unsigned)Hkv, (unsigned)b->n_req);
+  score_mma_partial_kernel<<<grid, kMmaThreads, smem, sm>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, b->cu_seqlens,
+                                                            window, H, Hkv, d, scale_log2, n_kb, rows_max, partial);
+  PK_CUDA(cudaGetLastError());
+  const int64_t n_lse = (int64_t)b->n_req * H * window;
+  score_lse_merge_kernel<<<(unsigned)((n_lse + 255) / 256), 256, 0, sm>>>(partial, b->cu_seqlens, window, H, Hkv, n_kb,
+                                                                         rows_max, b->n_req, lse2);
+  PK_CUDA(cudaGetLastError());
+  score_mma_colsum_kernel<<<grid, kMmaThreads, smem, sm>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, b->cu_seqlens,
+                                                           window, H, Hkv, d, scale_log2, lse2, b->total_tokens, c_out);
+  PK_CUDA(cudaGetLastError());
+  return PUREKV_OK;
+}
+
 template <typename T>
 static purekv_status launch_score(const void* q, const void* k, float* c_out, const purekv_batch* b, int32_t window,
                                   int32_t H, int32_t Hkv, int32_t d, float scale, float* lse2, cudaStream_t sm) {
@@ -252,8 +490,11 @@ static purekv_status launch_score(const void* q, const void* k, float* c_out, co
 using namespace purekv;
 
 extern "C" size_t purekv_score_ws_bytes(const purekv_batch* batch, int32_t window, int32_t n_q_heads) {
-  if (!batch || window < 0 || n_q_heads < 0) return 0;
-  return (size_t)batch->n_req * n_q_heads * (size_t)std::max(window, 1) * sizeof(float) + 256;
+  if (!batch || window < 0 || n_q_heads < 0 || !batch->h_cu_seqlens) return 0;
+  // log-sum-exp per (request, head, window row), plus (max, sum) pairs per 64-key block for the tensor-core path
+  const size_t rows = (size_t)batch->n_req * n_q_heads * (size_t)std::max(window, 1);
+  const size_t n_kb = ((size_t)max_len(batch) + kMmaKeys - 1) / kMmaKeys;
+  return (((rows + 63) & ~(size_t)63) + rows * 2 * n_kb) * sizeof(float) + 256;
 }
 
 extern "C" purekv_status purekv_lowlayer_score(const void* q, const void* k, float* c_out, const purekv_batch* batch,
@@ -277,6 +518,8 @@ extern "C" purekv_status purekv_lowlayer_score(const void* q, const void* k, flo
   float* lse2 = (float*)(((uintptr_t)ws + 255) & ~(uintptr_t)255);
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
   cudaStream_t sm = (cudaStream_t)stream;
+  if (dtype == PUREKV_BF16 && head_dim % 16 == 0)
+    return launch_score_mma(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
   if (dtype == PUREKV_BF16)
     return launch_score<__nv_bfloat16>(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
   return launch_score<float>(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
@@ -308,14 +551,14 @@ extern "C" purekv_status purekv_lowlayer_score_noalloc(const void* q, const void
   purekv_status st = check_batch(batch, true);
   if (st != PUREKV_OK) return st;
   PK_REQUIRE(window >= 1 && n_q_heads >= 1, PUREKV_ERR_INVALID_ARG, "window and n_q_heads must be >= 1");
-  const size_t need = (size_t)batch->n_req * (size_t)n_q_heads * (size_t)window;
+  const size_t need = (purekv_score_ws_bytes(batch, window, n_q_heads) - 256) / sizeof(float);
   PK_REQUIRE(need <= kNoallocScoreFloats, PUREKV_ERR_WORKSPACE,
-             "purekv_lowlayer_score_noalloc: n_req * n_q_heads * window = %zu exceeds the built-in scratch of %zu "
-             "values; use purekv_lowlayer_score with a caller-provided workspace",
+             "purekv_lowlayer_score_noalloc: this problem needs %zu scratch values, the built-in scratch holds %zu; "
+             "use purekv_lowlayer_score with a caller-provided workspace",
              need, kNoallocScoreFloats);
   float* scratch = nullptr;
   if ((st = noalloc_scratch(&scratch)) != PUREKV_OK) return st;
-  // The scratch needs no clearing: pass 1 writes every (request, head, window position) entry that pass 2 reads.
+  // The scratch needs no clearing: every entry that a later kernel of the call reads is written earlier in the call.
   return purekv_lowlayer_score(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, dtype, softmax_scale,
                                scratch, (kNoallocScoreFloats + 64) * sizeof(float), stream);
 }
