@@ -177,11 +177,11 @@ def purekv_plan_bytes(batch: Batch, params: StParams, dtype: int, head_dim: int,
 
 def purekv_plan_build(batch: Batch, params: StParams, dtype: int, head_dim: int, n_q_heads: int, n_kv_heads: int,
                       buf: Optional[torch.Tensor] = None, n_ctas: int = 0) -> Plan:
-    n = purekv_plan_bytes(batch, params, dtype, head_dim, n_q_heads, n_kv_heads, n_ctas)
-    if n == 0:
-        _check(_lib.purekv_plan_build(C.byref(batch.c), C.byref(params), dtype, head_dim, n_q_heads, n_kv_heads,
-                                      n_ctas, None, 0, C.byref(PlanInfo()), None), "purekv_plan_build")
-    if buf is None:
+    if buf is None:                 # size the buffer first (plans the batch once more); callers that plan often pass one
+        n = purekv_plan_bytes(batch, params, dtype, head_dim, n_q_heads, n_kv_heads, n_ctas)
+        if n == 0:
+            _check(_lib.purekv_plan_build(C.byref(batch.c), C.byref(params), dtype, head_dim, n_q_heads, n_kv_heads,
+                                          n_ctas, None, 0, C.byref(PlanInfo()), None), "purekv_plan_build")
         buf = torch.empty(n, dtype=torch.uint8, device="cuda")
     info = PlanInfo()
     _check(_lib.purekv_plan_build(C.byref(batch.c), C.byref(params), dtype, head_dim, n_q_heads, n_kv_heads, n_ctas,
