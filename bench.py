@@ -216,7 +216,7 @@ def run_reference(args, wl):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--cfg", type=int, default=1)
     ap.add_argument("--impl", default="purekv")
@@ -301,7 +301,7 @@ def main():
     prefill_ms_step = float(k_ms.sum(axis=1).mean())
     achieved = flops_step / (prefill_ms_step * 1e-3) / 1e12
     peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
-    roofline = {"kernel": f"prefill_tc_kernel<{info_s.tile_k}>", "bound": "tensor", "achieved": achieved, "peak": peak,
+    roofline = {"kernel": f"prefill_tc_kernel (128-key entries, skip granularity {info_s.tile_k})", "bound": "tensor", "achieved": achieved, "peak": peak,
                 "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
                 "peak_kind": f"{peak_kind} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']}, nominal dense 2250)",
                 "flops_per_step": flops_step, "launches_per_step": wl.n_layers, "avg_launch_ms": prefill_ms_step / wl.n_layers,

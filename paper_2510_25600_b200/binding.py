@@ -190,11 +190,17 @@ def purekv_plan_build(batch: Batch, params: StParams, dtype: int, head_dim: int,
 
 
 def purekv_plan_build_host(batch: Batch, params: StParams, dtype: int, head_dim: int, n_q_heads: int, n_kv_heads: int,
-                           n_ctas: int = 0):
-    """Plan bytes in host memory (numpy uint8) + PlanInfo; makes no CUDA call."""
+                           n_ctas: int = 0, out: Optional[torch.Tensor] = None):
+    """Plan bytes in host memory + PlanInfo; makes no CUDA call.  Without `out` the bytes come back as a numpy
+    uint8 array sized by a first planning pass; with `out` (a host uint8 tensor, e.g. pinned, large enough) they
+    are written there in one pass and the used prefix of `out` is returned, ready for an asynchronous copy."""
+    info = PlanInfo()
+    if out is not None:
+        _check(_lib.purekv_plan_build_host(C.byref(batch.c), C.byref(params), dtype, head_dim, n_q_heads, n_kv_heads,
+                                           n_ctas, out.data_ptr(), out.numel(), C.byref(info)), "purekv_plan_build_host")
+        return out[:info.bytes_used], info
     n = purekv_plan_bytes(batch, params, dtype, head_dim, n_q_heads, n_kv_heads, n_ctas)
     buf = np.zeros(max(n, 1), dtype=np.uint8)
-    info = PlanInfo()
     _check(_lib.purekv_plan_build_host(C.byref(batch.c), C.byref(params), dtype, head_dim, n_q_heads, n_kv_heads,
                                        n_ctas, buf.ctypes.data, n, C.byref(info)), "purekv_plan_build_host")
     return buf[:info.bytes_used], info

@@ -94,16 +94,23 @@ __device__ __forceinline__ uint32_t order_key(float f) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-constexpr int kSelThreads = 1024;
+constexpr int kSelThreads = 512;
 constexpr int kSelItems = 4;
 
-// One CTA per (request, KV head, layer).
+// One CTA per (request, KV head, layer).  FUSED = false: the scores come from `s` (written by vnorm_score_kernel).
+// FUSED = true: the CTA first streams its own segment of V (256-byte rows), forms S = C * ||V|| into shared memory
+// (and into s_out if asked), and selects from there, so V is the only large read and S never makes a round trip;
+// used when there are enough segments to keep every SM streaming.
+template <bool FUSED, typename T>
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ s, int64_t n_tokens,
                                                              const int32_t* __restrict__ cu_seqlens,
                                                              const int32_t* __restrict__ cu_kept,
                                                              const int32_t* __restrict__ keep, int32_t window,
                                                              int32_t k_tot, int32_t n_kv_heads,
-                                                             int32_t* __restrict__ idx_out) {
+                                                             int32_t* __restrict__ idx_out, const uint4* __restrict__ v,
+                                                             int64_t layer_stride_c, const float* __restrict__ c,
+                                                             float* __restrict__ s_out) {
+  extern __shared__ uint32_t skeys[];  // FUSED: order keys of the segment's non-recent scores
   __shared__ int32_t hist[256];
   __shared__ uint32_t sh_prefix;
   __shared__ int32_t sh_need;
@@ -121,6 +128,52 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   const int32_t tid = threadIdx.x;
 
   for (int32_t t = tid; t < w; t += kSelThreads) out[h + t] = nr + t;  // the recent window
+  if (tid < 32) { warp_gt[tid] = 0; warp_eq[tid] = 0; }  // entries past the CTA's warps stay zero
+  if constexpr (FUSED) {
+    // a half-warp reads one 256-byte row per step (16 x 16 bytes), 16 rows in flight per thread
+    const uint4* vl = v + layer * layer_stride_c;
+    const float* cg = c + (int64_t)g * n_tokens + base;
+    float* so = s_out ? s_out + ((int64_t)layer * n_kv_heads + g) * n_tokens + base : nullptr;
+    const int32_t lane = tid & 31, wrp = tid >> 5, half = lane >> 4, ch = lane & 15;
+    const int32_t n_score = so ? len : nr;  // the window's scores are 0 by definition and only matter for s_out
+    for (int32_t t0 = wrp * 32; t0 < n_score; t0 += (kSelThreads / 32) * 32) {
+      float part[16];
+#pragma unroll
+      for (int it = 0; it < 16; ++it) {
+        const int32_t t = t0 + it * 2 + half;
+        uint4 u = make_uint4(0, 0, 0, 0);
+        if (t < n_score) u = __ldg(vl + ((int64_t)(base + t) * n_kv_heads + g) * 16 + ch);
+        part[it] = Chunk<T>::sumsq(u);
+      }
+      float mine = 0.f;
+#pragma unroll
+      for (int it = 0; it < 16; ++it) {
+        float p = part[it];
+        p += __shfl_xor_sync(0xffffffffu, p, 8);
+        p += __shfl_xor_sync(0xffffffffu, p, 4);
+        p += __shfl_xor_sync(0xffffffffu, p, 2);
+        p += __shfl_xor_sync(0xffffffffu, p, 1);
+        const float v0 = __shfl_sync(0xffffffffu, p, 0), v1 = __shfl_sync(0xffffffffu, p, 16);
+        if (lane == it * 2) mine = v0;
+        if (lane == it * 2 + 1) mine = v1;
+      }
+      const int32_t t = t0 + lane;
+      if (t < n_score) {
+        const float sc = __ldg(cg + t) * sqrtf(mine);
+        if (so) so[t] = sc;
+        if (t < nr) skeys[t] = order_key(sc);
+      }
+    }
+    __syncthreads();
+  }
+  // Not fused: the keys are copied into shared memory once when the launch provided room for them (s_out is unused
+  // in this mode and doubles as that flag), so the radix passes do not go back to L2.
+  const bool staged = FUSED || s_out != nullptr;
+  if (!FUSED && staged) {
+    for (int32_t j = tid; j < nr; j += kSelThreads) skeys[j] = order_key(__ldg(seg + j));
+    __syncthreads();
+  }
+  auto key_at = [&](int32_t j) -> uint32_t { return staged ? skeys[j] : order_key(__ldg(seg + j)); };
   if (h <= 0) return;
 
   // ---- radix select: the h-th largest key --------------------------------------------
@@ -130,18 +183,36 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
     if (tid < 256) hist[tid] = 0;
     __syncthreads();
     for (int32_t j = tid; j < nr; j += kSelThreads) {
-      const uint32_t key = order_key(__ldg(seg + j));
+      const uint32_t key = key_at(j);
       if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
     }
     __syncthreads();
-    if (tid == 0) {
-      int32_t acc = 0, b = 255;
-      for (; b > 0; --b) {
-        if (acc + hist[b] >= need) break;
-        acc += hist[b];
+    if (tid < 32) {
+      // which bin holds the need-th largest key: bins taken from the top, 8 per lane, a warp scan over the lane sums
+      int32_t cnt[8], lane_sum = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        cnt[i] = hist[255 - 8 * tid - i];
+        lane_sum += cnt[i];
       }
-      sh_prefix = prefix | ((uint32_t)b << shift);
-      sh_need = need - acc;
+      int32_t inc = lane_sum;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) {
+        const int32_t x = __shfl_up_sync(0xffffffffu, inc, d);
+        if (tid >= d) inc += x;
+      }
+      int32_t acc = inc - lane_sum;  // keys in the bins above this lane's
+      if (acc < need && need <= inc) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (acc + cnt[i] >= need) {
+            sh_prefix = prefix | ((uint32_t)(255 - 8 * tid - i) << shift);
+            sh_need = need - acc;
+            break;
+          }
+          acc += cnt[i];
+        }
+      }
     }
     __syncthreads();
     prefix = sh_prefix;
@@ -162,7 +233,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
     int32_t n_gt = 0, n_eq = 0;
 #pragma unroll
     for (int i = 0; i < kSelItems; ++i) {
-      keys[i] = (j0 + i < nr) ? order_key(__ldg(seg + j0 + i)) : 0u;
+      keys[i] = (j0 + i < nr) ? key_at(j0 + i) : 0u;
       const bool valid = j0 + i < nr;
       n_gt += (valid && keys[i] > thr);
       n_eq += (valid && keys[i] == thr);
@@ -246,14 +317,38 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
   }
   const int64_t T = batch->total_tokens;
   if (n_layers == 0 || T == 0 || batch->n_req == 0) return PUREKV_OK;
+  cudaStream_t sm = (cudaStream_t)stream;
+  const int32_t cpr = (int32_t)(head_dim * esz / 16);
+  dim3 g2((unsigned)batch->n_req, (unsigned)n_kv_heads, (unsigned)n_layers);
+  const int32_t k_tot = h_cu_kept[batch->n_req];
+  // Fused path: each (request, head, layer) segment is streamed, scored and selected by one CTA.  It needs 256-byte
+  // rows, the segment's keys in shared memory, and enough segments to occupy the SMs; otherwise V is streamed by a
+  // grid-wide kernel first and the selection reads the scores back.
+  int32_t longest = 0;
+  for (int r = 0; r < batch->n_req; ++r) longest = std::max(longest, batch->h_cu_seqlens[r + 1] - batch->h_cu_seqlens[r]);
+  const size_t key_bytes = (size_t)longest * sizeof(uint32_t);
+  const int64_t segments = (int64_t)batch->n_req * n_kv_heads * n_layers;
+  if (cpr == 16 && key_bytes <= 200 * 1024 && segments >= 2 * 148) {
+    if (dtype == PUREKV_BF16) {
+      PK_CUDA(cudaFuncSetAttribute(select_kernel<true, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
+      select_kernel<true, __nv_bfloat16><<<g2, kSelThreads, key_bytes, sm>>>(
+          nullptr, T, batch->cu_seqlens, cu_kept, keep, window, k_tot, n_kv_heads, idx_out, (const uint4*)v,
+          v_layer_stride * esz / 16, c, s_out);
+    } else {
+      PK_CUDA(cudaFuncSetAttribute(select_kernel<true, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
+      select_kernel<true, float><<<g2, kSelThreads, key_bytes, sm>>>(nullptr, T, batch->cu_seqlens, cu_kept, keep, window,
+                                                                     k_tot, n_kv_heads, idx_out, (const uint4*)v,
+                                                                     v_layer_stride * esz / 16, c, s_out);
+    }
+    PK_CUDA(cudaGetLastError());
+    return PUREKV_OK;
+  }
   float* s_buf = s_out;
   if (!s_buf) {
     PK_REQUIRE(ws && ws_bytes >= purekv_select_ws_bytes(batch, n_layers, n_kv_heads), PUREKV_ERR_WORKSPACE,
                "purekv_select_topk: workspace of %zu bytes is too small", ws_bytes);
     s_buf = (float*)(((uintptr_t)ws + 255) & ~(uintptr_t)255);
   }
-  cudaStream_t sm = (cudaStream_t)stream;
-  const int32_t cpr = (int32_t)(head_dim * esz / 16);
   const int64_t n_blocks = (T + 31) / 32;
   // 148 SMs x 8 resident CTAs shared by the (head, layer) planes of the grid.
   const int64_t planes = (int64_t)n_kv_heads * n_layers;
@@ -266,9 +361,12 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
     vnorm_score_kernel<float><<<g1, 256, 0, sm>>>((const uint4*)v, v_layer_stride * esz / 16, c, T, n_kv_heads, cpr,
                                                   s_buf);
   PK_CUDA(cudaGetLastError());
-  dim3 g2((unsigned)batch->n_req, (unsigned)n_kv_heads, (unsigned)n_layers);
-  select_kernel<<<g2, kSelThreads, 0, sm>>>(s_buf, T, batch->cu_seqlens, cu_kept, keep, window, h_cu_kept[batch->n_req],
-                                            n_kv_heads, idx_out);
+  const bool stage_keys = key_bytes <= 200 * 1024;
+  if (stage_keys)
+    PK_CUDA(cudaFuncSetAttribute(select_kernel<false, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
+  select_kernel<false, float><<<g2, kSelThreads, stage_keys ? key_bytes : 0, sm>>>(
+      s_buf, T, batch->cu_seqlens, cu_kept, keep, window, k_tot, n_kv_heads, idx_out, nullptr, 0, nullptr,
+      stage_keys ? s_buf : nullptr);
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
 }

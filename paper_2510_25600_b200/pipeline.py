@@ -47,6 +47,10 @@ class PureKVPipeline:
         self.plan_buf_st = torch.empty(max(1, P.purekv_plan_bytes(self.batch, self.params_st, self.code, head_dim, *hh)),
                                        dtype=torch.uint8, device=dev)
         self.prefill_ws = None
+        self._h_plans = [(torch.empty(self.plan_buf_dense.numel(), dtype=torch.uint8, pin_memory=True),
+                          torch.empty(self.plan_buf_st.numel(), dtype=torch.uint8, pin_memory=True)) for _ in range(3)]
+        self._h_plan_events = [None] * len(self._h_plans)
+        self._plan_slot = 0
         self.o = torch.empty((n_layers, t, n_q_heads, head_dim), dtype=dtype, device=dev)
         self.c = torch.empty((len(self.scored), n_kv_heads, t), dtype=torch.float32, device=dev)
         self.score_ws = torch.empty(P.purekv_score_ws_bytes(self.batch, window, n_q_heads), dtype=torch.uint8, device=dev)
@@ -60,10 +64,23 @@ class PureKVPipeline:
         self.launches_per_step = n_layers + 2 * len(self.scored) + 2 + 1   # prefill, score (2 kernels), select (2), compact
 
     def build_plans(self) -> None:
-        self.plan_dense = P.purekv_plan_build(self.batch, self.params_dense, self.code, self.d, self.h, self.hkv,
-                                              self.plan_buf_dense)
-        self.plan_st = P.purekv_plan_build(self.batch, self.params_st, self.code, self.d, self.h, self.hkv,
-                                           self.plan_buf_st)
+        """Plans both masks on the host into pinned buffers and enqueues their copies on the current stream without
+        waiting, so planning overlaps the GPU work already in flight.  A small ring of pinned buffers keeps a plan
+        alive until its copy has run."""
+        slot = self._plan_slot
+        self._plan_slot = (slot + 1) % len(self._h_plans)
+        if self._h_plan_events[slot] is not None:
+            self._h_plan_events[slot].synchronize()
+        plans = []
+        for params, h_buf, d_buf in ((self.params_dense, self._h_plans[slot][0], self.plan_buf_dense),
+                                     (self.params_st, self._h_plans[slot][1], self.plan_buf_st)):
+            h_used, info = P.purekv_plan_build_host(self.batch, params, self.code, self.d, self.h, self.hkv, out=h_buf)
+            d_buf[:info.bytes_used].copy_(h_used, non_blocking=True)
+            plans.append(P.Plan(d_buf, info))
+        ev = torch.cuda.Event()
+        ev.record()
+        self._h_plan_events[slot] = ev
+        self.plan_dense, self.plan_st = plans
         need = max(16, self.plan_dense.info.ws_bytes, self.plan_st.info.ws_bytes)
         if self.prefill_ws is None or self.prefill_ws.numel() < need:
             self.prefill_ws = torch.empty(need, dtype=torch.uint8, device="cuda")

@@ -167,6 +167,14 @@ def test_compress_small(dtype, d, window, keep):
     check_compress(wl, 3, window, keep)
 
 
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("fp32", 64)])
+@pytest.mark.parametrize("window,keep", [(8, 0.3), (40, 0.05), (8, 1.0)])
+def test_compress_many_segments(dtype, d, window, keep):
+    # 3 requests x 4 KV heads x 25 layers = 300 segments of 256-byte rows: the selection kernel streams V itself
+    wl = make_wl(dtype, 8, 4, d, [5, 0, 9], [4, 3, 0], [17, 45, 30], 5, 6, 64)
+    check_compress(wl, 25, window, keep)
+
+
 def test_compress_cfg0():
     wl = inputs.workload(0)
     check_compress(wl, 1, wl.window, wl.keep_ratio)
