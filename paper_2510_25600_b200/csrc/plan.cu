@@ -102,17 +102,26 @@ purekv_status purekv_budget(int32_t len, int32_t window, double keep_ratio, int3
 }
 
 // Splits long kept-key lists into chunks and assigns (query tile, head pair, chunk) units to n_ctas persistent
-// CTAs, longest first onto the least loaded CTA.  The cost of a unit is its tile count plus a fixed overhead
-// (query load, pipeline fill, epilogue), in tiles.
-static void schedule_units(const std::vector<QTile>& qtiles, int32_t H, int32_t Hkv, int32_t n_ctas, int32_t tk,
+// CTAs, longest first onto the least loaded CTA.  Costs are in 64-key halves of a list entry: one per present
+// half, a fixed overhead per unit (query load, pipeline fill, epilogue: about three full entries as measured),
+// and a little more for a chunk of a split list (partial result written out, possibly the merge).
+static void schedule_units(const std::vector<QTile>& qtiles, const std::vector<int2>& entries, int32_t H, int32_t Hkv,
+                           int32_t n_ctas,
                            std::vector<Unit>& units, std::vector<int32_t>& cta_off, int32_t* n_counters,
                            int64_t* part_slots, int32_t* max_chunks) {
   const int32_t G = H / Hkv, ppg = (G + 1) / 2, n_pairs = Hkv * ppg;
-  const int32_t overhead = tk >= 128 ? 2 : 3;
+  const int32_t overhead = 6, split_extra = 3;
+  auto halves = [&](int32_t first, int32_t last) {  // cost of entries [first, last)
+    int32_t c = 0;
+    for (int32_t i = first; i < last; ++i) c += ((entries[i].x >> 2) & 3) == 3 ? 2 : 1;
+    return c;
+  };
   int64_t total = 0;
-  for (const QTile& q : qtiles) total += (int64_t)n_pairs * (q.entry_count + overhead);
-  const int64_t target = std::max<int64_t>(1, total / n_ctas);
-  const int32_t l_max = (int32_t)std::min<int64_t>(64, std::max<int64_t>(4, target / 2));
+  for (const QTile& q : qtiles)
+    total += (int64_t)n_pairs * (halves(q.entry_begin, q.entry_begin + q.entry_count) + overhead);
+  const int64_t target = std::max<int64_t>(1, total / n_ctas);  // halves per CTA
+  // longest list (in entries) a unit may carry: about a third of a CTA's share
+  const int32_t l_max = (int32_t)std::min<int64_t>(64, std::max<int64_t>(3, target / 6));
   struct Item { Unit u; int32_t cost; };
   std::vector<Item> items;
   int32_t counters = 0, mc = 1;
@@ -131,7 +140,7 @@ static void schedule_units(const std::vector<QTile>& qtiles, int32_t H, int32_t 
         u.pair = pr; u.chunk = c; u.n_chunks = nch;
         u.part_base = part_base; u.counter_base = counter_base;
         u.pad[0] = u.pad[1] = 0;
-        items.push_back({u, e - a + overhead});
+        items.push_back({u, halves(u.ent_begin, u.ent_begin + u.ent_count) + overhead + (nch > 1 ? split_extra : 0)});
       }
     }
   }
@@ -330,7 +339,7 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   int32_t n_counters = 0, max_chunks = 1;
   int64_t part_slots = 0;
   if (tq == 128 && nq > 0) {
-    schedule_units(qtiles, n_q_heads, n_kv_heads, n_ctas, tk, units, cta_off, &n_counters, &part_slots, &max_chunks);
+    schedule_units(qtiles, entries, n_q_heads, n_kv_heads, n_ctas, units, cta_off, &n_counters, &part_slots, &max_chunks);
   } else {
     n_ctas = 0;
   }
