@@ -35,6 +35,29 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one ST-SpAttn launch of the tensor-core prefill
+# kernel, from the ncu capture summarised under profiles/.  It is reported only while the kernel and planner
+# sources are the ones the capture was taken from (sha1 of their text); otherwise the roofline's traffic is null.
+NCU_TRAFFIC = {"cfg1_videollama2": {"bytes_per_launch": None, "source_sha1": None}}
+KERNEL_SOURCES = ("prefill_tc.cu", "plan.cu", "common.cuh", "prefill.cuh")
+
+
+def kernel_source_sha1() -> str:
+    import hashlib
+    h = hashlib.sha1()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2510_25600_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def ncu_traffic(workload: str):
+    rec = NCU_TRAFFIC.get(workload)
+    if rec and rec["bytes_per_launch"] is not None and rec["source_sha1"] == kernel_source_sha1():
+        return rec["bytes_per_launch"]
+    return None
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -222,7 +245,11 @@ def main():
     ap.add_argument("--impl", default="purekv")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--print-kernel-hash", action="store_true", help="sha1 of the prefill kernel sources, then exit")
     args = ap.parse_args()
+    if args.print_kernel_hash:
+        print(kernel_source_sha1())
+        return
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
     from paper_2510_25600_b200 import inputs
@@ -302,7 +329,8 @@ def main():
     achieved = flops_step / (prefill_ms_step * 1e-3) / 1e12
     peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
     roofline = {"kernel": f"prefill_tc_kernel (128-key entries, skip granularity {info_s.tile_k})", "bound": "tensor", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": ncu_traffic(wl.name),
+                "algorithmic_bytes_per_launch": b.total_tokens * wl.head_dim * 2 * (2 * wl.n_q_heads + 2 * wl.n_kv_heads),
                 "peak_kind": f"{peak_kind} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']}, nominal dense 2250)",
                 "flops_per_step": flops_step, "launches_per_step": wl.n_layers, "avg_launch_ms": prefill_ms_step / wl.n_layers,
                 "st_layer_ms": float(k_ms[:, n_dense:].mean()) if wl.n_layers > n_dense else None,

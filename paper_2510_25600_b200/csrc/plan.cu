@@ -102,26 +102,27 @@ purekv_status purekv_budget(int32_t len, int32_t window, double keep_ratio, int3
 }
 
 // Splits long kept-key lists into chunks and assigns (query tile, head pair, chunk) units to n_ctas persistent
-// CTAs, longest first onto the least loaded CTA.  Costs are in 64-key halves of a list entry: one per present
-// half, a fixed overhead per unit (query load, pipeline fill, epilogue: about three full entries as measured),
-// and a little more for a chunk of a split list (partial result written out, possibly the merge).
+// CTAs, longest first onto the least loaded CTA.  Costs are in quarters of a 64-key half of a list entry, fitted to
+// measured CTA times: 4 per present half (5 when the entry carries a bit mask), 10 per unit (query load, pipeline
+// fill, epilogue) and 28 more for a chunk of a split list (fp32 partial result written out, and the merge).
 static void schedule_units(const std::vector<QTile>& qtiles, const std::vector<int2>& entries, int32_t H, int32_t Hkv,
                            int32_t n_ctas,
                            std::vector<Unit>& units, std::vector<int32_t>& cta_off, int32_t* n_counters,
                            int64_t* part_slots, int32_t* max_chunks) {
   const int32_t G = H / Hkv, ppg = (G + 1) / 2, n_pairs = Hkv * ppg;
-  const int32_t overhead = 6, split_extra = 3;
+  const int32_t overhead = 10, split_extra = 28;
   auto halves = [&](int32_t first, int32_t last) {  // cost of entries [first, last)
     int32_t c = 0;
-    for (int32_t i = first; i < last; ++i) c += ((entries[i].x >> 2) & 3) == 3 ? 2 : 1;
+    for (int32_t i = first; i < last; ++i)
+      c += ((((entries[i].x >> 2) & 3) == 3) ? 2 : 1) * ((entries[i].x & 3) == kTileGeneral ? 5 : 4);
     return c;
   };
   int64_t total = 0;
   for (const QTile& q : qtiles)
     total += (int64_t)n_pairs * (halves(q.entry_begin, q.entry_begin + q.entry_count) + overhead);
-  const int64_t target = std::max<int64_t>(1, total / n_ctas);  // halves per CTA
-  // longest list (in entries) a unit may carry: about a third of a CTA's share
-  const int32_t l_max = (int32_t)std::min<int64_t>(64, std::max<int64_t>(3, target / 6));
+  const int64_t target = std::max<int64_t>(1, total / n_ctas);  // cost per CTA
+  // longest list (in entries of 8 cost units) a unit may carry: about 40 % of a CTA's share
+  const int32_t l_max = (int32_t)std::min<int64_t>(64, std::max<int64_t>(3, target / 20));
   struct Item { Unit u; int32_t cost; };
   std::vector<Item> items;
   int32_t counters = 0, mc = 1;
