@@ -12,15 +12,18 @@ __global__ void __launch_bounds__(256) compact_kernel(
     const uint4* __restrict__ k, const uint4* __restrict__ v, int64_t layer_stride_c /* chunks */,
     const int32_t* __restrict__ idx, const int32_t* __restrict__ cu_seqlens, const int32_t* __restrict__ cu_kept,
     int32_t n_req, int32_t k_tot, int32_t n_kv_heads, int32_t chunks_per_row, uint4* __restrict__ k_out,
-    uint4* __restrict__ v_out, int64_t out_layer_stride_c, int64_t total_chunks_per_layer) {
-  const int32_t layer = blockIdx.y;
-  const int32_t* idx_l = idx + (int64_t)layer * n_kv_heads * k_tot;
-  const uint4* k_l = k + layer * layer_stride_c;
-  const uint4* v_l = v + layer * layer_stride_c;
-  uint4* ko = k_out + layer * out_layer_stride_c;
-  uint4* vo = v_out + layer * out_layer_stride_c;
+    uint4* __restrict__ v_out, int64_t out_layer_stride_c, int64_t total_chunks_per_layer, int32_t n_layers) {
+  // one-dimensional grid of at most one full wave; the threads stride over the chunks of all layers
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < total_chunks_per_layer; x += stride) {
+  const int64_t total = total_chunks_per_layer * n_layers;
+  for (int64_t xf = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; xf < total; xf += stride) {
+    const int32_t layer = (int32_t)(xf / total_chunks_per_layer);
+    const int64_t x = xf - layer * total_chunks_per_layer;
+    const int32_t* idx_l = idx + (int64_t)layer * n_kv_heads * k_tot;
+    const uint4* k_l = k + layer * layer_stride_c;
+    const uint4* v_l = v + layer * layer_stride_c;
+    uint4* ko = k_out + layer * out_layer_stride_c;
+    uint4* vo = v_out + layer * out_layer_stride_c;
     const int32_t chunk = (int32_t)(x % chunks_per_row);
     const int64_t row = x / chunks_per_row;  // = t * n_kv_heads + g
     const int32_t g = (int32_t)(row % n_kv_heads);
@@ -78,14 +81,12 @@ extern "C" purekv_status purekv_compact_kv(const void* k, const void* v, int64_t
   if (n_layers == 0 || k_tot == 0) return PUREKV_OK;
   const int32_t cpr = (int32_t)(row_bytes / 16);
   const int64_t per_layer = (int64_t)k_tot * n_kv_heads * cpr;
-  const int64_t blocks = (per_layer + 255) / 256;
-  // 148 SMs x 8 resident CTAs of 256 threads; fewer blocks when the layer is small.
-  const int32_t max_x = std::max<int64_t>(1, (148 * 8 + n_layers - 1) / n_layers);
-  dim3 grid((unsigned)std::min<int64_t>(blocks, max_x), (unsigned)n_layers);
-  PK_REQUIRE(n_layers <= 65535, PUREKV_ERR_UNSUPPORTED, "more than 65535 layers per call");
+  const int64_t blocks = (per_layer * n_layers + 255) / 256;
+  // one wave: 148 SMs x 8 resident CTAs of 256 threads; fewer blocks when the job is small
+  dim3 grid((unsigned)std::min<int64_t>(blocks, 148 * 8));
   compact_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(
       (const uint4*)k, (const uint4*)v, layer_stride * esz / 16, idx, batch->cu_seqlens, cu_kept, batch->n_req, k_tot,
-      n_kv_heads, cpr, (uint4*)k_out, (uint4*)v_out, out_layer_stride * esz / 16, per_layer);
+      n_kv_heads, cpr, (uint4*)k_out, (uint4*)v_out, out_layer_stride * esz / 16, per_layer, n_layers);
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
 }

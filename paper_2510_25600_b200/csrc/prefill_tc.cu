@@ -255,8 +255,8 @@ __device__ __forceinline__ void setmaxnreg_dec() { asm volatile("setmaxnreg.dec.
 
 template <int BK>
 struct Cfg {
-  static constexpr int kStages = BK == 64 ? 4 : 2;  // K/V ring depth (32 KB resp. 64 KB per stage)
-  static constexpr int kSBuf = BK == 64 ? 2 : 1;    // S buffers per slot: kSBuf * BK = 128 TMEM columns
+  static constexpr int kStages = 2;                 // K/V ring depth (64 KB per stage)
+  static constexpr int kSBuf = 128 / BK;            // S buffers per slot: kSBuf * BK = 128 TMEM columns
   static constexpr int kMeta = 2 * kStages;         // ring of per-tile class words and bit masks
   static constexpr uint32_t kMaskBytes = kBQ * BK / 8;
 };
@@ -596,13 +596,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         if (cls == kTileGeneral) {  // this row's bits of the tile's mask
           const uint32_t* mrow = reinterpret_cast<const uint32_t*>(smem_raw + (sM - smem_u32(smem_raw)) + ms * kMaskBytes) +
                                  row * (BK / 32);
-          if constexpr (BK == 128) {
-            const uint4 w4 = *reinterpret_cast<const uint4*>(mrow);
-            keep[0] = w4.x; keep[1] = w4.y; keep[BK / 32 - 2] = w4.z; keep[BK / 32 - 1] = w4.w;
-          } else {
-            const uint2 w2 = *reinterpret_cast<const uint2*>(mrow);
-            keep[0] = w2.x; keep[1] = w2.y;
-          }
+          static_assert(BK == 128, "a mask row is four 32-bit words");
+          const uint4 w4 = *reinterpret_cast<const uint4*>(mrow);
+          keep[0] = w4.x; keep[1] = w4.y; keep[2] = w4.z; keep[3] = w4.w;
         } else if (cls == kTileDiag) {
           const int32_t n_ok = min(BK, max(0, i_rel - j0 + 1));  // causal: columns 0 .. n_ok-1
 #pragma unroll

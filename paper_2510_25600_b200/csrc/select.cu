@@ -1,11 +1,11 @@
 // purekv_select_topk: V-norm weighting (Eq. 3 / Eq. 4) and budgeted top-h selection (Sec. 3.1).
 //
-// Two kernels.  vnorm_score_kernel streams V once (the only large traffic of this step):
-// a warp owns 32 consecutive tokens of one KV head, each half-warp reads one 16-byte-chunked
-// row per step, reduces the squared norm with shuffles, and the warp writes 32 consecutive
-// scores S = C * ||V||.  select_kernel then handles one (layer, KV head, request) segment per
-// CTA: a 4 x 8-bit MSB-first radix select over the fp32 bit patterns finds the h-th largest
-// score, and a block-scan compaction emits the chosen positions in ascending order; among
+// Two paths.  With few (request, head, layer) segments, vnorm_score_kernel streams V once over the whole GPU (the
+// only large traffic of this step): a warp owns 32 consecutive (token, head) rows, each half-warp reads one
+// 16-byte-chunked row per step and reduces the squared norm with shuffles; select_kernel then handles one segment
+// per CTA.  With many segments one CTA does both for its segment and the scores never leave the SM.  The selection
+// is a 4 x 8-bit MSB-first radix select over the fp32 bit patterns (keys staged in shared memory) that finds the
+// h-th largest score, then a block-scan compaction that emits the chosen positions in ascending order; among
 // scores equal to the threshold the lowest positions win, so the result is deterministic.
 #include <algorithm>
 
@@ -38,30 +38,33 @@ struct Chunk<__nv_bfloat16> {
   }
 };
 
-// grid: (ceil(T/32) token blocks split over x, n_kv_heads, n_layers); block: 256 threads = 8 warps.
+// grid: one dimension, at most 8 CTAs per SM (a single full wave whatever the number of layers and heads); the warps
+// stride over blocks of 32 consecutive (token, head) rows of a layer, i.e. over contiguous memory.
+// block: 256 threads = 8 warps.
 template <typename T>
 __global__ void __launch_bounds__(256) vnorm_score_kernel(const uint4* __restrict__ v, int64_t layer_stride_c,
                                                           const float* __restrict__ c, int64_t n_tokens,
-                                                          int32_t n_kv_heads, int32_t chunks_per_row,
+                                                          int32_t n_kv_heads, int32_t n_layers, int32_t chunks_per_row,
                                                           float* __restrict__ s_out) {
   const int32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int32_t g = blockIdx.y, layer = blockIdx.z;
-  const uint4* vl = v + layer * layer_stride_c;
-  float* so = s_out + ((int64_t)layer * n_kv_heads + g) * n_tokens;
-  const float* cg = c + (int64_t)g * n_tokens;
-  const int64_t n_blocks = (n_tokens + 31) / 32;
-  for (int64_t blk = (int64_t)blockIdx.x * 8 + warp; blk < n_blocks; blk += (int64_t)gridDim.x * 8) {
-    const int64_t t0 = blk * 32;
+  const int64_t n_rows = n_tokens * n_kv_heads;  // rows of one layer, row = token * n_kv_heads + head
+  const int64_t n_blocks = (n_rows + 31) / 32;
+  const int64_t n_items = n_blocks * n_layers;
+  for (int64_t item = (int64_t)blockIdx.x * 8 + warp; item < n_items; item += (int64_t)gridDim.x * 8) {
+    const int64_t blk = item % n_blocks;
+    const int32_t layer = (int32_t)(item / n_blocks);
+    const uint4* vl = v + layer * layer_stride_c;
+    const int64_t r0 = blk * 32;
     float mine = 0.f;
     if (chunks_per_row == 16) {
-      // 256-byte rows: a half-warp covers one row per step, 16 steps cover 32 tokens.
+      // 256-byte rows: a half-warp covers one row per step, 16 steps cover 32 rows (8 KB of contiguous memory).
       const int32_t half = lane >> 4, ch = lane & 15;
       float part[16];
 #pragma unroll
       for (int it = 0; it < 16; ++it) {
-        const int64_t t = t0 + it * 2 + half;
+        const int64_t r = r0 + it * 2 + half;
         uint4 u = make_uint4(0, 0, 0, 0);
-        if (t < n_tokens) u = __ldg(vl + (t * n_kv_heads + g) * 16 + ch);
+        if (r < n_rows) u = __ldg(vl + r * 16 + ch);
         part[it] = Chunk<T>::sumsq(u);
       }
 #pragma unroll
@@ -71,21 +74,25 @@ __global__ void __launch_bounds__(256) vnorm_score_kernel(const uint4* __restric
         p += __shfl_xor_sync(0xffffffffu, p, 4);
         p += __shfl_xor_sync(0xffffffffu, p, 2);
         p += __shfl_xor_sync(0xffffffffu, p, 1);
-        // lanes 0..15 now hold token 2*it's sum, lanes 16..31 token 2*it+1's; lane L keeps token L
+        // lanes 0..15 now hold row 2*it's sum, lanes 16..31 row 2*it+1's; lane L keeps row L
         const float v0 = __shfl_sync(0xffffffffu, p, 0), v1 = __shfl_sync(0xffffffffu, p, 16);
         if (lane == it * 2) mine = v0;
         if (lane == it * 2 + 1) mine = v1;
       }
     } else {
-      // generic row length: one token per lane, sequential chunks
-      const int64_t t = t0 + lane;
-      if (t < n_tokens) {
-        const uint4* row = vl + (t * n_kv_heads + g) * chunks_per_row;
+      // generic row length: one row per lane, sequential chunks
+      const int64_t r = r0 + lane;
+      if (r < n_rows) {
+        const uint4* row = vl + r * chunks_per_row;
         for (int32_t ch = 0; ch < chunks_per_row; ++ch) mine += Chunk<T>::sumsq(__ldg(row + ch));
       }
     }
-    const int64_t t = t0 + lane;
-    if (t < n_tokens) so[t] = __ldg(cg + t) * sqrtf(mine);
+    const int64_t r = r0 + lane;
+    if (r < n_rows) {
+      const int64_t t = r / n_kv_heads;
+      const int32_t g = (int32_t)(r % n_kv_heads);
+      s_out[((int64_t)layer * n_kv_heads + g) * n_tokens + t] = __ldg(c + (int64_t)g * n_tokens + t) * sqrtf(mine);
+    }
   }
 }
 
@@ -349,17 +356,14 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
                "purekv_select_topk: workspace of %zu bytes is too small", ws_bytes);
     s_buf = (float*)(((uintptr_t)ws + 255) & ~(uintptr_t)255);
   }
-  const int64_t n_blocks = (T + 31) / 32;
-  // 148 SMs x 8 resident CTAs shared by the (head, layer) planes of the grid.
-  const int64_t planes = (int64_t)n_kv_heads * n_layers;
-  const int64_t want = std::max<int64_t>(1, (148 * 8 + planes - 1) / planes);
-  dim3 g1((unsigned)std::min<int64_t>((n_blocks + 7) / 8, want), (unsigned)n_kv_heads, (unsigned)n_layers);
+  const int64_t n_items = ((T * n_kv_heads + 31) / 32) * n_layers;  // blocks of 32 (token, head) rows per layer
+  dim3 g1((unsigned)std::min<int64_t>((n_items + 7) / 8, 148 * 4));   // one wave: 4 CTAs of 256 threads per SM (measured best)
   if (dtype == PUREKV_BF16)
     vnorm_score_kernel<__nv_bfloat16><<<g1, 256, 0, sm>>>((const uint4*)v, v_layer_stride * esz / 16, c, T, n_kv_heads,
-                                                          cpr, s_buf);
+                                                          n_layers, cpr, s_buf);
   else
-    vnorm_score_kernel<float><<<g1, 256, 0, sm>>>((const uint4*)v, v_layer_stride * esz / 16, c, T, n_kv_heads, cpr,
-                                                  s_buf);
+    vnorm_score_kernel<float><<<g1, 256, 0, sm>>>((const uint4*)v, v_layer_stride * esz / 16, c, T, n_kv_heads, n_layers,
+                                                  cpr, s_buf);
   PK_CUDA(cudaGetLastError());
   const bool stage_keys = key_bytes <= 200 * 1024;
   if (stage_keys)
