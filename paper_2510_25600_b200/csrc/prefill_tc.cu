@@ -34,7 +34,10 @@ constexpr int kD = 128;
 constexpr int kBQ = 128;
 constexpr int kThreads = 384;  // warps 0-3 softmax of slot 0, warps 4-7 of slot 1, warp 8 producer, warp 9 MMA, 10-11 idle
 constexpr int kWarpProducer = 8, kWarpMma = 9;
-constexpr int kRegsSoftmax = 208, kRegsOther = 88;  // per-thread registers after the warpgroups trade them
+// Per-thread registers after the warpgroups trade them.  setmaxnreg only moves registers inside the CTA's launch
+// allocation (kThreads x the count ptxas gives the kernel, 168 at 384 threads); asking for more would block forever,
+// so the launch code checks the budget against the compiled register count.
+constexpr int kRegsSoftmax = 208, kRegsOther = 88;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 256;
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
@@ -898,6 +901,14 @@ static purekv_status launch(const PrefillArgs& a, const CUtensorMap& mq, const C
   constexpr int BK = 128;
   const size_t smem = 1024 + 2 * 2 * (size_t)kBQ * 128 + 2 * (size_t)Cfg<BK>::kStages * 2 * BK * 128 +
                       (size_t)Cfg<BK>::kMeta * Cfg<BK>::kMaskBytes;
+  static int launch_regs = 0;
+  if (launch_regs == 0) {
+    cudaFuncAttributes fa;
+    PK_CUDA(cudaFuncGetAttributes(&fa, prefill_tc_kernel<BK>));
+    launch_regs = fa.numRegs;
+  }
+  PK_REQUIRE(256 * kRegsSoftmax + 128 * kRegsOther <= kThreads * launch_regs, PUREKV_ERR_UNSUPPORTED,
+             "prefill kernel was compiled with %d registers per thread, too few for its register hand-over", launch_regs);
   PK_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid((unsigned)a.info->n_ctas);
   prefill_tc_kernel<BK><<<grid, kThreads, smem, a.stream>>>(mq, mk, mv, mk64, mv64, (__nv_bfloat16*)a.o, a.lse,
