@@ -459,7 +459,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
       const uint32_t v_lo0 = ((sV & 0x3FFFFu) >> 4) | ((kPanelKV >> 4) << 16);
       // S(slot, n) = Q_slot K_n^T; the last slot to read K_n releases its stage
-      auto issue_qk = [&](int32_t sl, int32_t n) -> bool {
+      auto issue_qk = [&](auto sl_c, int32_t n) -> bool {
+        constexpr int sl = decltype(sl_c)::value;  // compile-time slot: the per-slot counters stay in registers
         const uint32_t it = it_base + (uint32_t)n;
         const uint32_t s = it % ST, b = tq[sl] % SB;
         // the stage was already awaited for slot 0 of the same tile
@@ -491,7 +492,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         return true;
       };
       // O(slot) += P(slot, n) V_n; the last slot to read V_n releases its stage
-      auto issue_pv = [&](int32_t sl, int32_t n) -> bool {
+      auto issue_pv = [&](auto sl_c, int32_t n) -> bool {
+        constexpr int sl = decltype(sl_c)::value;
         const uint32_t it = it_base + (uint32_t)n;
         const uint32_t s = it % ST, b = tp[sl] % SB;
         if (sl == 0 && !mbar_wait(smem_u32(&bars.v_full[s]), (it / ST) & 1u, abort_flag)) return false;
@@ -526,13 +528,20 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         nt = u.ent_count;
         n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
         ok = mbar_wait(smem_u32(&bars.q_full), (uint32_t)(k - u_begin) & 1u, abort_flag);
-        for (int32_t n = 0; ok && n < SB && n < nt; ++n)
-          for (int32_t sl = 0; ok && sl < n_slots; ++sl) ok = issue_qk(sl, n);
-        for (int32_t n = 0; ok && n < nt; ++n)
-          for (int32_t sl = 0; ok && sl < n_slots; ++sl) {
-            ok = issue_pv(sl, n);
-            if (ok && n + SB < nt) ok = issue_qk(sl, n + SB);  // in order behind P.V of tile n, which frees S(slot, n % SB)
+        constexpr std::integral_constant<int, 0> s0{};
+        constexpr std::integral_constant<int, 1> s1{};
+        for (int32_t n = 0; ok && n < SB && n < nt; ++n) {
+          ok = issue_qk(s0, n);
+          if (ok && n_slots == 2) ok = issue_qk(s1, n);
+        }
+        for (int32_t n = 0; ok && n < nt; ++n) {
+          ok = issue_pv(s0, n);
+          if (ok && n + SB < nt) ok = issue_qk(s0, n + SB);  // in order behind P.V of tile n, which frees S(slot, n % SB)
+          if (ok && n_slots == 2) {
+            ok = issue_pv(s1, n);
+            if (ok && n + SB < nt) ok = issue_qk(s1, n + SB);
           }
+        }
         it_base += (uint32_t)nt;
         u = nxt;
       }
