@@ -236,6 +236,75 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
+def run_sweep(args):
+    """--sweep: the long-video workload (cfg 3) under masks of growing block density, and its compression at
+    three keep ratios.  Prints one JSON line with a table; a companion to the default line, not a replacement."""
+    import torch
+    from paper_2510_25600_b200 import binding as P, inputs
+    wl = inputs.workload(3)
+    b = wl.batch
+    peaks, peak_kind = load_peaks()
+    pool = ThreadPoolExecutor(len(os.sched_getaffinity(0)))
+    x = inputs.make_qkv(wl, 0, pool=pool)
+    up = lambda n: torch.from_numpy(x[n + "_bits"].view(np.int16)).cuda().view(torch.bfloat16)
+    q, k, v = up("q"), up("k"), up("v")
+    db = P.Batch(b.seq_lens, b.n_prefix, b.n_frames)
+    g = b.grid_h
+    M = inputs.STMask
+    masks = [("paper mask", wl.mask)]
+    masks += [(f"whole-frame links, depth {d}", M(g, g, 1, -1, d, 1, -1, tile=128)) for d in (1, 2, 4, 8, 16)]
+    masks += [(f"same cell of all earlier frames at stride {st}", M(g, g, 1, -1, -1, st, 0, tile=128)) for st in (10, 5, 3)]
+    masks += [("spatial radius 4", M(g, g, 1, 4, 1, 1, 0, tile=128)), ("dense causal", M(g, g, tile=128, dense_causal=True))]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    o = torch.empty_like(q)
+
+    def timed(fn, reps):
+        out = []
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            out.append(e0.elapsed_time(e1))
+        return float(np.median(out))
+
+    rows = []
+    peak = float(peaks["bf16_tflops"])
+    for name, m in masks:
+        plan = P.purekv_plan_build(db, P.st_params(m), P.BF16, wl.head_dim, wl.n_q_heads, wl.n_kv_heads)
+        ws = torch.empty(max(16, plan.info.ws_bytes), dtype=torch.uint8, device="cuda")
+        fn = lambda: P.purekv_st_sparse_prefill(q, k, v, db, plan, out=o, status=status, ws=ws)
+        for _ in range(3):
+            fn()
+        ms = timed(fn, max(3, min(args.steps, 10)))
+        info = plan.info
+        tf = 4.0 * info.tile_q * info.tile_k * wl.head_dim * wl.n_q_heads * info.tiles_kept / ms / 1e9
+        rows.append({"mask": name, "block_density": info.tiles_kept / info.tiles_causal, "ms": ms, "TFLOPs": tf,
+                     "frac_of_burst_peak": tf / peak, "tokens_per_s": b.total_tokens / (ms * 1e-3)})
+    P.purekv_poll_status(status)
+    comp = []
+    hbm = float(peaks["hbm_gbs"])
+    kk, vv = k[None].contiguous(), v[None].contiguous()
+    row = wl.n_kv_heads * wl.head_dim * 2
+    for keep in (0.1, 0.2, 0.5):
+        bud = P.Budget(db, wl.window, keep)
+        c = P.purekv_lowlayer_score(q, k, db, wl.window)
+        idx = P.purekv_select_topk(c, vv, db, bud)
+        t_sel = timed(lambda: P.purekv_select_topk(c, vv, db, bud, idx_out=idx), 5)
+        kc, vc = P.purekv_compact_kv(kk, vv, idx, db, bud)
+        t_cmp = timed(lambda: P.purekv_compact_kv(kk, vv, idx, db, bud, k_out=kc, v_out=vc), 5)
+        by = 4 * bud.total_kept * row + wl.n_kv_heads * bud.total_kept * 4
+        comp.append({"keep_ratio": keep, "kept": bud.total_kept, "select_ms": t_sel, "compact_ms": t_cmp,
+                     "compact_GBps": by / t_cmp / 1e6, "compact_frac_hbm": by / t_cmp / 1e6 / hbm})
+    t_score = timed(lambda: P.purekv_lowlayer_score(q, k, db, wl.window, c_out=c), 5)
+    print(json.dumps({"sweep": wl.name, "tokens": b.total_tokens, "peak_TFLOPs": peak, "peak_kind": peak_kind + " burst (kernel timed alone)",
+                      "prefill": rows, "score_ms": t_score, "compression": comp,
+                      "timing": "cold L2 (256 MiB fill before each call), median"}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -246,12 +315,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--print-kernel-hash", action="store_true", help="sha1 of the prefill kernel sources, then exit")
+    ap.add_argument("--sweep", action="store_true", help="long-video workload: TFLOP/s against block density, compaction")
     args = ap.parse_args()
     if args.print_kernel_hash:
         print(kernel_source_sha1())
         return
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
+    if args.sweep:
+        run_sweep(args)
+        return
     from paper_2510_25600_b200 import inputs
     wl = inputs.workload(args.cfg)
     if args.impl == "reference":
