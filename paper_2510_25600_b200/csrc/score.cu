@@ -227,13 +227,15 @@ static int32_t max_len(const purekv_batch* b) {
 }
 
 // ---- bf16 path on tensor cores ------------------------------------------------------------------
-// Both passes use the same tiling: a CTA owns one block of 64 keys of one (request, KV head) and walks the
-// G*w stacked window rows in blocks of 128; warp wi computes the 16 x 64 logits of rows 16*wi .. 16*wi+15 with
-// mma.sync m16n8k16 (bf16 x bf16 -> fp32: products exact, fp32 accumulation).  Pass 1 leaves, per key block and
-// row, the maximum and the sum of exponentials of the causal logits; a small kernel folds those into the row's
-// log-sum-exp; pass 2 forms exp(s - lse) and sums down the rows.  Every key block is an independent CTA, so the
-// grid is (key blocks) x (KV heads) x (requests) in both passes.
-constexpr int kMmaKeys = 64;
+// Both passes use the same tiling: a CTA owns one block of 128 keys of one (request, KV head) and walks the
+// G*w stacked window rows in blocks of 128; its 8 warps form a 4 x 2 grid, warp (wr, wc) computing the 32 x 64
+// logits of rows 32*wr .. +31 against keys 64*wc .. +63 with mma.sync m16n8k16 (bf16 x bf16 -> fp32: products
+// exact, fp32 accumulation).  Pass 1 leaves, per 64-key block and row, the maximum and the sum of exponentials of
+// the causal logits; a small kernel folds those into the row's log-sum-exp; pass 2 forms exp(s - lse) and sums down
+// the rows.  Every key block is an independent CTA, so the grid is (key blocks) x (KV heads) x (requests) in both
+// passes.
+constexpr int kMmaKeys = 64;    // keys per warp column, and the granularity of the pass-1 (max, sum) pairs
+constexpr int kCtaKeys = 128;   // keys per CTA
 constexpr int kMmaRows = 128;
 constexpr int kMmaThreads = 256;
 
@@ -266,80 +268,119 @@ __device__ __forceinline__ void stage_rows_bf16(__nv_bfloat16* dst, const __nv_b
   }
 }
 
-// acc[nb][0..3] = logits of rows (16*warp + lane/4, +8) x keys (8*nb + 2*(lane%4), +1) of the staged tiles
-__device__ __forceinline__ void logits_16x64(const __nv_bfloat16* qs, const __nv_bfloat16* ks, int d, float (&acc)[8][4]) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, ld = d + 8;
+// The same copy with cp.async (16 bytes per request, zero fill for absent rows): returns at once, the data is
+// there after cp_async_wait.  Used to load the next block of query rows while the current one is multiplied.
+template <typename RowOf>
+__device__ __forceinline__ void stage_rows_bf16_async(__nv_bfloat16* dst, const __nv_bfloat16* src, int rows, int d, RowOf row_of) {
+  const int cpr = d / 8;
+  for (int x = threadIdx.x; x < rows * cpr; x += kMmaThreads) {
+    const int r = x / cpr, c = x % cpr;
+    const int64_t off = row_of(r);
+    const uint32_t sa = (uint32_t)__cvta_generic_to_shared(dst + r * (d + 8) + c * 8);
+    const void* ga = off >= 0 ? (const void*)(reinterpret_cast<const uint4*>(src + off) + c) : (const void*)src;
+    const uint32_t bytes = off >= 0 ? 16u : 0u;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(sa), "l"(ga), "r"(bytes) : "memory");
+  }
+  asm volatile("cp.async.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// acc[mb][nb][0..3] = logits of rows (32*wr + 16*mb + lane/4, +8) x keys (64*wc + 8*nb + 2*(lane%4), +1) of the
+// staged tiles: per 16-wide K step two A fragments and four ldmatrix.x4 of K feed sixteen MMAs.
+__device__ __forceinline__ void logits_32x64(const __nv_bfloat16* qs, const __nv_bfloat16* ks, int d, float (&acc)[2][8][4]) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wr = warp >> 1, wc = warp & 1, ld = d + 8;
 #pragma unroll
-  for (int nb = 0; nb < 8; ++nb)
+  for (int mb = 0; mb < 2; ++mb)
 #pragma unroll
-    for (int x = 0; x < 4; ++x) acc[nb][x] = 0.f;
-  const uint32_t qa = (uint32_t)__cvta_generic_to_shared(qs + (16 * warp + (lane & 7) + 8 * ((lane >> 3) & 1)) * ld + 8 * (lane >> 4));
-  const uint32_t ka = (uint32_t)__cvta_generic_to_shared(ks + (lane & 7) * ld + 8 * ((lane >> 3) & 1));
+    for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+      for (int x = 0; x < 4; ++x) acc[mb][nb][x] = 0.f;
+  const uint32_t qa = (uint32_t)__cvta_generic_to_shared(qs + (32 * wr + (lane & 7) + 8 * ((lane >> 3) & 1)) * ld + 8 * (lane >> 4));
+  // K: one x4 covers two 8-key blocks: matrices (keys +0, k 0-7), (keys +0, k 8-15), (keys +8, k 0-7), (keys +8, k 8-15)
+  const uint32_t ka = (uint32_t)__cvta_generic_to_shared(ks + (64 * wc + (lane & 7) + 8 * (lane >> 4)) * ld + 8 * ((lane >> 3) & 1));
   for (int k0 = 0; k0 < d; k0 += 16) {
-    uint32_t a[4];
-    ldmatrix_x4(qa + k0 * 2, a);
+    uint32_t a0[4], a1[4];
+    ldmatrix_x4(qa + k0 * 2, a0);
+    ldmatrix_x4(qa + (16 * ld + k0) * 2, a1);
 #pragma unroll
-    for (int nb = 0; nb < 8; ++nb) {
-      uint32_t b[2];
-      ldmatrix_x2(ka + (nb * 8 * ld + k0) * 2, b);
-      mma_bf16_16x8x16(acc[nb], a, b);
+    for (int nb = 0; nb < 8; nb += 2) {
+      uint32_t b4[4];
+      ldmatrix_x4(ka + (nb * 8 * ld + k0) * 2, b4);
+      const uint32_t b0[2] = {b4[0], b4[1]}, b1[2] = {b4[2], b4[3]};
+      mma_bf16_16x8x16(acc[0][nb], a0, b0);
+      mma_bf16_16x8x16(acc[1][nb], a1, b0);
+      mma_bf16_16x8x16(acc[0][nb + 1], a0, b1);
+      mma_bf16_16x8x16(acc[1][nb + 1], a1, b1);
     }
   }
 }
 
-// Pass 1.  partial[((r * Hkv + g) * n_kb + kb) * rows_max + row] = (max, sum of exp2) of the causal logits of the
-// stacked row against key block kb, in log2 units of the scaled logits.
+// Pass 1.  partial[((r * Hkv + g) * n_kb + kb64) * rows_max + row] = (max, sum of exp2) of the causal logits of the
+// stacked row against the 64-key block kb64, in log2 units of the scaled logits.
 __global__ void __launch_bounds__(kMmaThreads) score_mma_partial_kernel(
     const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k, const int32_t* __restrict__ cu_seqlens,
     int32_t window, int32_t n_q_heads, int32_t n_kv_heads, int32_t d, float scale_log2, int32_t n_kb, int32_t rows_max,
     float2* __restrict__ partial) {
   extern __shared__ __align__(16) uint8_t smem_mma[];
   __nv_bfloat16* ks = reinterpret_cast<__nv_bfloat16*>(smem_mma);
-  __nv_bfloat16* qs = ks + kMmaKeys * (d + 8);
-  const int32_t r = blockIdx.z, g = blockIdx.y, kb = blockIdx.x;
+  __nv_bfloat16* qs = ks + kCtaKeys * (d + 8);
+  const int32_t r = blockIdx.z, g = blockIdx.y;
   const int32_t G = n_q_heads / n_kv_heads;
   const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
-  const int32_t w = min(window, len), n_rows = G * w, j0 = kb * kMmaKeys;
+  const int32_t w = min(window, len), n_rows = G * w, j0 = blockIdx.x * kCtaKeys;
   if (j0 >= len) return;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  stage_rows_bf16(ks, k, kMmaKeys, d, [&](int rr) -> int64_t {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wr = warp >> 1, wc = warp & 1;
+  stage_rows_bf16(ks, k, kCtaKeys, d, [&](int rr) -> int64_t {
     return j0 + rr < len ? ((int64_t)(base + j0 + rr) * n_kv_heads + g) * d : -1;
   });
-  float2* out = partial + ((int64_t)(r * n_kv_heads + g) * n_kb + kb) * rows_max;
-  for (int32_t row0 = 0; row0 < n_rows; row0 += kMmaRows) {
-    __syncthreads();
-    stage_rows_bf16(qs, q, kMmaRows, d, [&](int rr) -> int64_t {
-      const int32_t row = row0 + rr;
-      return row < n_rows ? ((int64_t)(base + len - w + row % w) * n_q_heads + g * G + row / w) * d : -1;
-    });
-    __syncthreads();
-    float acc[8][4];
-    logits_16x64(qs, ks, d, acc);
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {  // the thread's two rows
-      const int32_t row = row0 + 16 * warp + (lane >> 2) + 8 * h;
-      const int32_t i = row < n_rows ? len - w + row % w : -1;  // causal limit of the row (-1: no row)
-      float m = -INFINITY;
-#pragma unroll
-      for (int nb = 0; nb < 8; ++nb)
-#pragma unroll
-        for (int x = 0; x < 2; ++x) {
-          const int32_t j = j0 + 8 * nb + 2 * (lane & 3) + x;
-          const float s = j <= i ? acc[nb][2 * h + x] * scale_log2 : -INFINITY;
-          acc[nb][2 * h + x] = s;
-          m = fmaxf(m, s);
-        }
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
-      m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
-      float l = 0.f;
-      if (m > -INFINITY) {
-#pragma unroll
-        for (int nb = 0; nb < 8; ++nb) l += exp2f(acc[nb][2 * h] - m) + exp2f(acc[nb][2 * h + 1] - m);
-      }
-      l += __shfl_xor_sync(0xffffffffu, l, 1);
-      l += __shfl_xor_sync(0xffffffffu, l, 2);
-      if ((lane & 3) == 0 && row < n_rows) out[row] = make_float2(m, l);
+  const int32_t kb64 = 2 * blockIdx.x + wc;  // this warp's 64-key block
+  float2* out = partial + ((int64_t)(r * n_kv_heads + g) * n_kb + kb64) * rows_max;
+  const bool block_live = j0 + 64 * wc < len;  // the second half of the last CTA may lie past the request
+  auto q_row = [&](int32_t row) -> int64_t {
+    return row < n_rows ? ((int64_t)(base + len - w + row % w) * n_q_heads + g * G + row / w) * d : -1;
+  };
+  __nv_bfloat16* qbuf[2] = {qs, qs + kMmaRows * (d + 8)};
+  stage_rows_bf16_async(qbuf[0], q, kMmaRows, d, [&](int rr) { return q_row(rr); });
+  for (int32_t row0 = 0, it = 0; row0 < n_rows; row0 += kMmaRows, ++it) {
+    __syncthreads();  // everyone is done with the buffer the next copy overwrites (and, first time, K is staged)
+    if (row0 + kMmaRows < n_rows) {
+      stage_rows_bf16_async(qbuf[(it + 1) & 1], q, kMmaRows, d, [&](int rr) { return q_row(row0 + kMmaRows + rr); });
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
     }
+    __syncthreads();
+    const __nv_bfloat16* qcur = qbuf[it & 1];
+    float acc[2][8][4];
+    logits_32x64(qcur, ks, d, acc);
+#pragma unroll
+    for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {  // the thread's four rows
+        const int32_t row = row0 + 32 * wr + 16 * mb + (lane >> 2) + 8 * h;
+        const int32_t i = row < n_rows ? len - w + row % w : -1;  // causal limit of the row (-1: no row)
+        float m = -INFINITY;
+#pragma unroll
+        for (int nb = 0; nb < 8; ++nb)
+#pragma unroll
+          for (int x = 0; x < 2; ++x) {
+            const int32_t j = j0 + 64 * wc + 8 * nb + 2 * (lane & 3) + x;
+            const float sv = j <= i ? acc[mb][nb][2 * h + x] * scale_log2 : -INFINITY;
+            acc[mb][nb][2 * h + x] = sv;
+            m = fmaxf(m, sv);
+          }
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 2));
+        float l = 0.f;
+        if (m > -INFINITY) {
+#pragma unroll
+          for (int nb = 0; nb < 8; ++nb) l += exp2f(acc[mb][nb][2 * h] - m) + exp2f(acc[mb][nb][2 * h + 1] - m);
+        }
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        if ((lane & 3) == 0 && row < n_rows && block_live) out[row] = make_float2(m, l);
+      }
   }
 }
 
@@ -368,57 +409,67 @@ __global__ void __launch_bounds__(256) score_lse_merge_kernel(const float2* __re
   lse2[((int64_t)r * n_q_heads + hq) * window + iw] = m + log2f(l);
 }
 
-// Pass 2 (Eq. 2).  C[g, j] = (1/G) * sum over the stacked rows of exp2(s - lse) for the non-recent keys of block kb.
+// Pass 2 (Eq. 2).  C[g, j] = (1/G) * sum over the stacked rows of exp2(s - lse) for the non-recent keys of the CTA's block.
 __global__ void __launch_bounds__(kMmaThreads) score_mma_colsum_kernel(
     const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k, const int32_t* __restrict__ cu_seqlens,
     int32_t window, int32_t n_q_heads, int32_t n_kv_heads, int32_t d, float scale_log2, const float* __restrict__ lse2,
     int64_t n_tokens, float* __restrict__ c_out) {
   extern __shared__ __align__(16) uint8_t smem_mma[];
-  __shared__ float red[kMmaThreads / 32][kMmaKeys];
+  __shared__ float red[4][kCtaKeys];  // per row group of warps
   __nv_bfloat16* ks = reinterpret_cast<__nv_bfloat16*>(smem_mma);
-  __nv_bfloat16* qs = ks + kMmaKeys * (d + 8);
-  const int32_t r = blockIdx.z, g = blockIdx.y, j0 = blockIdx.x * kMmaKeys;
+  __nv_bfloat16* qs = ks + kCtaKeys * (d + 8);
+  const int32_t r = blockIdx.z, g = blockIdx.y, j0 = blockIdx.x * kCtaKeys;
   const int32_t G = n_q_heads / n_kv_heads;
   const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
   const int32_t w = min(window, len), nr = len - w, n_rows = G * w;
   if (j0 >= len) return;
   float* cg = c_out + (int64_t)g * n_tokens + base;
   if (j0 >= nr) {  // block inside the window: defined as 0
-    for (int c = threadIdx.x; c < kMmaKeys; c += kMmaThreads)
+    for (int c = threadIdx.x; c < kCtaKeys; c += kMmaThreads)
       if (j0 + c < len) cg[j0 + c] = 0.f;
     return;
   }
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  stage_rows_bf16(ks, k, kMmaKeys, d, [&](int rr) -> int64_t {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wr = warp >> 1, wc = warp & 1;
+  stage_rows_bf16(ks, k, kCtaKeys, d, [&](int rr) -> int64_t {
     return j0 + rr < len ? ((int64_t)(base + j0 + rr) * n_kv_heads + g) * d : -1;
   });
   float col[8][2];
 #pragma unroll
   for (int nb = 0; nb < 8; ++nb) col[nb][0] = col[nb][1] = 0.f;
-  for (int32_t row0 = 0; row0 < n_rows; row0 += kMmaRows) {
+  auto q_row = [&](int32_t row) -> int64_t {
+    return row < n_rows ? ((int64_t)(base + len - w + row % w) * n_q_heads + g * G + row / w) * d : -1;
+  };
+  __nv_bfloat16* qbuf[2] = {qs, qs + kMmaRows * (d + 8)};
+  stage_rows_bf16_async(qbuf[0], q, kMmaRows, d, [&](int rr) { return q_row(rr); });
+  for (int32_t row0 = 0, it = 0; row0 < n_rows; row0 += kMmaRows, ++it) {
+    __syncthreads();  // everyone is done with the buffer the next copy overwrites (and, first time, K is staged)
+    if (row0 + kMmaRows < n_rows) {
+      stage_rows_bf16_async(qbuf[(it + 1) & 1], q, kMmaRows, d, [&](int rr) { return q_row(row0 + kMmaRows + rr); });
+      cp_async_wait<1>();
+    } else {
+      cp_async_wait<0>();
+    }
     __syncthreads();
-    stage_rows_bf16(qs, q, kMmaRows, d, [&](int rr) -> int64_t {
-      const int32_t row = row0 + rr;
-      return row < n_rows ? ((int64_t)(base + len - w + row % w) * n_q_heads + g * G + row / w) * d : -1;
-    });
-    __syncthreads();
-    float acc[8][4];
-    logits_16x64(qs, ks, d, acc);
+    const __nv_bfloat16* qcur = qbuf[it & 1];
+    float acc[2][8][4];
+    logits_32x64(qcur, ks, d, acc);
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int32_t row = row0 + 16 * warp + (lane >> 2) + 8 * h;
-      if (row < n_rows) {
-        // every non-recent key precedes every window row, so causality holds for all of them
-        const float lse = __ldg(lse2 + ((int64_t)r * n_q_heads + g * G + row / w) * window + row % w);
+    for (int mb = 0; mb < 2; ++mb)
 #pragma unroll
-        for (int nb = 0; nb < 8; ++nb) {
-          col[nb][0] += exp2f(fmaf(acc[nb][2 * h], scale_log2, -lse));
-          col[nb][1] += exp2f(fmaf(acc[nb][2 * h + 1], scale_log2, -lse));
+      for (int h = 0; h < 2; ++h) {
+        const int32_t row = row0 + 32 * wr + 16 * mb + (lane >> 2) + 8 * h;
+        if (row < n_rows) {
+          // every non-recent key precedes every window row, so causality holds for all of them
+          const float lse = __ldg(lse2 + ((int64_t)r * n_q_heads + g * G + row / w) * window + row % w);
+#pragma unroll
+          for (int nb = 0; nb < 8; ++nb) {
+            col[nb][0] += exp2f(fmaf(acc[mb][nb][2 * h], scale_log2, -lse));
+            col[nb][1] += exp2f(fmaf(acc[mb][nb][2 * h + 1], scale_log2, -lse));
+          }
         }
       }
-    }
   }
-  // sum over the 8 row groups of the warp (lanes with equal lane % 4 hold the same columns), then over the warps
+  // sum over the 8 row groups of the warp (lanes with equal lane % 4 hold the same columns), then over the 4 row warps
 #pragma unroll
   for (int nb = 0; nb < 8; ++nb)
 #pragma unroll
@@ -427,13 +478,11 @@ __global__ void __launch_bounds__(kMmaThreads) score_mma_colsum_kernel(
       v += __shfl_xor_sync(0xffffffffu, v, 4);
       v += __shfl_xor_sync(0xffffffffu, v, 8);
       v += __shfl_xor_sync(0xffffffffu, v, 16);
-      if (lane < 4) red[warp][8 * nb + 2 * lane + x] = v;
+      if (lane < 4) red[wr][64 * wc + 8 * nb + 2 * lane + x] = v;
     }
   __syncthreads();
-  if (threadIdx.x < kMmaKeys) {
-    float sum = 0.f;
-#pragma unroll
-    for (int t = 0; t < kMmaThreads / 32; ++t) sum += red[t][threadIdx.x];
+  if (threadIdx.x < kCtaKeys) {
+    const float sum = (red[0][threadIdx.x] + red[1][threadIdx.x]) + (red[2][threadIdx.x] + red[3][threadIdx.x]);
     const int32_t j = j0 + threadIdx.x;
     if (j < len) cg[j] = j < nr ? sum / (float)G : 0.f;
   }
@@ -446,11 +495,11 @@ static purekv_status launch_score_mma(const void* q, const void* k, float* c_out
   float* lse2 = ws_f;                                                             // [n_req][H][window]
   // the pairs start on a 256-byte boundary behind the log-sum-exp values
   float2* partial = reinterpret_cast<float2*>(ws_f + (((int64_t)b->n_req * H * window + 63) & ~(int64_t)63));  // [n_req][Hkv][n_kb][rows_max]
-  const size_t smem = (size_t)(kMmaKeys + kMmaRows) * (d + 8) * sizeof(__nv_bfloat16);
+  const size_t smem = (size_t)(kCtaKeys + 2 * kMmaRows) * (d + 8) * sizeof(__nv_bfloat16);  // K block + two Q blocks
   PK_CUDA(cudaFuncSetAttribute(score_mma_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   PK_CUDA(cudaFuncSetAttribute(score_mma_colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   const float scale_log2 = scale * 1.4426950408889634f;
-  dim3 grid((unsigned)n_kb, (unsigned)Hkv, (unsigned)b->n_req);
+  dim3 grid((unsigned)((ml + kCtaKeys - 1) / kCtaKeys), (unsigned)Hkv, (unsigned)b->n_req);
   score_mma_partial_kernel<<<grid, kMmaThreads, smem, sm>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, b->cu_seqlens,
                                                             window, H, Hkv, d, scale_log2, n_kb, rows_max, partial);
   PK_CUDA(cudaGetLastError());
