@@ -431,7 +431,12 @@ def main():
     lo, hi = pipe.compacted[0], pipe.compacted[-1] + 1
     nc = hi - lo
     sl = pipe.scored[-1]
-    t_score = time_call(lambda: P.purekv_lowlayer_score(q[sl], k[sl], pipe.batch, wl.window, c_out=pipe.c[0], ws=pipe.score_ws))
+    if pipe.one_pass_scores:          # as the pipeline runs it: from the log-sum-exp the scored layer's prefill left
+        t_score = time_call(lambda: P.purekv_lowlayer_score_lse(q[sl], k[sl], pipe.lse[len(pipe.scored) - 1], pipe.batch,
+                                                                wl.window, c_out=pipe.c[0], status=pipe.status))
+    else:
+        t_score = time_call(lambda: P.purekv_lowlayer_score(q[sl], k[sl], pipe.batch, wl.window, c_out=pipe.c[0],
+                                                            ws=pipe.score_ws))
     t_select = time_call(lambda: P.purekv_select_topk(pipe.c[len(pipe.scored) - 1], v[lo:hi], pipe.batch, pipe.budget,
                                                       idx_out=pipe.idx, ws=pipe.select_ws))
     t_compact = time_call(lambda: P.purekv_compact_kv(k[lo:hi], v[lo:hi], pipe.idx, pipe.batch, pipe.budget,
@@ -447,7 +452,10 @@ def main():
     hbm = float(peaks["hbm_gbs"])
     steps_detail = {
         "plan_build_ms": t_plan,
-        "score": {"ms": t_score, "GBps": bytes_score / t_score / 1e6, "frac_hbm": bytes_score / t_score / 1e6 / hbm},
+        "score": {"ms": t_score, "GBps": bytes_score / t_score / 1e6, "frac_hbm": bytes_score / t_score / 1e6 / hbm,
+                  "kernel": "one pass, tcgen05, from the prefill's log-sum-exp" if pipe.one_pass_scores else "two passes",
+                  "TFLOPs": (1 if pipe.one_pass_scores else 2) * 2.0 * wl.n_q_heads * min(wl.window, tokens) * tokens *
+                  wl.head_dim / t_score / 1e9},
         "select": {"ms": t_select, "GBps": bytes_select / t_select / 1e6, "frac_hbm": bytes_select / t_select / 1e6 / hbm},
         "compact": {"ms": t_compact, "GBps": bytes_compact / t_compact / 1e6, "frac_hbm": bytes_compact / t_compact / 1e6 / hbm},
         "hbm_peak_GBps": hbm, "hbm_peak_kind": peak_kind, "timing": "cold L2 (256 MiB flush before each call), median of 5",

@@ -158,6 +158,17 @@ purekv_status purekv_lowlayer_score(const void *q, const void *k, float *c_out, 
                                     int32_t head_dim, purekv_dtype dtype, float softmax_scale,
                                     void *ws, size_t ws_bytes, void *stream);
 
+/* The same scores in one pass, for a layer whose dense causal prefill has already produced the rows' log-sum-exp
+ * (Eq. 1's row normaliser): lse is the [H, T] fp32 output of purekv_st_sparse_prefill run on the same Q, K with
+ * PUREKV_FLAG_DENSE_CAUSAL (natural log), so C = (1/G) sum over the window rows of exp(s - lse) needs no first
+ * pass and no workspace.  Runs on the tcgen05 tensor cores; supports bf16, head_dim 128 and a window that is a
+ * multiple of 8 (requests shorter than the window must then have a multiple of 8 tokens), and returns
+ * PUREKV_ERR_UNSUPPORTED otherwise -- use purekv_lowlayer_score for those.  `status` as in the prefill call. */
+purekv_status purekv_lowlayer_score_lse(const void *q, const void *k, const float *lse, float *c_out,
+                                        const purekv_batch *batch, int32_t window, int32_t n_q_heads,
+                                        int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                        float softmax_scale, int32_t *status, void *stream);
+
 /* ---- the same scores for callers that cannot hand over a workspace ---------------------------
  * (The paper has no counterpart: this is a packaging variant of purekv_lowlayer_score.)
  * Some callers cannot obtain device memory at the moment they need the scores: a serving engine that

@@ -26,7 +26,7 @@ FLAG_DENSE_CAUSAL = 1
 
 EXPORTS = ("purekv_version", "purekv_last_error", "purekv_budget", "purekv_plan_bytes", "purekv_plan_build",
            "purekv_plan_build_host",
-           "purekv_st_sparse_prefill", "purekv_score_ws_bytes", "purekv_lowlayer_score", "purekv_lowlayer_score_noalloc",
+           "purekv_st_sparse_prefill", "purekv_score_ws_bytes", "purekv_lowlayer_score", "purekv_lowlayer_score_lse", "purekv_lowlayer_score_noalloc",
            "purekv_select_ws_bytes",
            "purekv_select_topk", "purekv_compact_kv", "purekv_poll_status")
 
@@ -69,6 +69,8 @@ _lib.purekv_st_sparse_prefill.argtypes = [C.c_void_p] * 5 + [C.POINTER(CBatch), 
 _lib.purekv_score_ws_bytes.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_int32]
 _lib.purekv_lowlayer_score.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32, C.c_int32,
                                        C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.purekv_lowlayer_score_lse.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32,
+                                           C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p, C.c_void_p]
 _lib.purekv_lowlayer_score_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32,
                                                C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p]
 _lib.purekv_select_ws_bytes.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_int32]
@@ -244,6 +246,21 @@ def purekv_lowlayer_score(q: torch.Tensor, k: torch.Tensor, batch: Batch, window
     _check(_lib.purekv_lowlayer_score(q.data_ptr(), k.data_ptr(), c_out.data_ptr(), C.byref(batch.c), window, h, hkv,
                                       d, _dtype_code(q), softmax_scale, ws.data_ptr(), ws.numel(), _stream()),
            "purekv_lowlayer_score")
+    return c_out
+
+
+def purekv_lowlayer_score_lse(q: torch.Tensor, k: torch.Tensor, lse: torch.Tensor, batch: Batch, window: int,
+                              c_out: Optional[torch.Tensor] = None, softmax_scale: float = 0.0,
+                              status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """C [H_kv, T] fp32 from the rows' log-sum-exp `lse` [H, T] of the same layer's dense causal prefill."""
+    assert q.is_contiguous() and k.is_contiguous() and lse.is_contiguous() and lse.dtype == torch.float32
+    t, h, d = q.shape
+    hkv = k.shape[1]
+    if c_out is None:
+        c_out = torch.empty((hkv, t), dtype=torch.float32, device=q.device)
+    _check(_lib.purekv_lowlayer_score_lse(q.data_ptr(), k.data_ptr(), lse.data_ptr(), c_out.data_ptr(), C.byref(batch.c),
+                                          window, h, hkv, d, _dtype_code(q), softmax_scale, _ptr(status), _stream()),
+           "purekv_lowlayer_score_lse")
     return c_out
 
 

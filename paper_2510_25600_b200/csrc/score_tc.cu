@@ -1,0 +1,243 @@
+// purekv_lowlayer_score_lse: window column sums (Eq. 2) on the tcgen05 tensor cores, given the rows' log-sum-exp.
+//
+// When the scored layer's dense causal prefill has already produced the log-sum-exp of every row (Eq. 1's row
+// normaliser), the scores need one pass: C[g, j] = (1/G) sum over the G*w stacked window rows of exp(s - lse).
+// A CTA owns 128 keys of one (request, KV head) -- one key per TMEM lane -- and walks the stacked rows in blocks
+// of 128 columns: S^T = K Q_w^T with tcgen05.mma (A = the K tile, B = a block of window rows, both K-major from
+// shared memory, fp32 accumulators in TMEM, two buffers).  Roles:
+//   warp 0      producer: the K tile once, then per block of rows sixteen 8-row boxes per 64-column panel (a block
+//               of stacked rows may span several query heads; an 8-row box never does when w is a multiple of 8)
+//   warp 1      owns the TMEM columns; one lane issues the products
+//   warps 2-5   one thread per key: S^T row from TMEM, exp2 against the column's log-sum-exp, running sum
+// bf16, head_dim 128, window a multiple of 8.  Every wait is bounded; on expiry the status word is set.
+#include <algorithm>
+
+#include "tc_util.cuh"
+
+namespace purekv {
+namespace sc {
+using namespace tc;
+
+constexpr int kKeys = 128, kRows = 128;
+constexpr int kThreads = 192;
+constexpr int kStages = 2;         // Q-row blocks in flight
+constexpr uint32_t kTmemCols = 256;  // two 128-column accumulators
+constexpr uint32_t kPanel = kRows * 128;  // bytes of one 64-column panel of a 128-row tile
+constexpr uint32_t kTile = 2 * kPanel;
+
+struct __align__(8) Barriers {
+  uint64_t k_full;
+  uint64_t q_full[kStages], q_empty[kStages];
+  uint64_t d_full[2], d_empty[2];
+  uint64_t drain;
+};
+
+__global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
+    const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q8, const float* __restrict__ lse,
+    float* __restrict__ c_out, const int32_t* __restrict__ cu_seqlens, int32_t window, int32_t n_q_heads,
+    int32_t n_kv_heads, float scale_log2, int64_t n_tokens, int32_t* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ Barriers bars;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int abort_s;
+  const int32_t r = blockIdx.z, g = blockIdx.y, j0 = blockIdx.x * kKeys;
+  const int32_t G = n_q_heads / n_kv_heads;
+  const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
+  const int32_t w = min(window, len), nr = len - w, n_rows = G * w;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (j0 >= len) return;
+  float* cg = c_out + (int64_t)g * n_tokens + base;
+  if (j0 >= nr) {  // block inside the window: defined as 0 (before any barrier or TMEM work)
+    for (int c = tid; c < kKeys; c += kThreads)
+      if (j0 + c < len) cg[j0 + c] = 0.f;
+    return;
+  }
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sK = smem0;          // [2 panels][128 keys x 128 B]
+  const uint32_t sQ = sK + kTile;     // [kStages][2 panels][128 rows x 128 B]
+  const int32_t n_blocks = (n_rows + kRows - 1) / kRows;
+  volatile int* abort_flag = &abort_s;
+
+  if (tid == 0) {
+    abort_s = *reinterpret_cast<volatile int32_t*>(status) != 0;
+    mbar_init(smem_u32(&bars.k_full), 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&bars.q_full[s]), 1);
+      mbar_init(smem_u32(&bars.q_empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars.d_full[b]), 1);
+      mbar_init(smem_u32(&bars.d_empty[b]), 4);  // one arrival per epilogue warp
+    }
+    mbar_init(smem_u32(&bars.drain), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tmem_base_s), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = tmem_base_s;
+  const bool start_ok = abort_s == 0;
+
+  if (start_ok && warp == 0) {
+    // ---------------- producer ----------------
+    if (lane == 0) {
+      mbar_expect_tx(smem_u32(&bars.k_full), kTile);
+      tma_load_3d(sK, &tm_k, smem_u32(&bars.k_full), 0, g, base + j0);
+      tma_load_3d(sK + kPanel, &tm_k, smem_u32(&bars.k_full), 64, g, base + j0);
+      int32_t issued = 0;
+      for (int32_t t = 0; t < n_blocks; ++t) {
+        const int32_t s = t % kStages;
+        if (t >= kStages && !mbar_wait(smem_u32(&bars.q_empty[s]), ((t / kStages) - 1) & 1, abort_flag)) break;
+        mbar_expect_tx(smem_u32(&bars.q_full[s]), kTile);
+        for (int32_t grp = 0; grp < kRows / 8; ++grp) {
+          const int32_t row = t * kRows + 8 * grp;
+          // rows past the stacked list read from beyond the tensor: zero fill
+          int32_t tok = (int32_t)n_tokens, head = 0;
+          if (row < n_rows) {
+            tok = base + len - w + row % w;
+            head = g * G + row / w;
+          }
+          const uint32_t dst = sQ + s * kTile + grp * 1024;
+          tma_load_3d(dst, &tm_q8, smem_u32(&bars.q_full[s]), 0, head, tok);
+          tma_load_3d(dst + kPanel, &tm_q8, smem_u32(&bars.q_full[s]), 64, head, tok);
+        }
+        issued = t + 1;
+      }
+      if (*abort_flag) {  // every issued copy must have landed before shared memory is released
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(smem_u32(&bars.k_full), 0) && global_ns() - t0 < kWaitLimitNs) {}
+        for (int32_t t = max(0, issued - kStages); t < issued; ++t)
+          while (!mbar_try_wait(smem_u32(&bars.q_full[t % kStages]), (t / kStages) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else if (start_ok && warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = instr_desc(kRows, false);
+      constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
+      const uint32_t q_lo0 = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
+      bool ok = mbar_wait(smem_u32(&bars.k_full), 0, abort_flag);
+      for (int32_t t = 0; ok && t < n_blocks; ++t) {
+        const int32_t s = t % kStages, b = t & 1;
+        ok = mbar_wait(smem_u32(&bars.q_full[s]), (t / kStages) & 1, abort_flag);
+        if (ok && t >= 2) ok = mbar_wait(smem_u32(&bars.d_empty[b]), ((t >> 1) - 1) & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t q_lo = q_lo0 + s * (kTile >> 4);
+#pragma unroll
+        for (int ks = 0; ks < kD / 16; ++ks)
+          mma_ss_lh(tmem + b * kRows, k_lo0 + (ks >> 2) * (kPanel >> 4) + (ks & 3) * 2, kDescHi,
+                    q_lo + (ks >> 2) * (kPanel >> 4) + (ks & 3) * 2, kDescHi, idesc, ks > 0 ? 1u : 0u);
+        tc_commit(smem_u32(&bars.d_full[b]));
+        tc_commit(smem_u32(&bars.q_empty[s]));
+      }
+      if (!ok) {  // leaving early: let every issued MMA finish before TMEM is released
+        tc_commit(smem_u32(&bars.drain));
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(smem_u32(&bars.drain), 0) && global_ns() - t0 < kWaitLimitNs) {}
+      }
+    }
+  } else if (start_ok && warp >= 2) {
+    // ---------------- column sums: one thread per key ----------------
+    const int quad = warp & 3;  // TMEM lane quadrant this warp may access
+    const int key = quad * 32 + lane;
+    const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
+    const float kLog2e = 1.4426950408889634f;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    bool ok = true;
+    for (int32_t t = 0; ok && t < n_blocks; ++t) {
+      const int32_t b = t & 1;
+      // the block's log-sum-exp values (log2 units), lane i holding columns i, i+32, i+64, i+96; +inf for absent rows
+      float lv[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const int32_t row = t * kRows + 32 * c + lane;
+        lv[c] = INFINITY;
+        if (row < n_rows)
+          lv[c] = __ldg(lse + (int64_t)(g * G + row / w) * n_tokens + base + len - w + row % w) * kLog2e;
+      }
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.d_full[b]), (t >> 1) & 1, abort_flag) ? 1 : 0) != 0;
+      if (!ok) break;
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t rr[32];
+        tmem_ld32(t_lane + b * kRows + 32 * c, rr);
+        tc_wait_ld();
+#pragma unroll
+        for (int x = 0; x < 32; ++x) {
+          const float l = __shfl_sync(0xffffffffu, lv[c], x);
+          acc[x & 3] += ex2(fmaf(__uint_as_float(rr[x]), scale_log2, -l));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars.d_empty[b]));
+    }
+    if (ok) {
+      const int32_t j = j0 + key;
+      if (j < len) cg[j] = j < nr ? ((acc[0] + acc[1]) + (acc[2] + acc[3])) / (float)G : 0.f;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kTmemCols);
+  }
+  if (tid == 0 && abort_s && start_ok) atomicExch(status, (int32_t)PUREKV_ERR_TIMEOUT);
+}
+
+__device__ int32_t g_score_status;
+
+}  // namespace sc
+}  // namespace purekv
+
+using namespace purekv;
+
+extern "C" purekv_status purekv_lowlayer_score_lse(const void* q, const void* k, const float* lse, float* c_out,
+                                                   const purekv_batch* batch, int32_t window, int32_t n_q_heads,
+                                                   int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                                   float softmax_scale, int32_t* status, void* stream) {
+  using namespace sc;
+  purekv_status st = check_batch(batch, true);
+  if (st != PUREKV_OK) return st;
+  if (batch->total_tokens == 0 || batch->n_req == 0) return PUREKV_OK;  // empty batch: nothing to do
+  PK_REQUIRE(q && k && lse && c_out, PUREKV_ERR_INVALID_ARG, "purekv_lowlayer_score_lse: null pointer");
+  PK_REQUIRE(n_q_heads >= 1 && n_kv_heads >= 1 && n_q_heads % n_kv_heads == 0, PUREKV_ERR_INVALID_ARG,
+             "n_q_heads %d must be a positive multiple of n_kv_heads %d", n_q_heads, n_kv_heads);
+  PK_REQUIRE(window >= 1, PUREKV_ERR_INVALID_ARG, "window must be >= 1");
+  PK_REQUIRE(dtype == PUREKV_BF16 && head_dim == kD && window % 8 == 0, PUREKV_ERR_UNSUPPORTED,
+             "purekv_lowlayer_score_lse needs bf16, head_dim 128 and a window that is a multiple of 8 "
+             "(use purekv_lowlayer_score otherwise)");
+  PK_REQUIRE(n_kv_heads <= 65535 && batch->n_req <= 65535, PUREKV_ERR_UNSUPPORTED, "too many heads or requests");
+  PK_REQUIRE(((uintptr_t)q | (uintptr_t)k) % 16 == 0, PUREKV_ERR_INVALID_ARG, "Q/K must be 16-byte aligned");
+  int32_t ml = 0;
+  for (int r = 0; r < batch->n_req; ++r) {
+    const int32_t len = batch->h_cu_seqlens[r + 1] - batch->h_cu_seqlens[r];
+    ml = std::max(ml, len);
+    // a request shorter than the window clips it; the clipped window must keep the 8-row boxes inside one head
+    PK_REQUIRE(len >= window || len % 8 == 0, PUREKV_ERR_UNSUPPORTED,
+               "request %d: %d tokens, shorter than the window and not a multiple of 8", r, len);
+  }
+  const int64_t T = batch->total_tokens;
+  CUtensorMap mk, mq8;
+  if ((st = make_map(&mk, k, T, n_kv_heads, kKeys)) != PUREKV_OK) return st;
+  if ((st = make_map(&mq8, q, T, n_q_heads, 8)) != PUREKV_OK) return st;
+  if (!status) PK_CUDA(cudaGetSymbolAddress((void**)&status, g_score_status));
+  const size_t smem = 1024 + (size_t)(1 + kStages) * kTile;
+  PK_CUDA(cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+  dim3 grid((unsigned)((ml + kKeys - 1) / kKeys), (unsigned)n_kv_heads, (unsigned)batch->n_req);
+  score_tc_kernel<<<grid, kThreads, smem, (cudaStream_t)stream>>>(mk, mq8, lse, c_out, batch->cu_seqlens, window, n_q_heads,
+                                                                   n_kv_heads, scale * 1.4426950408889634f, T, status);
+  PK_CUDA(cudaGetLastError());
+  return PUREKV_OK;
+}

@@ -53,6 +53,11 @@ class PureKVPipeline:
         self._plan_slot = 0
         self.o = torch.empty((n_layers, t, n_q_heads, head_dim), dtype=dtype, device=dev)
         self.c = torch.empty((len(self.scored), n_kv_heads, t), dtype=torch.float32, device=dev)
+        # one-pass tensor-core scores where the entry point supports the shape (bf16, head_dim 128, window and any
+        # clipped window a multiple of 8); the two-pass kernels otherwise
+        self.one_pass_scores = (dtype == torch.bfloat16 and head_dim == 128 and window % 8 == 0 and
+                                all(l >= window or l % 8 == 0 for l in seq_lens))
+        self.lse = torch.empty((len(self.scored), n_q_heads, t), dtype=torch.float32, device=dev)
         self.score_ws = torch.empty(P.purekv_score_ws_bytes(self.batch, window, n_q_heads), dtype=torch.uint8, device=dev)
         nc = len(self.compacted)
         self.select_ws = torch.empty(P.purekv_select_ws_bytes(self.batch, nc, n_kv_heads), dtype=torch.uint8, device=dev)
@@ -61,7 +66,8 @@ class PureKVPipeline:
         self.v_c = torch.empty_like(self.k_c)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.plan_dense = self.plan_st = None
-        self.launches_per_step = n_layers + 2 * len(self.scored) + 2 + 1   # prefill, score (2 kernels), select (2), compact
+        # prefill per layer, score (1 kernel one-pass, 3 otherwise), select (2), compact
+        self.launches_per_step = n_layers + (1 if self.one_pass_scores else 3) * len(self.scored) + 2 + 1
 
     def build_plans(self) -> None:
         """Plans both masks on the host into pinned buffers and enqueues their copies on the current stream without
@@ -87,7 +93,10 @@ class PureKVPipeline:
 
     def prefill_layer(self, layer: int, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor) -> None:
         plan = self.plan_dense if layer <= self.clie else self.plan_st
-        P.purekv_st_sparse_prefill(q, k, v, self.batch, plan, out=self.o[layer], status=self.status, ws=self.prefill_ws)
+        # a scored layer is dense causal: its prefill also leaves the rows' log-sum-exp for the one-pass scores
+        lse = self.lse[self.scored.index(layer)] if (self.one_pass_scores and layer in self.scored) else None
+        P.purekv_st_sparse_prefill(q, k, v, self.batch, plan, out=self.o[layer], lse=lse, status=self.status,
+                                   ws=self.prefill_ws)
 
     def run_device(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, events=None) -> None:
         """q [n_layers,T,H,d], k,v [kv_layers,T,H_kv,d] on the GPU.  Results in self.o / idx / k_c / v_c.
@@ -100,7 +109,11 @@ class PureKVPipeline:
             if events is not None:
                 events[layer][1].record()
         for n, layer in enumerate(self.scored):
-            P.purekv_lowlayer_score(q[layer], k[layer], self.batch, self.window, c_out=self.c[n], ws=self.score_ws)
+            if self.one_pass_scores:
+                P.purekv_lowlayer_score_lse(q[layer], k[layer], self.lse[n], self.batch, self.window, c_out=self.c[n],
+                                            status=self.status)
+            else:
+                P.purekv_lowlayer_score(q[layer], k[layer], self.batch, self.window, c_out=self.c[n], ws=self.score_ws)
         lo, hi = self.compacted[0], self.compacted[-1] + 1
         P.purekv_select_topk(self.c[len(self.scored) - 1], v[lo:hi], self.batch, self.budget, idx_out=self.idx,
                              ws=self.select_ws)

@@ -175,6 +175,36 @@ def test_compress_many_segments(dtype, d, window, keep):
     check_compress(wl, 25, window, keep)
 
 
+@pytest.mark.parametrize("window", [8, 64, 200, 1000])
+@pytest.mark.parametrize("H,Hkv", [(8, 2), (7, 1), (2, 2)])
+def test_scores_from_prefill_lse(window, H, Hkv):
+    # the one-pass tensor-core scores, fed with the log-sum-exp of the dense causal prefill of the same layer
+    P = gc.pk()
+    wl = make_wl("bf16", H, Hkv, 128, [5, 0, 9, 0], [4, 3, 0, 0], [27, 45, 30, 16], 5, 6, 64)      # lengths 152, 135, 39, 16
+    x = inputs.make_qkv(wl, 0)
+    db = gc.device_batch(wl)
+    q, k, v = (gc.upload(x, n, "bf16") for n in "qkv")
+    dense = inputs.STMask(5, 6, tile=64, dense_causal=True)
+    plan = P.purekv_plan_build(db, P.st_params(dense), P.BF16, 128, H, Hkv)
+    lse = torch.empty((H, db.total_tokens), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P.purekv_st_sparse_prefill(q, k, v, db, plan, lse=lse, status=status)
+    if any(l < window and l % 8 for l in wl.batch.seq_lens):
+        with pytest.raises(P.PureKVError) as e:                      # a clipped window that is not a multiple of 8
+            P.purekv_lowlayer_score_lse(q, k, lse, db, window)
+        assert e.value.status == P.ERR_UNSUPPORTED
+        return
+    c = torch.full((Hkv, db.total_tokens), float("nan"), dtype=torch.float32, device="cuda")
+    P.purekv_lowlayer_score_lse(q, k, lse, db, window, c_out=c, status=status)
+    assert P.purekv_poll_status(status) == 0
+    c_two_pass = P.purekv_lowlayer_score(q, k, db, window)
+    torch.cuda.synchronize()
+    c_ref = po.lowlayer_score(x["q"], x["k"], wl.batch.cu_seqlens, window)
+    assert np.isfinite(c.cpu().numpy()).all()
+    assert gc.score_error(c.cpu().numpy(), c_ref) <= gc.SCORE_RTOL
+    assert gc.score_error(c.cpu().numpy(), c_two_pass.cpu().numpy().astype(np.float64)) <= gc.SCORE_RTOL
+
+
 def test_compress_cfg0():
     wl = inputs.workload(0)
     check_compress(wl, 1, wl.window, wl.keep_ratio)

@@ -59,6 +59,15 @@ def check_scores_selection_compaction(wl, x0, layers_x, groups=None):
     G = wl.n_q_heads // wl.n_kv_heads
     q0, k0 = gc.upload(x0, "q", "bf16"), gc.upload(x0, "k", "bf16")
     c = P.purekv_lowlayer_score(q0, k0, db, wl.window)
+    if wl.window % 8 == 0 and all(l >= wl.window or l % 8 == 0 for l in b.seq_lens):
+        # the one-pass tensor-core scores from the dense prefill's log-sum-exp must give the same selection input
+        dense = inputs.STMask(b.grid_h, b.grid_w, tile=wl.mask.tile, dense_causal=True)
+        plan = P.purekv_plan_build(db, P.st_params(dense), P.BF16, wl.head_dim, wl.n_q_heads, wl.n_kv_heads)
+        lse = torch.empty((wl.n_q_heads, db.total_tokens), dtype=torch.float32, device="cuda")
+        P.purekv_st_sparse_prefill(q0, k0, gc.upload(x0, "v", "bf16"), db, plan, lse=lse)
+        c_two_pass = c
+        c = P.purekv_lowlayer_score_lse(q0, k0, lse, db, wl.window)
+        assert gc.score_error(c.cpu().numpy(), c_two_pass.cpu().numpy().astype(np.float64)) <= gc.SCORE_RTOL
     vs = torch.stack([gc.upload(x, "v", "bf16") for x in layers_x])
     ks = torch.stack([gc.upload(x, "k", "bf16") for x in layers_x])
     s = torch.empty((len(layers_x), wl.n_kv_heads, db.total_tokens), dtype=torch.float32, device="cuda")
