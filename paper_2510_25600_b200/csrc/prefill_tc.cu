@@ -89,18 +89,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
   const uint32_t sM = sV + ST * kTileKV;     // [MR][128 rows x BK/8 B]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(plan);
-  const int2* entries = reinterpret_cast<const int2*>(plan + hdr->off_entries);
-  const uint32_t* masks = reinterpret_cast<const uint32_t*>(plan + hdr->off_masks);
-  const int32_t* cta_off = reinterpret_cast<const int32_t*>(plan + hdr->off_cta);
-  const Unit* units = reinterpret_cast<const Unit*>(plan + hdr->off_units);
-  int32_t* counters = reinterpret_cast<int32_t*>(plan + hdr->off_counters);
-  const int32_t G = n_q_heads / n_kv_heads, ppg = (G + 1) >> 1;
-  const int32_t u_begin = cta_off[blockIdx.x], u_end = cta_off[blockIdx.x + 1];
+  // Programmatic dependent launch: the next kernel in the stream may start its CTAs as ours retire and set up its
+  // barriers and TMEM meanwhile; nothing the previous kernel may have written is read before griddep_wait below.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   volatile int* abort_flag = &abort_s;
 
   if (tid == 0) {
-    abort_s = *reinterpret_cast<volatile int32_t*>(status) != 0;  // an earlier CTA or launch already failed
     mbar_init(smem_u32(&bars.q_full), 1);
     mbar_init(smem_u32(&bars.q_empty), 1);
     for (int s = 0; s < ST; ++s) {
@@ -127,10 +121,20 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     tmem_alloc(smem_u32(&tmem_base_s), kTmemCols);
     tmem_relinquish();
   }
+  asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream's earlier work is complete and visible from here on
+  if (tid == 0) abort_s = *reinterpret_cast<volatile int32_t*>(status) != 0;  // an earlier CTA or launch already failed
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
+  const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(plan);
+  const int2* entries = reinterpret_cast<const int2*>(plan + hdr->off_entries);
+  const uint32_t* masks = reinterpret_cast<const uint32_t*>(plan + hdr->off_masks);
+  const int32_t* cta_off = reinterpret_cast<const int32_t*>(plan + hdr->off_cta);
+  const Unit* units = reinterpret_cast<const Unit*>(plan + hdr->off_units);
+  int32_t* counters = reinterpret_cast<int32_t*>(plan + hdr->off_counters);
+  const int32_t G = n_q_heads / n_kv_heads, ppg = (G + 1) >> 1;
+  const int32_t u_begin = cta_off[blockIdx.x], u_end = cta_off[blockIdx.x + 1];
   const bool start_ok = abort_s == 0 && u_begin < u_end;
   // the two softmax warpgroups take registers from the warpgroup of the producer and MMA warps
 
@@ -671,9 +675,19 @@ static purekv_status launch(const PrefillArgs& a, const CUtensorMap& mq, const C
              "prefill kernel was compiled with %d registers per thread, too few for its register hand-over", launch_regs);
   PK_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid((unsigned)a.info->n_ctas);
-  prefill_tc_kernel<BK><<<grid, kThreads, smem, a.stream>>>(mq, mk, mv, mk64, mv64, (__nv_bfloat16*)a.o, a.lse,
-                                                            (uint8_t*)a.plan, (float*)a.ws, a.n_q_heads, a.n_kv_heads,
-                                                            a.scale * 1.4426950408889634f, status);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = a.stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol in the kernel
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  PK_CUDA(cudaLaunchKernelEx(&cfg, prefill_tc_kernel<BK>, mq, mk, mv, mk64, mv64, (__nv_bfloat16*)a.o, a.lse,
+                             (uint8_t*)a.plan, (float*)a.ws, a.n_q_heads, a.n_kv_heads,
+                             a.scale * 1.4426950408889634f, status));
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
 }

@@ -94,6 +94,27 @@ def test_prefill_tensor_core_extreme_logits(tile, kind):
     gc.check_prefill(wl, x, mask=inputs.STMask(6, 7, tile=tile, dense_causal=True), n_ctas=300)
 
 
+def test_prefill_refuses_to_run_on_a_raised_status_word():
+    # A bounded wait that expires raises the device status word; every later CTA and launch that is given the same
+    # word returns at once instead of working on a context that may be inconsistent, and the host sees the code.
+    P = gc.pk()
+    wl = make_wl("bf16", 4, 2, 128, [10], [6], [50], 8, 8, 128)
+    x = inputs.make_qkv(wl, 0)
+    db = gc.device_batch(wl)
+    q, k, v = (gc.upload(x, n, "bf16") for n in "qkv")
+    plan = P.purekv_plan_build(db, P.st_params(wl.mask), P.BF16, 128, 4, 2)
+    out = torch.full_like(q, 7.0)
+    status = torch.full((1,), P.ERR_TIMEOUT, dtype=torch.int32, device="cuda")     # as a timed-out CTA would leave it
+    P.purekv_st_sparse_prefill(q, k, v, db, plan, out=out, status=status)
+    with pytest.raises(P.PureKVError) as e:
+        P.purekv_poll_status(status)
+    assert e.value.status == P.ERR_TIMEOUT
+    assert (out == 7.0).all()                                                       # nothing was computed
+    status.zero_()                                                                  # the context is still usable
+    P.purekv_st_sparse_prefill(q, k, v, db, plan, out=out, status=status)
+    assert P.purekv_poll_status(status) == 0 and torch.isfinite(out.float()).all()
+
+
 def test_prefill_tensor_core_single_token_and_tiny_requests():
     wl = make_wl("bf16", 2, 1, 128, [1, 0, 3], [0, 1, 0], [0, 0, 126], 1, 1, 128)
     gc.check_prefill(wl, inputs.make_qkv(wl, 0))
