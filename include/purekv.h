@@ -108,13 +108,14 @@ size_t purekv_plan_bytes(const purekv_batch *batch, const purekv_st_params *para
                          purekv_dtype dtype, int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads,
                          int32_t n_ctas);
 /* Builds, on the host, the per-query-tile lists of key tiles the mask keeps (each tagged
- * full / causal-only / general, the latter with a bit mask), and for the tensor-core kernel a
- * static schedule: lists longer than about half a CTA's share are split into chunks, and the
- * (query tile, head pair, chunk) units are spread over n_ctas CTAs, longest first.  The result
+ * full / causal-only / general, the latter with a bit mask), and for the tensor-core kernel
+ * its work list: lists longer than about half a CTA's share are split into chunks, and the
+ * (query tile, head pair, chunk) units are put in order of decreasing estimated cost; the
+ * kernel's n_ctas persistent CTAs draw them in that order as they become free.  The result
  * is copied into `plan` (device, plan_bytes >= purekv_plan_bytes) on `stream`, and the call
  * waits for that copy.  A plan depends only on the batch shape, the mask and the head layout,
- * not on Q/K/V, and serves every layer.  It holds a few counters the kernel uses to combine
- * split lists (they return to zero when a launch ends), so one plan serves one launch at a
+ * not on Q/K/V, and serves every layer.  It holds a few counters the kernel uses to hand out
+ * units and to combine split lists (they return to zero when a launch ends), so one plan serves one launch at a
  * time: launches that share a plan must be ordered, e.g. on one stream, and a plan whose launch
  * reported PUREKV_ERR_TIMEOUT must be rebuilt. */
 purekv_status purekv_plan_build(const purekv_batch *batch, const purekv_st_params *params,

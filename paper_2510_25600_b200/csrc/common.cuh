@@ -40,9 +40,9 @@ __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162flo
 
 // ---- plan buffer layout (device memory, written by purekv_plan_build) -------------------
 // [PlanHeader][QTile x n_qtiles][order int32 x n_qtiles][entries int2 x n_entries][masks uint32 x n_mask_words]
-// [cta_off int32 x (n_ctas+1)][Unit x n_units][merge counters int32 x n_counters]
+// [Unit x n_units][merge counters int32 x n_counters][scheduling counters int32 x 2]
 // all sections 16-byte aligned.  The last three sections exist only in plans for the tensor-core kernel.
-constexpr uint32_t kPlanMagic = 0x504B5633u;  // "PKV3"
+constexpr uint32_t kPlanMagic = 0x504B5634u;  // "PKV4"
 
 enum TileClass : int32_t { kTileFull = 0, kTileDiag = 1, kTileGeneral = 2 };
 
@@ -56,7 +56,7 @@ struct PlanHeader {
   int64_t off_qtiles, off_order, off_entries, off_masks;  // byte offsets from the plan base
   int32_t words_per_row;                                  // max(1, tile_k / 32)
   int32_t n_ctas, n_units, n_counters;
-  int64_t off_cta, off_units, off_counters;
+  int64_t off_units, off_counters;
   int32_t n_q_heads, n_kv_heads;
   int64_t part_slots;  // partial-result slots of the workspace (split chunks x query heads)
 };
@@ -79,7 +79,9 @@ struct QTile {
 // (causality already applied; rows past q_rows are zero); -1 otherwise.
 
 // One unit of work of the tensor-core kernel: a query tile x a pair of query heads x a contiguous
-// chunk of the tile's kept-key list.  CTA c runs units cta_off[c] .. cta_off[c+1]-1 in order.
+// chunk of the tile's kept-key list.  The list is sorted by decreasing estimated cost; CTA c of n_ctas starts with
+// unit c and draws further units (n_ctas, n_ctas + 1, ...) from the first scheduling counter as it finishes one;
+// the second counts finished CTAs, and the last of them sets both back to zero.
 // A list split into n_chunks > 1 chunks leaves one partial result per chunk and head in the
 // workspace; the chunk that arrives last (merge counter) combines them.
 struct __align__(16) Unit {

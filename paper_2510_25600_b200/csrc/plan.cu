@@ -10,6 +10,7 @@
 #include <algorithm>
 #include <cstring>
 #include <string>
+#include <queue>
 #include <vector>
 
 #include "common.cuh"
@@ -101,71 +102,91 @@ purekv_status purekv_budget(int32_t len, int32_t window, double keep_ratio, int3
   return PUREKV_OK;
 }
 
-// Splits long kept-key lists into chunks and assigns (query tile, head pair, chunk) units to n_ctas persistent
-// CTAs, longest first onto the least loaded CTA.  Costs are in quarters of a 64-key half of a list entry, fitted to
-// measured CTA times: 4 per present half (5 when the entry carries a bit mask), 10 per unit (query load, pipeline
-// fill, epilogue) and 28 more for a chunk of a split list (fp32 partial result written out, and the merge).
+// Splits long kept-key lists into chunks and orders the (query tile, head pair, chunk) units by decreasing cost:
+// the kernel's n_ctas persistent CTAs start with the first n_ctas units and draw the rest from a counter as they
+// finish, so the order is longest-first list scheduling carried out at run time.  The costs also decide how finely
+// long lists are cut.  They are in quarters of a 64-key half of a list entry, fitted
+// to measured unit times: 4 per present half (5 when the entry carries a bit mask), 6 per unit (query load, pipeline
+// fill, epilogue) and 14 more for a chunk of a split list (fp32 partial result written out, and the merge).
 static void schedule_units(const std::vector<QTile>& qtiles, const std::vector<int2>& entries, int32_t H, int32_t Hkv,
                            int32_t n_ctas,
-                           std::vector<Unit>& units, std::vector<int32_t>& cta_off, int32_t* n_counters,
+                           std::vector<Unit>& units, int32_t* n_counters,
                            int64_t* part_slots, int32_t* max_chunks) {
   const int32_t G = H / Hkv, ppg = (G + 1) / 2, n_pairs = Hkv * ppg;
-  const int32_t overhead = 10, split_extra = 28;
+  const int32_t overhead = 6, split_extra = 14;
   auto halves = [&](int32_t first, int32_t last) {  // cost of entries [first, last)
     int32_t c = 0;
     for (int32_t i = first; i < last; ++i)
       c += ((((entries[i].x >> 2) & 3) == 3) ? 2 : 1) * ((entries[i].x & 3) == kTileGeneral ? 5 : 4);
     return c;
   };
-  int64_t total = 0;
-  for (const QTile& q : qtiles)
-    total += (int64_t)n_pairs * (halves(q.entry_begin, q.entry_begin + q.entry_count) + overhead);
-  const int64_t target = std::max<int64_t>(1, total / n_ctas);  // cost per CTA
-  // longest list (in entries of 8 cost units) a unit may carry: about 40 % of a CTA's share
-  const int32_t l_max = (int32_t)std::min<int64_t>(64, std::max<int64_t>(3, target / 20));
   struct Item { Unit u; int32_t cost; };
   std::vector<Item> items;
   int32_t counters = 0, mc = 1;
   int64_t slots = 0;
-  for (const QTile& q : qtiles) {
-    const int32_t nch = std::max(1, (q.entry_count + l_max - 1) / l_max);
-    mc = std::max(mc, nch);
-    const int32_t part_base = nch > 1 ? (int32_t)slots : -1, counter_base = nch > 1 ? counters : -1;
-    if (nch > 1) { slots += nch; counters += H; }
-    for (int32_t c = 0; c < nch; ++c) {
-      const int32_t a = (int32_t)((int64_t)q.entry_count * c / nch), e = (int32_t)((int64_t)q.entry_count * (c + 1) / nch);
-      for (int32_t pr = 0; pr < n_pairs; ++pr) {
-        Unit u;
-        u.q_start = q.q_start; u.q_rows = q.q_rows; u.req_start = q.req_start;
-        u.ent_begin = q.entry_begin + a; u.ent_count = e - a;
-        u.pair = pr; u.chunk = c; u.n_chunks = nch;
-        u.part_base = part_base; u.counter_base = counter_base;
-        u.pad[0] = u.pad[1] = 0;
-        items.push_back({u, halves(u.ent_begin, u.ent_begin + u.ent_count) + overhead + (nch > 1 ? split_extra : 0)});
+  // the units when no chunk of a list may be longer than l_max entries
+  auto make_items = [&](int32_t l_max) {
+    items.clear();
+    counters = 0; mc = 1; slots = 0;
+    for (const QTile& q : qtiles) {
+      const int32_t nch = std::max(1, (q.entry_count + l_max - 1) / l_max);
+      mc = std::max(mc, nch);
+      const int32_t part_base = nch > 1 ? (int32_t)slots : -1, counter_base = nch > 1 ? counters : -1;
+      if (nch > 1) { slots += nch; counters += H; }
+      for (int32_t c = 0; c < nch; ++c) {
+        const int32_t a = (int32_t)((int64_t)q.entry_count * c / nch), e = (int32_t)((int64_t)q.entry_count * (c + 1) / nch);
+        const int32_t cost = halves(q.entry_begin + a, q.entry_begin + e) + overhead + (nch > 1 ? split_extra : 0);
+        for (int32_t pr = 0; pr < n_pairs; ++pr) {
+          Unit u;
+          u.q_start = q.q_start; u.q_rows = q.q_rows; u.req_start = q.req_start;
+          u.ent_begin = q.entry_begin + a; u.ent_count = e - a;
+          u.pair = pr; u.chunk = c; u.n_chunks = nch;
+          u.part_base = part_base; u.counter_base = counter_base;
+          u.pad[0] = u.pad[1] = 0;
+          items.push_back({u, cost});
+        }
       }
     }
+    std::stable_sort(items.begin(), items.end(), [](const Item& x, const Item& y) { return x.cost > y.cost; });
+  };
+  // the time the last CTA ends when the CTAs draw units of these costs in decreasing order, each as it becomes free
+  std::vector<int32_t> costs;
+  auto makespan = [&](int32_t l_max) {
+    costs.clear();
+    for (const QTile& q : qtiles) {
+      const int32_t nch = std::max(1, (q.entry_count + l_max - 1) / l_max);
+      for (int32_t c = 0; c < nch; ++c) {
+        const int32_t a = (int32_t)((int64_t)q.entry_count * c / nch), e = (int32_t)((int64_t)q.entry_count * (c + 1) / nch);
+        costs.insert(costs.end(), (size_t)n_pairs,
+                     halves(q.entry_begin + a, q.entry_begin + e) + overhead + (nch > 1 ? split_extra : 0));
+      }
+    }
+    std::sort(costs.begin(), costs.end(), std::greater<int32_t>());
+    std::priority_queue<int64_t, std::vector<int64_t>, std::greater<int64_t>> load;
+    for (int32_t c = 0; c < n_ctas; ++c) load.push(0);
+    int64_t end = 0;
+    for (int32_t cost : costs) {
+      const int64_t t = load.top() + cost;
+      load.pop();
+      load.push(t);
+      end = std::max(end, t);
+    }
+    return end;
+  };
+  // Splitting shortens the units the CTAs end on but costs a partial result and a merge per chunk.  With few units
+  // per CTA the trade is decided by trying: the cap on a chunk's length that ends soonest under the cost model wins.
+  // With many units the ends even out by themselves and only the very longest lists are cut.
+  int32_t l_best = 64;
+  if ((int64_t)qtiles.size() * n_pairs < 12 * (int64_t)n_ctas) {
+    int64_t t_best = -1;
+    for (int32_t l_max : {64, 24, 12, 9, 7, 5}) {
+      const int64_t t = makespan(l_max);
+      if (t_best < 0 || t <= t_best) { t_best = t; l_best = l_max; }  // on a tie the finer cut
+    }
   }
-  std::stable_sort(items.begin(), items.end(), [](const Item& x, const Item& y) { return x.cost > y.cost; });
-  std::vector<std::vector<int32_t>> bins((size_t)n_ctas);
-  std::vector<int64_t> load((size_t)n_ctas, 0);
-  // min-heap of (load, cta)
-  std::vector<std::pair<int64_t, int32_t>> heap;
-  for (int32_t c = 0; c < n_ctas; ++c) heap.push_back({0, c});
-  auto cmp = [](const std::pair<int64_t, int32_t>& x, const std::pair<int64_t, int32_t>& y) { return x > y; };
-  std::make_heap(heap.begin(), heap.end(), cmp);
-  for (size_t i = 0; i < items.size(); ++i) {
-    std::pop_heap(heap.begin(), heap.end(), cmp);
-    auto& top = heap.back();
-    bins[top.second].push_back((int32_t)i);
-    top.first += items[i].cost;
-    std::push_heap(heap.begin(), heap.end(), cmp);
-  }
+  make_items(l_best);
   units.clear();
-  cta_off.assign(1, 0);
-  for (int32_t c = 0; c < n_ctas; ++c) {
-    for (int32_t i : bins[c]) units.push_back(items[i].u);
-    cta_off.push_back((int32_t)units.size());
-  }
+  for (const Item& it : items) units.push_back(it.u);
   *n_counters = counters;
   *part_slots = slots * H;
   *max_chunks = mc;
@@ -336,11 +357,10 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
 
   // tensor-core plans carry the persistent kernel's schedule
   std::vector<Unit> units;
-  std::vector<int32_t> cta_off;
   int32_t n_counters = 0, max_chunks = 1;
   int64_t part_slots = 0;
   if (tq == 128 && nq > 0) {
-    schedule_units(qtiles, entries, n_q_heads, n_kv_heads, n_ctas, units, cta_off, &n_counters, &part_slots, &max_chunks);
+    schedule_units(qtiles, entries, n_q_heads, n_kv_heads, n_ctas, units, &n_counters, &part_slots, &max_chunks);
   } else {
     n_ctas = 0;
   }
@@ -365,10 +385,10 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   h.n_q_heads = n_q_heads;
   h.n_kv_heads = n_kv_heads;
   h.part_slots = part_slots;
-  h.off_cta = h.off_masks + align16(h.n_mask_words * 4);
-  h.off_units = h.off_cta + align16(((int64_t)h.n_ctas + 1) * 4);
+  h.off_units = h.off_masks + align16(h.n_mask_words * 4);
   h.off_counters = h.off_units + align16((int64_t)h.n_units * sizeof(Unit));
-  const int64_t total = h.off_counters + align16((int64_t)n_counters * 4);
+  // the merge counters, then the kernel's two scheduling counters; all start at zero and the kernel leaves them so
+  const int64_t total = h.off_counters + align16(((int64_t)n_counters + 2) * 4);
 
   host.assign((size_t)total, 0);
   memcpy(host.data(), &h, sizeof(h));
@@ -377,7 +397,6 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   if (!entries.empty()) memcpy(host.data() + h.off_entries, entries.data(), entries.size() * 8);
   if (!masks.empty()) memcpy(host.data() + h.off_masks, masks.data(), masks.size() * 4);
   if (!units.empty()) {
-    memcpy(host.data() + h.off_cta, cta_off.data(), cta_off.size() * 4);
     memcpy(host.data() + h.off_units, units.data(), units.size() * sizeof(Unit));
   }
 

@@ -38,6 +38,7 @@ constexpr int kWarpProducer = 8, kWarpMma = 9;
 constexpr int kRegsSoftmax = 208, kRegsOther = 88;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint32_t kColO = 256;
+constexpr int kUnitRing = 4;  // units in flight between the producer's publication and the other roles' copies
 
 template <int BK>
 struct Cfg {
@@ -58,6 +59,8 @@ struct __align__(8) Barriers {
   uint64_t o_done[2];      // one completion per P.V product of the slot
   uint64_t o_final[2];     // one completion per unit, after the slot's last P.V product
   uint64_t rows_sync[2];   // the 128 row threads of a slot meet here around the merge-counter update
+  uint64_t u_full[kUnitRing];   // the producer published a unit (or the end mark) in unit_s[]
+  uint64_t u_empty[kUnitRing];  // the MMA thread and the eight softmax warps have copied it
   uint64_t drain;
 };
 
@@ -78,6 +81,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
   extern __shared__ uint8_t smem_raw[];
   __shared__ Barriers<BK> bars;
   __shared__ int2 meta_s[MR];
+  __shared__ Unit unit_s[kUnitRing];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
   __shared__ int merge_s[2];
@@ -113,6 +117,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       mbar_init(smem_u32(&bars.o_final[sl]), 1);
       mbar_init(smem_u32(&bars.rows_sync[sl]), 128);
     }
+    for (int s = 0; s < kUnitRing; ++s) {
+      mbar_init(smem_u32(&bars.u_full[s]), 1);
+      mbar_init(smem_u32(&bars.u_empty[s]), 9);
+    }
     mbar_init(smem_u32(&bars.drain), 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -130,12 +138,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
   const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(plan);
   const int2* entries = reinterpret_cast<const int2*>(plan + hdr->off_entries);
   const uint32_t* masks = reinterpret_cast<const uint32_t*>(plan + hdr->off_masks);
-  const int32_t* cta_off = reinterpret_cast<const int32_t*>(plan + hdr->off_cta);
   const Unit* units = reinterpret_cast<const Unit*>(plan + hdr->off_units);
   int32_t* counters = reinterpret_cast<int32_t*>(plan + hdr->off_counters);
   const int32_t G = n_q_heads / n_kv_heads, ppg = (G + 1) >> 1;
-  const int32_t u_begin = cta_off[blockIdx.x], u_end = cta_off[blockIdx.x + 1];
-  const bool start_ok = abort_s == 0 && u_begin < u_end;
+  // Units are handed out at run time: CTA c starts with unit c of the list (sorted by decreasing cost) and draws
+  // every further one from a counter behind the merge counters, so the CTAs finish within one small unit of one
+  // another whatever the units really cost.  The producer draws and publishes; the other roles follow unit_s[].
+  const int32_t n_units = hdr->n_units;
+  int32_t* sched = counters + hdr->n_counters;  // [0] units drawn beyond the first round, [1] CTAs that drew their last
+  const bool start_ok = abort_s == 0;
   // the two softmax warpgroups take registers from the warpgroup of the producer and MMA warps
 
   if (warp >= 8) {
@@ -145,14 +156,47 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     uint32_t it = 0;  // key tiles issued so far by this CTA, over all units
     int32_t issued_k = 0, issued_v = 0;
     bool ok = true;
-    Unit u = units[u_begin];
-    for (int32_t k = u_begin; ok && k < u_end; ++k) {
-      const Unit nxt = units[min(k + 1, u_end - 1)];
+    // unit idx of the list, or the end mark (ent_count 0) past its end
+    auto fetch = [&](int32_t idx) -> Unit {
+      Unit uu = {};
+      if (idx < n_units) uu = units[idx];
+      return uu;
+    };
+    // lane 0: put a fetched unit into the ring as the CTA's unit number uo
+    auto publish = [&](const Unit& uu, uint32_t uo) -> bool {
+      const uint32_t us = uo % kUnitRing;
+      if (uo >= (uint32_t)kUnitRing && !mbar_wait(smem_u32(&bars.u_empty[us]), ((uo / kUnitRing) - 1u) & 1u, abort_flag))
+        return false;
+      unit_s[us] = uu;
+      mbar_arrive(smem_u32(&bars.u_full[us]));
+      if (uu.ent_count == 0) {
+        // This CTA has drawn for the last time.  The CTA that does so last of all rewinds both counters for the
+        // plan's next launch (nobody reads them any more in this one).
+        __threadfence();
+        if (atomicAdd(sched + 1, 1) == (int32_t)gridDim.x - 1) {
+          sched[0] = 0;
+          sched[1] = 0;
+        }
+      }
+      return true;
+    };
+    if (lane == 0) ok = publish(fetch((int32_t)blockIdx.x), 0u);
+    for (uint32_t uo = 0;; ++uo) {
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      __syncwarp();
+      const Unit u = unit_s[uo % kUnitRing];
+      if (u.ent_count == 0) break;
+      // The next unit is drawn now and fetched once this unit's first tile is on its way, so that neither the
+      // counter's nor the list's latency falls between two units.
+      int32_t idx_next = 0;
+      Unit nxt = {};
+      if (lane == 0) idx_next = atomicAdd(sched, 1) + (int32_t)gridDim.x;
       const int32_t nt = u.ent_count;
       const int32_t g = u.pair / ppg, hq0 = g * G + 2 * (u.pair % ppg);
       const int32_t n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
       if (lane == 0) {
-        if (k > u_begin) ok = mbar_wait(smem_u32(&bars.q_empty), (uint32_t)(k - u_begin - 1) & 1u, abort_flag);
+        if (uo > 0) ok = mbar_wait(smem_u32(&bars.q_empty), (uo - 1u) & 1u, abort_flag);
         if (ok) {
           mbar_expect_tx(smem_u32(&bars.q_full), n_slots * kTileQ);
           for (int sl = 0; sl < n_slots; ++sl) {
@@ -211,12 +255,13 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
               }
               issued_v = (int32_t)it + 1;
             }
+            if (n == 0) nxt = fetch(idx_next);
           }
           ++it;
           ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         }
       }
-      u = nxt;
+      if (lane == 0 && ok) ok = publish(nxt, uo + 1u);
     }
     if (lane == 0 && *abort_flag) {
       // drain: every issued copy must have landed before shared memory is released
@@ -309,12 +354,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         return true;
       };
       bool ok = true;
-      Unit u = units[u_begin];
-      for (int32_t k = u_begin; ok && k < u_end; ++k) {
-        const Unit nxt = units[min(k + 1, u_end - 1)];
+      for (uint32_t uo = 0; ok; ++uo) {
+        const uint32_t us = uo % kUnitRing;
+        if (!mbar_wait(smem_u32(&bars.u_full[us]), (uo / kUnitRing) & 1u, abort_flag)) { ok = false; break; }
+        const Unit u = unit_s[us];
+        mbar_arrive(smem_u32(&bars.u_empty[us]));
+        if (u.ent_count == 0) break;
         nt = u.ent_count;
         n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
-        ok = mbar_wait(smem_u32(&bars.q_full), (uint32_t)(k - u_begin) & 1u, abort_flag);
+        ok = mbar_wait(smem_u32(&bars.q_full), uo & 1u, abort_flag);
         constexpr std::integral_constant<int, 0> s0{};
         constexpr std::integral_constant<int, 1> s1{};
         for (int32_t n = 0; ok && n < SB && n < nt; ++n) {
@@ -330,7 +378,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
           }
         }
         it_base += (uint32_t)nt;
-        u = nxt;
       }
       if (!ok) {
         // leaving early: let every issued MMA finish before TMEM is released
@@ -364,21 +411,28 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       ++row_syncs;
       return r;
     };
-    Unit u = units[u_begin];
-    for (int32_t k = u_begin; ok && k < u_end; ++k) {
-      const Unit nxt = units[min(k + 1, u_end - 1)];
+    for (uint32_t uo = 0; ok; ++uo) {
+      const uint32_t us = uo % kUnitRing;
+      if (!wait_w(smem_u32(&bars.u_full[us]), (uo / kUnitRing) & 1u)) { ok = false; break; }
+      // read in place (the fields wanted after the tile loop are not held in registers meanwhile); the ring slot is
+      // given back at the end of the unit
+      const Unit& u = unit_s[us];
+      auto release_unit = [&]() {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars.u_empty[us]));
+      };
       const int32_t nt = u.ent_count;
+      if (nt == 0) break;
       const int32_t pr = u.pair % ppg, g = u.pair / ppg;
       const int32_t n_slots = (2 * pr + 1 < G) ? 2 : 1;
       if (sl >= n_slots) {
-        // A single-head unit: this slot sits it out, but still follows the tile ring step by step.  A parity wait
-        // only tells the current phase from the one before, so a waiter must never get a whole ring ahead.
-        for (int32_t n = 0; ok && n < nt; ++n) {
-          const uint32_t it = it_base + (uint32_t)n;
-          ok = wait_w(smem_u32(&bars.m_full[it % MR]), (it / MR) & 1u);
-        }
+        // A single-head unit: this slot sits it out.  It takes no part in the tile ring meanwhile: a parity wait only
+        // tells a barrier's current phase from the one before, and a slot with nothing to deliver is held back by
+        // nobody, so it could fall (or run) a whole ring away from the producer.  The unit ring is a full handshake
+        // instead, and the next unit is published only after every tile of this one has been issued, which puts the
+        // slot's next tile within the ring's reach again.
         it_base += (uint32_t)nt;
-        u = nxt;
+        release_unit();
         continue;
       }
       const int32_t hq = g * G + 2 * pr + sl;
@@ -579,20 +633,18 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         }
         part[128 * 128 + row] = m_ref;
         part[128 * 128 + 128 + row] = l_sum;
-        __threadfence();
+        // The 128 rows meet (ordering their stores before row 0 inside the CTA), then row 0 alone publishes with one
+        // release / acquire update of the merge counter at GPU scope: release is cumulative over what the meeting
+        // ordered before it, so no thread needs a fence of its own.
         if (!sync_rows()) { ok = false; break; }
         if (row == 0) {
-          __threadfence();
           int32_t* cnt = counters + u.counter_base + hq;
-          const int32_t old = atomicAdd(cnt, 1);
-          const int last = old == u.n_chunks - 1;
-          if (last) atomicExch(cnt, 0);  // every chunk has arrived: ready for the next launch
-          __threadfence();
+          const int last = atom_add_acq_rel(cnt, 1) == u.n_chunks - 1;
+          if (last) *cnt = 0;  // every chunk has arrived: ready for the next launch (nobody touches it before then)
           merge_s[sl] = last;
         }
         if (!sync_rows()) { ok = false; break; }
         if (merge_s[sl]) {
-          __threadfence();
           const float* p0 = ws + ((int64_t)u.part_base * n_q_heads + hq) * kPartFloats;
           const int64_t cstride = (int64_t)n_q_heads * kPartFloats;
           float m_all = -INFINITY;
@@ -644,7 +696,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
             lse[(int64_t)hq * hdr->total_tokens + u.q_start + row] = (m_all + log2f(l_all)) * 0.6931471805599453f;
         }
       }
-      u = nxt;
+      release_unit();
     }
   }
   }

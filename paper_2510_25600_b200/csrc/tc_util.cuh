@@ -178,8 +178,8 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 // nothing beside the row's largest term (2^0 .. 2^-8 after lazy rescaling).
 __device__ __forceinline__ float2 exp2_poly2(float2 x) {
   const float kMagic = 12582912.f;  // 1.5 * 2^23
-  x.x = fmaxf(x.x, -126.f);
-  x.y = fmaxf(x.y, -126.f);
+  x.x = fminf(fmaxf(x.x, -126.f), 128.f);  // 2^128 lands on the bit pattern of +inf, which the caller's overflow test sees
+  x.y = fminf(fmaxf(x.y, -126.f), 128.f);
   const float2 r = __fadd2_rn(x, make_float2(kMagic, kMagic));
   const float2 f = __ffma2_rn(__fadd2_rn(r, make_float2(-kMagic, -kMagic)), make_float2(-1.f, -1.f), x);  // x - n
   float2 p = __ffma2_rn(make_float2(0.05517115443944931f, 0.05517115443944931f), f,
@@ -196,6 +196,12 @@ __device__ __forceinline__ void st_global_v8(void* p, const uint32_t (&w)[8]) {
   asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]),
                "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
                : "memory");
+}
+// Adds to a counter in global memory with release and acquire semantics at GPU scope; returns the old value.
+__device__ __forceinline__ int32_t atom_add_acq_rel(int32_t* p, int32_t v) {
+  int32_t old;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;

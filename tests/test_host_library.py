@@ -34,29 +34,30 @@ def test_budget_matches_oracle_rule():
 
 def parse_plan(buf: np.ndarray):
     raw = buf.tobytes()
-    (magic, tq, tk, nq, T, ne, nm, oq, oo, oe, om, wpr, n_ctas, n_units, n_counters, o_cta, o_units, o_counters, H, Hkv,
-     part_slots) = struct.unpack_from("<Iiiiqqqqqqqiiiiqqqiiq", raw, 0)
-    assert magic == 0x504B5633
+    (magic, tq, tk, nq, T, ne, nm, oq, oo, oe, om, wpr, n_ctas, n_units, n_counters, o_units, o_counters, H, Hkv,
+     part_slots) = struct.unpack_from("<Iiiiqqqqqqqiiiiqqiiq", raw, 0)
+    assert magic == 0x504B5634
     qt = np.frombuffer(raw, dtype=np.int32, count=nq * 8, offset=oq).reshape(nq, 8)
     order = np.frombuffer(raw, dtype=np.int32, count=nq, offset=oo)
     entries = np.frombuffer(raw, dtype=np.int32, count=2 * ne, offset=oe).reshape(ne, 2)
     masks = np.frombuffer(raw, dtype=np.uint32, count=nm, offset=om)
-    cta_off = np.frombuffer(raw, dtype=np.int32, count=n_ctas + 1 if n_units else 0, offset=o_cta)
     units = np.frombuffer(raw, dtype=np.int32, count=12 * n_units, offset=o_units).reshape(n_units, 12)
     counters = np.frombuffer(raw, dtype=np.int32, count=n_counters, offset=o_counters)
+    sched = np.frombuffer(raw, dtype=np.int32, count=2 if n_units else 0, offset=o_counters + 4 * n_counters)
     return dict(tq=tq, tk=tk, nq=nq, T=T, qt=qt, order=order, entries=entries, masks=masks, wpr=wpr, n_ctas=n_ctas,
-                cta_off=cta_off, units=units, counters=counters, H=H, Hkv=Hkv, part_slots=part_slots)
+                sched=sched, units=units, counters=counters, H=H, Hkv=Hkv, part_slots=part_slots)
 
 
 def check_schedule(p, info, H, Hkv, n_ctas):
     """The persistent kernel's schedule: every (query tile, head pair, list entry) is covered exactly once, chunks
-    of a split list are contiguous and complete, workspace slots and merge counters do not collide, and no CTA
-    carries much more than its share."""
+    of a split list are contiguous and complete, workspace slots and merge counters do not collide, the units
+    come in order of decreasing cost, and handing them out in that order to whichever CTA is free first leaves no CTA
+    with much more than its share."""
     G = H // Hkv
     n_pairs = Hkv * ((G + 1) // 2)
-    units, cta_off = p["units"], p["cta_off"]
-    assert p["n_ctas"] == n_ctas == info.n_ctas and len(units) == info.n_units == cta_off[-1] and cta_off[0] == 0
-    assert (np.diff(cta_off) >= 0).all() and (p["counters"] == 0).all()
+    units = p["units"]
+    assert p["n_ctas"] == n_ctas == info.n_ctas and len(units) == info.n_units
+    assert (p["counters"] == 0).all() and (p["sched"] == 0).all()
     by_start = {int(r[0]): r for r in p["qt"]}
     covered = {}
     chunks = {}
@@ -98,8 +99,12 @@ def check_schedule(p, info, H, Hkv, n_ctas):
     def cost(u):                                          # the scheduler's cost model
         e = ent[u[3]:u[3] + u[4], 0]
         c = np.where(((e >> 2) & 3) == 3, 2, 1) * np.where((e & 3) == 2, 5, 4)
-        return int(c.sum()) + 10 + (28 if u[7] > 1 else 0)
-    load = np.array([sum(cost(u) for u in units[a:b]) for a, b in zip(cta_off[:-1], cta_off[1:])])
+        return int(c.sum()) + 6 + (14 if u[7] > 1 else 0)
+    costs = [cost(u) for u in units]
+    assert all(a >= b for a, b in zip(costs, costs[1:]))
+    load = np.zeros(n_ctas, dtype=np.int64)               # each unit goes to the CTA that is free first
+    for c in costs:
+        load[int(load.argmin())] += c
     if len(units) >= 4 * n_ctas:
         assert load.max() <= 1.25 * load.mean() + 40
     return load
@@ -188,7 +193,11 @@ def test_plan_for_tensor_core_shapes_and_workload_counts():
         for H, Hkv, n_ctas in ((4, 2, 0), (7, 1, 5), (6, 2, 3), (2, 2, 400)):
             info = check_plan(batch, inputs.STMask(12, 12, tile=tile), pk.BF16, 128, H, Hkv, n_ctas)
             assert info.tile_q == 128 and info.tile_k == tile
-        assert info.max_chunks > 1                       # many CTAs, little work each: the long text lists are split
+    # many CTAs and one long request: its lists (text rows see every key) are cut into chunks
+    long_batch = inputs.make_batch([4], [40], [20], 12, 12)
+    for n_ctas in (0, 400):
+        info = check_plan(long_batch, inputs.STMask(12, 12, tile=64), pk.BF16, 128, 2, 2, n_ctas)
+        assert info.max_chunks > 1 and info.ws_bytes > 0
     # cfg 0: pair count of the paper's mask (closed form) and the block density quoted for 16-tiles
     wl = inputs.workload(0)
     info = check_plan(wl.batch, wl.mask, pk.FP32, 64)
