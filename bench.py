@@ -38,8 +38,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one ST-SpAttn launch of the tensor-core prefill
 # kernel, from the ncu capture summarised under profiles/.  It is reported only while the kernel and planner
 # sources are the ones the capture was taken from (sha1 of their text); otherwise the roofline's traffic is null.
-NCU_TRAFFIC = {"cfg1_videollama2": {"bytes_per_launch": 31.3e6, "source_sha1": "756bdd914587bbfafc37839d81f316e89f72889b"}}
-KERNEL_SOURCES = ("prefill_tc.cu", "plan.cu", "common.cuh", "prefill.cuh")
+NCU_TRAFFIC = {"cfg1_videollama2": {"bytes_per_launch": 30.8e6, "source_sha1": "0672d8a16609d18596ba06b6f7dfa995e9fdd055"}}
+KERNEL_SOURCES = ("prefill_tc.cu", "tc_util.cuh", "plan.cu", "common.cuh", "prefill.cuh")
 
 
 def kernel_source_sha1() -> str:
