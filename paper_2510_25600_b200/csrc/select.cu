@@ -38,11 +38,11 @@ struct Chunk<__nv_bfloat16> {
   }
 };
 
-// grid: one dimension, at most 8 CTAs per SM (a single full wave whatever the number of layers and heads); the warps
+// grid: one dimension, at most 3 CTAs per SM (a single full wave whatever the number of layers and heads); the warps
 // stride over blocks of 32 consecutive (token, head) rows of a layer, i.e. over contiguous memory.
 // block: 256 threads = 8 warps.
 template <typename T>
-__global__ void __launch_bounds__(256) vnorm_score_kernel(const uint4* __restrict__ v, int64_t layer_stride_c,
+__global__ void __launch_bounds__(256, 3) vnorm_score_kernel(const uint4* __restrict__ v, int64_t layer_stride_c,
                                                           const float* __restrict__ c, int64_t n_tokens,
                                                           int32_t n_kv_heads, int32_t n_layers, int32_t chunks_per_row,
                                                           float* __restrict__ s_out) {
@@ -60,13 +60,17 @@ __global__ void __launch_bounds__(256) vnorm_score_kernel(const uint4* __restric
       // 256-byte rows: a half-warp covers one row per step, 16 steps cover 32 rows (8 KB of contiguous memory).
       const int32_t half = lane >> 4, ch = lane & 15;
       float part[16];
+      // all 16 loads are issued before the first use (volatile asm keeps them ahead of the arithmetic): with the 8 KB
+      // of a warp in flight at once, three CTAs per SM keep enough bytes outstanding to stream V near the DRAM rate
+      uint4 buf[16];
 #pragma unroll
       for (int it = 0; it < 16; ++it) {
-        const int64_t r = r0 + it * 2 + half;
-        uint4 u = make_uint4(0, 0, 0, 0);
-        if (r < n_rows) u = __ldg(vl + r * 16 + ch);
-        part[it] = Chunk<T>::sumsq(u);
+        const int64_t r = min(r0 + it * 2 + half, n_rows - 1);  // rows past the end re-read the last one; never stored
+        const uint4* p = vl + r * 16 + ch;
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(buf[it].x), "=r"(buf[it].y), "=r"(buf[it].z), "=r"(buf[it].w) : "l"(p));
       }
+#pragma unroll
+      for (int it = 0; it < 16; ++it) part[it] = Chunk<T>::sumsq(buf[it]);
 #pragma unroll
       for (int it = 0; it < 16; ++it) {
         float p = part[it];
@@ -357,7 +361,7 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
     s_buf = (float*)(((uintptr_t)ws + 255) & ~(uintptr_t)255);
   }
   const int64_t n_items = ((T * n_kv_heads + 31) / 32) * n_layers;  // blocks of 32 (token, head) rows per layer
-  dim3 g1((unsigned)std::min<int64_t>((n_items + 7) / 8, 148 * 4));   // one wave: 4 CTAs of 256 threads per SM (measured best)
+  dim3 g1((unsigned)std::min<int64_t>((n_items + 7) / 8, 148 * 3));   // one wave: 3 CTAs of 256 threads per SM (measured best)
   if (dtype == PUREKV_BF16)
     vnorm_score_kernel<__nv_bfloat16><<<g1, 256, 0, sm>>>((const uint4*)v, v_layer_stride * esz / 16, c, T, n_kv_heads,
                                                           n_layers, cpr, s_buf);
