@@ -15,6 +15,9 @@
 //   pko_select         Sec. 3.1: keep the recent window w plus the top-h non-recent keys.
 //   pko_compact        the compacted cache implied by that selection.
 //   pko_budget         integer budget from a keep ratio.
+//   pko_decode         one decoding step over the compacted cache (the stage Table 3 times as
+//                      decode latency): the new token's softmax attention, Eq. 1 for a single
+//                      row, over the keys its request kept; every kept key is visible.
 // Readings taken where the paper is silent (token order inside a frame, prefix
 // tokens always visible, text rows dense, mean over the query heads of a GQA
 // group, tie-break by position) are listed in the repository's design notes.
@@ -238,6 +241,43 @@ void pko_compact(const uint8_t* src /* [T,H_kv,row_bytes] */, const int32_t* idx
 }
 
 // Budget: w <- min(w, l); k = max(w, floor(keep*l)) capped at l; h = k - w.
+// Decode step over the compacted cache (Sec. 3.1: later tokens attend to the compressed cache;
+// Table 3, decode column).  q [n_req, H, d]: one new query per request; kc, vc [K_tot, H_kv, d]:
+// the compact cache of one layer, request r owning rows cu_kept[r] .. cu_kept[r+1]-1; query
+// head hq reads KV head hq / G.  out [n_req, H, d] float64; lse [n_req, H] float64 (natural
+// log; may be NULL).  A request with no kept key gives out = 0 and lse = -inf.
+// scale <= 0 means 1/sqrt(d) (Eq. 1).
+void pko_decode(const float* q, const float* kc, const float* vc, int32_t n_req, const int32_t* cu_kept,
+                int32_t n_q_heads, int32_t n_kv_heads, int32_t d, double scale, double* out, double* lse) {
+  if (scale <= 0.0) scale = 1.0 / std::sqrt((double)d);
+  const int32_t G = n_q_heads / n_kv_heads;
+  for (int32_t r = 0; r < n_req; ++r) {
+    const int64_t j0 = cu_kept[r], j1 = cu_kept[r + 1];
+    for (int32_t hq = 0; hq < n_q_heads; ++hq) {
+      const int32_t g = hq / G;
+      const float* qi = q + ((int64_t)r * n_q_heads + hq) * d;
+      double* o = out + ((int64_t)r * n_q_heads + hq) * d;
+      for (int32_t c = 0; c < d; ++c) o[c] = 0.0;
+      std::vector<double> s((size_t)(j1 - j0));
+      double m = -std::numeric_limits<double>::infinity();
+      for (int64_t j = j0; j < j1; ++j) {
+        s[j - j0] = scale * dot_fd(qi, kc + (j * n_kv_heads + g) * d, d);
+        m = std::max(m, s[j - j0]);
+      }
+      double z = 0.0;
+      for (int64_t j = j0; j < j1; ++j) {
+        const double e = std::exp(s[j - j0] - m);
+        z += e;
+        const float* vj = vc + (j * n_kv_heads + g) * d;
+        for (int32_t c = 0; c < d; ++c) o[c] += e * (double)vj[c];
+      }
+      if (j1 > j0)
+        for (int32_t c = 0; c < d; ++c) o[c] /= z;
+      if (lse) lse[(int64_t)r * n_q_heads + hq] = j1 > j0 ? m + std::log(z) : -std::numeric_limits<double>::infinity();
+    }
+  }
+}
+
 void pko_budget(int32_t len, int32_t window, double keep_ratio, int32_t* h_out, int32_t* k_out) {
   const int32_t w = std::min(window, len);
   int32_t k = (int32_t)std::floor(keep_ratio * (double)len);

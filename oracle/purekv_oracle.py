@@ -138,6 +138,23 @@ def compact(src: np.ndarray, idx: np.ndarray, cu_seqlens, cu_kept) -> np.ndarray
     return out
 
 
+def decode(q, kc, vc, cu_kept, scale: float = 0.0):
+    """q [B,H,d], kc, vc [K_tot,H_kv,d] float32, cu_kept [B+1].  Returns (out [B,H,d] f64, lse [B,H] f64)."""
+    q = np.ascontiguousarray(q, dtype=np.float32)
+    kc = np.ascontiguousarray(kc, dtype=np.float32)
+    vc = np.ascontiguousarray(vc, dtype=np.float32)
+    ck = _i32(cu_kept)
+    b, h, d = q.shape
+    hkv = kc.shape[1]
+    assert len(ck) == b + 1 and kc.shape == vc.shape and kc.shape[0] >= int(ck[-1]) and kc.shape[2] == d
+    out = np.zeros((b, h, d), dtype=np.float64)
+    lse = np.zeros((b, h), dtype=np.float64)
+    lib().pko_decode(_p(q, C.c_float), _p(kc, C.c_float), _p(vc, C.c_float), C.c_int32(b), _p(ck, C.c_int32),
+                     C.c_int32(h), C.c_int32(hkv), C.c_int32(d), C.c_double(scale), _p(out, C.c_double),
+                     _p(lse, C.c_double))
+    return out, lse
+
+
 def budget(length: int, window: int, keep_ratio: float):
     h, k = C.c_int32(), C.c_int32()
     lib().pko_budget(C.c_int32(length), C.c_int32(window), C.c_double(keep_ratio), C.byref(h), C.byref(k))
