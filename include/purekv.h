@@ -222,6 +222,26 @@ purekv_status purekv_compact_kv(const void *k, const void *v, int64_t layer_stri
                                 purekv_dtype dtype, void *k_out, void *v_out, int64_t out_layer_stride,
                                 void *stream);
 
+/* ---- decode step over the compacted cache, one layer per call (Sec. 3.1; the stage Table 3
+ * times as decode latency) ---------------------------------------------------------------
+ * o[r, hq, :] = sum_j softmax_j(q[r, hq, :] . k_cache[j, hq / G, :] * scale) * v_cache[j, hq / G, :]
+ * over the kept rows j = cu_kept[r] .. cu_kept[r+1]-1 of request r: one new query per request
+ * and head, every kept key visible.  q, o: [n_req, H, d] (dtype); k_cache, v_cache:
+ * [K_tot, H_kv, d] as written by purekv_compact_kv for one layer; lse (nullable): [n_req, H]
+ * fp32, natural log.  A request with no kept row gets o = 0 and lse = -inf.  Rows must be 256
+ * bytes (bf16 with d = 128, fp32 with d = 64) and G = H / H_kv at most 8, else
+ * PUREKV_ERR_UNSUPPORTED.  All device pointers 16-byte aligned; cu_kept on the device and
+ * h_cu_kept on the host hold the same n_req + 1 offsets.  ws: purekv_decode_ws_bytes for the
+ * largest per-request count (may be NULL when that returns 0); nothing is allocated, nothing
+ * synchronises.  softmax_scale <= 0 means 1/sqrt(d). */
+size_t purekv_decode_ws_bytes(int32_t n_req, int32_t max_kept, int32_t n_q_heads, int32_t n_kv_heads,
+                              int32_t head_dim);
+purekv_status purekv_decode_attention(const void *q, const void *k_cache, const void *v_cache, void *o,
+                                      float *lse, const int32_t *cu_kept /* device [n_req+1] */,
+                                      const int32_t *h_cu_kept, int32_t n_req, int32_t n_q_heads,
+                                      int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                      float softmax_scale, void *ws, size_t ws_bytes, void *stream);
+
 /* Synchronises `stream`, copies the device status word to *h_status_out and returns
  * PUREKV_ERR_TIMEOUT if it is non-zero, PUREKV_ERR_CUDA if the stream reported an error. */
 purekv_status purekv_poll_status(const int32_t *status, int32_t *h_status_out, void *stream);

@@ -28,7 +28,8 @@ EXPORTS = ("purekv_version", "purekv_last_error", "purekv_budget", "purekv_plan_
            "purekv_plan_build_host",
            "purekv_st_sparse_prefill", "purekv_score_ws_bytes", "purekv_lowlayer_score", "purekv_lowlayer_score_lse", "purekv_lowlayer_score_noalloc",
            "purekv_select_ws_bytes",
-           "purekv_select_topk", "purekv_compact_kv", "purekv_poll_status")
+           "purekv_select_topk", "purekv_compact_kv", "purekv_decode_ws_bytes", "purekv_decode_attention",
+           "purekv_poll_status")
 
 _i32p = C.POINTER(C.c_int32)
 
@@ -73,6 +74,10 @@ _lib.purekv_lowlayer_score_lse.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C
                                            C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p, C.c_void_p]
 _lib.purekv_lowlayer_score_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32,
                                                C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p]
+_lib.purekv_decode_ws_bytes.restype = C.c_size_t
+_lib.purekv_decode_ws_bytes.argtypes = [C.c_int32] * 5
+_lib.purekv_decode_attention.argtypes = [C.c_void_p] * 7 + [C.c_int32] * 4 + [C.c_int, C.c_float, C.c_void_p, C.c_size_t,
+                                                                             C.c_void_p]
 _lib.purekv_select_ws_bytes.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_int32]
 _lib.purekv_select_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.POINTER(CBatch), C.c_int32,
                                     C.c_void_p, _i32p, C.c_void_p, _i32p, C.c_int32, C.c_int32, C.c_int, C.c_void_p,
@@ -317,6 +322,31 @@ def purekv_compact_kv(k: torch.Tensor, v: torch.Tensor, idx: torch.Tensor, batch
                                   _dtype_code(k), k_out.data_ptr(), v_out.data_ptr(), k_out.stride(0), _stream()),
            "purekv_compact_kv")
     return k_out, v_out
+
+
+def purekv_decode_ws_bytes(n_req: int, max_kept: int, n_q_heads: int, n_kv_heads: int, head_dim: int) -> int:
+    return int(_lib.purekv_decode_ws_bytes(n_req, max_kept, n_q_heads, n_kv_heads, head_dim))
+
+
+def purekv_decode_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, budget: Budget,
+                            out: Optional[torch.Tensor] = None, lse: Optional[torch.Tensor] = None,
+                            softmax_scale: float = 0.0, ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q [B,H,d]; k_cache, v_cache [K_tot,H_kv,d] (one layer of the compact cache); returns o [B,H,d]."""
+    assert q.is_contiguous() and k_cache.is_contiguous() and v_cache.is_contiguous()
+    b, h, d = q.shape
+    hkv = k_cache.shape[1]
+    if out is None:
+        out = torch.empty_like(q)
+    kept = np.diff(budget.h_cu_kept)
+    need = purekv_decode_ws_bytes(b, int(kept.max()) if len(kept) else 0, h, hkv, d)
+    if need and (ws is None or ws.numel() * ws.element_size() < need):
+        ws = torch.empty(need, dtype=torch.uint8, device=q.device)
+    _check(_lib.purekv_decode_attention(q.data_ptr(), k_cache.data_ptr(), v_cache.data_ptr(), out.data_ptr(), _ptr(lse),
+                                        budget.cu_kept.data_ptr(), budget.h_cu_kept.ctypes.data_as(_i32p), b, h, hkv, d,
+                                        _dtype_code(q), softmax_scale, _ptr(ws),
+                                        ws.numel() * ws.element_size() if ws is not None else 0, _stream()),
+           "purekv_decode_attention")
+    return out
 
 
 def purekv_poll_status(status: Optional[torch.Tensor]) -> int:

@@ -12,7 +12,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB = os.path.join(_HERE, "libpurekv.so")
-SOURCES = ["plan.cu", "compact.cu", "select.cu", "score.cu", "score_tc.cu", "prefill.cu", "prefill_simt.cu", "prefill_tc.cu"]
+SOURCES = ["plan.cu", "compact.cu", "decode.cu", "select.cu", "score.cu", "score_tc.cu", "prefill.cu", "prefill_simt.cu", "prefill_tc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 
