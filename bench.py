@@ -453,6 +453,19 @@ def main():
                                                       idx_out=pipe.idx, ws=pipe.select_ws))
     t_compact = time_call(lambda: P.purekv_compact_kv(k[lo:hi], v[lo:hi], pipe.idx, pipe.batch, pipe.budget,
                                                       k_out=pipe.k_c, v_out=pipe.v_c))
+    # what the compact cache is for: one decode step (one new query per request) over all compacted layers,
+    # one call per layer; not part of the timed step or of `value`
+    kept_max = int(np.diff(pipe.budget.h_cu_kept).max())
+    q_dec = torch.randn((b.n_req, wl.n_q_heads, wl.head_dim), device="cuda").to(q.dtype)
+    o_dec = torch.empty_like(q_dec)
+    dec_need = P.purekv_decode_ws_bytes(b.n_req, kept_max, wl.n_q_heads, wl.n_kv_heads, wl.head_dim)
+    dec_ws = torch.empty(max(16, dec_need), dtype=torch.uint8, device="cuda")
+
+    def decode_all_layers():
+        for layer in range(nc):
+            P.purekv_decode_attention(q_dec, pipe.k_c[layer], pipe.v_c[layer], pipe.budget, out=o_dec, ws=dec_ws)
+    decode_ok = wl.n_q_heads // wl.n_kv_heads <= 8 and wl.head_dim * (2 if wl.dtype == "bf16" else 4) == 256
+    t_decode = time_call(decode_all_layers) if decode_ok else None
     t_plan = time.perf_counter()
     pipe.build_plans()
     t_plan = (time.perf_counter() - t_plan) * 1e3
@@ -472,6 +485,13 @@ def main():
         "compact": {"ms": t_compact, "GBps": bytes_compact / t_compact / 1e6, "frac_hbm": bytes_compact / t_compact / 1e6 / hbm},
         "hbm_peak_GBps": hbm, "hbm_peak_kind": peak_kind, "timing": "cold L2 (256 MiB flush before each call), median of 5",
     }
+    if t_decode is not None:
+        bytes_decode = nc * (2 * kt * row + 2 * b.n_req * wl.n_q_heads * wl.head_dim * esz)
+        steps_detail["decode_step_after"] = {
+            "ms": t_decode, "launches": nc * (2 if dec_need else 1), "us_per_layer": 1e3 * t_decode / nc,
+            "GBps": bytes_decode / t_decode / 1e6, "frac_hbm": bytes_decode / t_decode / 1e6 / hbm,
+            "note": "one new query per request over the compact cache of every compacted layer, one call per layer; "
+                    "outside the timed step"}
 
     # ---- end to end: pinned host inputs, compact cache read back ---------------------------------------------
     e2e = None

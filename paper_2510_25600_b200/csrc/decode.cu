@@ -16,7 +16,7 @@
 namespace purekv {
 
 constexpr int kDecThreads = 128;
-constexpr int kUnroll = 4;         // rows a half-warp has in flight
+constexpr int kUnroll = 8;         // rows a half-warp has in flight
 constexpr int kDecChunkMax = 512;  // keys per CTA: logits of 8 heads x 512 keys take 16 KB of shared memory
 
 template <typename T>
@@ -240,6 +240,7 @@ __global__ void decode_merge_kernel(const float* __restrict__ part, int32_t n_q_
 }
 
 // keys per CTA and CTAs per (request, KV head): enough CTAs for two per SM when the batch alone does not give them
+// (more and shorter chunks were measured slower: the merge kernel walks a head's chunks one after the other)
 static void decode_split(int32_t n_req, int32_t max_kept, int32_t n_kv_heads, int32_t* chunk, int32_t* n_splits) {
   const int64_t base = std::max<int64_t>(1, (int64_t)n_req * n_kv_heads);
   const int64_t want = std::max<int64_t>(1, (2 * 148 + base - 1) / base);
