@@ -297,8 +297,15 @@ def run_sweep(args):
         kc, vc = P.purekv_compact_kv(kk, vv, idx, db, bud)
         t_cmp = timed(lambda: P.purekv_compact_kv(kk, vv, idx, db, bud, k_out=kc, v_out=vc), 5)
         by = 4 * bud.total_kept * row + wl.n_kv_heads * bud.total_kept * 4
+        # one decode step (one new query) over this layer's compact cache
+        q_dec = q[-1:].contiguous()
+        o_dec = torch.empty_like(q_dec)
+        ws_dec = torch.empty(max(16, P.purekv_decode_ws_bytes(1, bud.total_kept, wl.n_q_heads, wl.n_kv_heads, wl.head_dim)),
+                             dtype=torch.uint8, device="cuda")
+        t_dec = timed(lambda: P.purekv_decode_attention(q_dec, kc[0], vc[0], bud, out=o_dec, ws=ws_dec), 5)
         comp.append({"keep_ratio": keep, "kept": bud.total_kept, "select_ms": t_sel, "compact_ms": t_cmp,
-                     "compact_GBps": by / t_cmp / 1e6, "compact_frac_hbm": by / t_cmp / 1e6 / hbm})
+                     "compact_GBps": by / t_cmp / 1e6, "compact_frac_hbm": by / t_cmp / 1e6 / hbm,
+                     "decode_ms": t_dec, "decode_GBps": 2 * bud.total_kept * row / t_dec / 1e6})
     t_score = timed(lambda: P.purekv_lowlayer_score(q, k, db, wl.window, c_out=c), 5)
     # the same scores in one pass from the dense layer's log-sum-exp (what the pipeline runs for this shape)
     dense = inputs.STMask(b.grid_h, b.grid_w, tile=wl.mask.tile, dense_causal=True)
@@ -308,9 +315,25 @@ def run_sweep(args):
     P.purekv_st_sparse_prefill(q, k, v, db, plan_d, out=o, lse=lse, status=status, ws=ws_d)
     t_score_lse = timed(lambda: P.purekv_lowlayer_score_lse(q, k, lse, db, wl.window, c_out=c, status=status), 5)
     P.purekv_poll_status(status)
+    # the decode step where it is bandwidth bound: many requests, each with a few thousand kept rows (synthetic cache)
+    n_big, kept_big = 128, 4096
+
+    class _Kept:
+        h_cu_kept = np.arange(n_big + 1, dtype=np.int32) * kept_big
+        cu_kept = torch.from_numpy(h_cu_kept.copy()).cuda()
+    kc_big = torch.randn((n_big * kept_big, wl.n_kv_heads, wl.head_dim), device="cuda").to(torch.bfloat16)
+    vc_big = torch.randn_like(kc_big)
+    q_big = torch.randn((n_big, wl.n_q_heads, wl.head_dim), device="cuda").to(torch.bfloat16)
+    o_big = torch.empty_like(q_big)
+    ws_big = torch.empty(max(16, P.purekv_decode_ws_bytes(n_big, kept_big, wl.n_q_heads, wl.n_kv_heads, wl.head_dim)),
+                         dtype=torch.uint8, device="cuda")
+    t_big = timed(lambda: P.purekv_decode_attention(q_big, kc_big, vc_big, _Kept, out=o_big, ws=ws_big), 5)
+    by_big = 2 * kc_big.numel() * 2 + 2 * q_big.numel() * 2
+    decode_big = {"requests": n_big, "kept_per_request": kept_big, "heads": [wl.n_q_heads, wl.n_kv_heads], "ms": t_big,
+                  "GBps": by_big / t_big / 1e6, "frac_hbm": by_big / t_big / 1e6 / hbm, "bytes": by_big}
     print(json.dumps({"sweep": wl.name, "tokens": b.total_tokens, "peak_TFLOPs": peak, "peak_kind": peak_kind + " burst (kernel timed alone)",
                       "prefill": rows, "score_ms": t_score, "score_one_pass_ms": t_score_lse,
-                      "compression": comp,
+                      "compression": comp, "decode_large_batch": decode_big,
                       "timing": "cold L2 (256 MiB fill before each call), median"}), flush=True)
 
 

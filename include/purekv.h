@@ -229,8 +229,8 @@ purekv_status purekv_compact_kv(const void *k, const void *v, int64_t layer_stri
  * and head, every kept key visible.  q, o: [n_req, H, d] (dtype); k_cache, v_cache:
  * [K_tot, H_kv, d] as written by purekv_compact_kv for one layer; lse (nullable): [n_req, H]
  * fp32, natural log.  A request with no kept row gets o = 0 and lse = -inf.  Rows must be 256
- * bytes (bf16 with d = 128, fp32 with d = 64) and G = H / H_kv at most 8, else
- * PUREKV_ERR_UNSUPPORTED.  All device pointers 16-byte aligned; cu_kept on the device and
+ * bytes (bf16 with d = 128, fp32 with d = 64) and G = H / H_kv at most 16 (bf16) or 8 (fp32),
+ * else PUREKV_ERR_UNSUPPORTED.  All device pointers 16-byte aligned; cu_kept on the device and
  * h_cu_kept on the host hold the same n_req + 1 offsets.  ws: purekv_decode_ws_bytes for the
  * largest per-request count (may be NULL when that returns 0); nothing is allocated, nothing
  * synchronises.  softmax_scale <= 0 means 1/sqrt(d). */

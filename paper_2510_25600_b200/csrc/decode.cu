@@ -3,7 +3,8 @@
 // query head hq reads KV head hq / G of the request's kept rows.
 //
 // Split-KV, HBM bound: a CTA owns a chunk of one (request, KV head)'s kept keys and serves all G query heads of the
-// group from one read of K and one of V.  Rows are 256 bytes (bf16 d = 128 or fp32 d = 64): a half-warp covers a
+// group from one read of K and one of V.  bf16 runs on tensor cores (decode_tc_kernel, further down); the kernel
+// described next serves fp32.  Rows are 256 bytes (bf16 d = 128 or fp32 d = 64): a half-warp covers a
 // row with one 16-byte load per lane, so a warp instruction fetches two rows.  Pass 1 forms the G logits of every
 // key (q slices in registers; the 16 lanes' partial dot products are folded by a butterfly that halves the number of
 // values per step) into shared memory; the chunk's maxima and exp2 weights are then taken once per element; pass 2
@@ -217,6 +218,191 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(
   }
 }
 
+// ---- bf16, d = 128 on tensor cores ---------------------------------------------------------------------------
+// The CUDA-core kernel above spends about 100 instructions per key at G = 8; with mma.sync the group's heads are
+// the 16 rows of an m16n8k16 tile and the arithmetic all but disappears beside the loads.  A warp takes 16 keys per
+// trip: S = Q K^T as two n8 tiles (8 k-steps each), online softmax on the accumulator registers, which then serve
+// unchanged as the A operand of O += P V (16 n8 tiles over d).  No shared-memory staging and no transposes: a dot
+// product does not care in which order its terms are taken, so each thread feeds the k (and n) slots of the
+// fragments from contiguous bytes of a row and the same order is used for the other operand --
+//   Q K^T: thread (row lane/4, t = lane%4) holds d = 32t .. 32t+31 of its Q rows and of its key's K row;
+//          k-step ks takes elements 4ks, 4ks+1 (k slots 2t, 2t+1) and 4ks+2, 4ks+3 (k slots 2t+8, 2t+9);
+//   P V:   thread (g8 = lane/4, t) holds d = 16 g8 .. 16 g8+15 of the V rows of keys 2t, 2t+1, 8+2t, 9+2t of the trip;
+//          n tile nt covers d = 16 j + nt (j = 0 .. 7), two keys' values paired per register by a byte permute.
+__device__ __forceinline__ uint4 ldg16_stream(const uint4* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+  return r;
+}
+__device__ __forceinline__ void dec_mma(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t dec_pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+
+constexpr float kDecRescale = 8.f;  // the reference maximum of a row moves only when a logit exceeds it by this (log2)
+
+// grid (n_splits, H_kv, n_req), 128 threads; G <= 16.  Same outputs as decode_partial_kernel.
+__global__ void __launch_bounds__(kDecThreads) decode_tc_kernel(
+    const uint4* __restrict__ q, const uint4* __restrict__ kc, const uint4* __restrict__ vc,
+    const int32_t* __restrict__ cu_kept, int32_t n_q_heads, int32_t n_kv_heads, int32_t chunk, float scale_log2,
+    __nv_bfloat16* __restrict__ o, float* __restrict__ lse, float* __restrict__ part, int32_t n_splits) {
+  constexpr int D = 128;
+  // a row's 128 columns as four runs of 32 padded to 33, rows 132 apart: the 32 lanes of a store (8 rows x 4 runs)
+  // fall into 32 different banks
+  __shared__ float s_o[kDecThreads / 32][16][4 * 33];
+  __shared__ float s_ml[kDecThreads / 32][16][2];
+
+  const int32_t sp = blockIdx.x, g = blockIdx.y, r = blockIdx.z;
+  const int32_t G = n_q_heads / n_kv_heads;
+  const int32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t = lane & 3;
+  const int64_t j0 = (int64_t)cu_kept[r] + (int64_t)sp * chunk;
+  const int32_t n = (int32_t)max((int64_t)0, min((int64_t)cu_kept[r + 1], j0 + chunk) - j0);
+
+  // A fragments of Q: rows g8 and g8 + 8 (heads of the group; rows past G are zero)
+  uint32_t qa[8][4];
+  {
+    uint4 lo[4], hi[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      lo[c] = g8 < G ? __ldg(q + ((int64_t)r * n_q_heads + g * G + g8) * 16 + t * 4 + c) : make_uint4(0, 0, 0, 0);
+      hi[c] = g8 + 8 < G ? __ldg(q + ((int64_t)r * n_q_heads + g * G + g8 + 8) * 16 + t * 4 + c) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      qa[2 * c][0] = lo[c].x; qa[2 * c][1] = hi[c].x; qa[2 * c][2] = lo[c].y; qa[2 * c][3] = hi[c].y;
+      qa[2 * c + 1][0] = lo[c].z; qa[2 * c + 1][1] = hi[c].z; qa[2 * c + 1][2] = lo[c].w; qa[2 * c + 1][3] = hi[c].w;
+    }
+  }
+
+  float oacc[16][4];
+#pragma unroll
+  for (int nt = 0; nt < 16; ++nt)
+#pragma unroll
+    for (int x = 0; x < 4; ++x) oacc[nt][x] = 0.f;
+  float m_ref[2] = {-INFINITY, -INFINITY}, l_part[2] = {0.f, 0.f};  // rows g8 and g8 + 8
+
+  for (int32_t k0 = warp * 16; k0 < n; k0 += (kDecThreads / 32) * 16) {
+    // every load of the trip is requested before the first use; rows past the end repeat the last one (weight 0)
+    uint4 kr[2][4], vr[4][2];
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl) {
+      const uint4* row = kc + ((j0 + min(k0 + 8 * tl + g8, n - 1)) * n_kv_heads + g) * 16 + t * 4;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) kr[tl][c] = ldg16_stream(row + c);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {  // keys 2t, 2t+1, 8+2t, 9+2t of the trip
+      const int32_t key = k0 + (i >> 1) * 8 + 2 * t + (i & 1);
+      const uint4* row = vc + ((j0 + min(key, n - 1)) * n_kv_heads + g) * 16 + g8 * 2;
+      vr[i][0] = ldg16_stream(row);
+      vr[i][1] = ldg16_stream(row + 1);
+    }
+    // S for the two tiles of 8 keys
+    float sc[2][4];
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl) {
+#pragma unroll
+      for (int x = 0; x < 4; ++x) sc[tl][x] = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        dec_mma(sc[tl], qa[2 * c], kr[tl][c].x, kr[tl][c].y);
+        dec_mma(sc[tl], qa[2 * c + 1], kr[tl][c].z, kr[tl][c].w);
+      }
+    }
+    // log2 units; keys past the end weigh nothing.  sc[tl][0..1]: row g8, keys 2t, 2t+1 of tile tl; [2..3]: row g8 + 8
+#pragma unroll
+    for (int tl = 0; tl < 2; ++tl)
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        const int32_t key = k0 + 8 * tl + 2 * t + (x & 1);
+        sc[tl][x] = key < n ? sc[tl][x] * scale_log2 : -INFINITY;
+      }
+    uint32_t pa[4];
+#pragma unroll
+    for (int rw = 0; rw < 2; ++rw) {
+      float mx = fmaxf(fmaxf(sc[0][2 * rw], sc[0][2 * rw + 1]), fmaxf(sc[1][2 * rw], sc[1][2 * rw + 1]));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+      mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+      if (mx > m_ref[rw] + kDecRescale) {  // the same for the four threads of the row
+        const float alpha = m_ref[rw] == -INFINITY ? 0.f : dec_ex2(m_ref[rw] - mx);
+        l_part[rw] *= alpha;
+#pragma unroll
+        for (int nt = 0; nt < 16; ++nt) {
+          oacc[nt][2 * rw] *= alpha;
+          oacc[nt][2 * rw + 1] *= alpha;
+        }
+        m_ref[rw] = mx;
+      }
+      const float p00 = dec_ex2(sc[0][2 * rw] - m_ref[rw]), p01 = dec_ex2(sc[0][2 * rw + 1] - m_ref[rw]);
+      const float p10 = dec_ex2(sc[1][2 * rw] - m_ref[rw]), p11 = dec_ex2(sc[1][2 * rw + 1] - m_ref[rw]);
+      l_part[rw] += (p00 + p01) + (p10 + p11);
+      pa[rw] = dec_pack_bf16(p00, p01);      // k slots 2t, 2t+1: keys 2t, 2t+1 of tile 0
+      pa[2 + rw] = dec_pack_bf16(p10, p11);  // k slots 2t+8, 2t+9: the same keys of tile 1
+    }
+    // O += P V
+    const uint32_t* x0 = reinterpret_cast<const uint32_t*>(vr[0]);
+    const uint32_t* y0 = reinterpret_cast<const uint32_t*>(vr[1]);
+    const uint32_t* x1 = reinterpret_cast<const uint32_t*>(vr[2]);
+    const uint32_t* y1 = reinterpret_cast<const uint32_t*>(vr[3]);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      dec_mma(oacc[2 * j], pa, __byte_perm(x0[j], y0[j], 0x5410), __byte_perm(x1[j], y1[j], 0x5410));
+      dec_mma(oacc[2 * j + 1], pa, __byte_perm(x0[j], y0[j], 0x7632), __byte_perm(x1[j], y1[j], 0x7632));
+    }
+  }
+  // a row's sum over its four threads; then the warps' results side by side in shared memory
+#pragma unroll
+  for (int rw = 0; rw < 2; ++rw) {
+    l_part[rw] += __shfl_xor_sync(0xffffffffu, l_part[rw], 1);
+    l_part[rw] += __shfl_xor_sync(0xffffffffu, l_part[rw], 2);
+  }
+#pragma unroll
+  for (int nt = 0; nt < 16; ++nt)
+#pragma unroll
+    for (int x = 0; x < 4; ++x) s_o[warp][g8 + 8 * (x >> 1)][t * 33 + (x & 1) * 16 + nt] = oacc[nt][x];  // d = 32t + 16(x&1) + nt
+  if (t == 0) {
+    s_ml[warp][g8][0] = m_ref[0];
+    s_ml[warp][g8][1] = l_part[0];
+    s_ml[warp][g8 + 8][0] = m_ref[1];
+    s_ml[warp][g8 + 8][1] = l_part[1];
+  }
+  __syncthreads();
+  for (int32_t x = tid; x < G * D; x += kDecThreads) {
+    const int32_t h = x / D, c = x % D;
+    float m_all = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < kDecThreads / 32; ++w)
+      if (s_ml[w][h][1] > 0.f) m_all = fmaxf(m_all, s_ml[w][h][0]);
+    float a = 0.f, l = 0.f;
+#pragma unroll
+    for (int w = 0; w < kDecThreads / 32; ++w)
+      if (s_ml[w][h][1] > 0.f) {
+        const float wgt = dec_ex2(s_ml[w][h][0] - m_all);
+        a = fmaf(wgt, s_o[w][h][(c >> 5) * 33 + (c & 31)], a);
+        l = fmaf(wgt, s_ml[w][h][1], l);
+      }
+    const int32_t hq = g * G + h;
+    if (n_splits == 1) {
+      o[((int64_t)r * n_q_heads + hq) * D + c] = __float2bfloat16(l > 0.f ? a / l : 0.f);
+      if (c == 0 && lse) lse[(int64_t)r * n_q_heads + hq] = l > 0.f ? (m_all + log2f(l)) * 0.6931471805599453f : -INFINITY;
+    } else {
+      float* dst = part + (((int64_t)r * n_q_heads + hq) * n_splits + sp) * (D + 2);
+      dst[c] = a;
+      if (c == 0) {
+        dst[D] = m_all;
+        dst[D + 1] = l;
+      }
+    }
+  }
+}
+
 // grid (H, n_req), D threads: thread c merges column c of the splits' partial results.
 template <typename T>
 __global__ void decode_merge_kernel(const float* __restrict__ part, int32_t n_q_heads, int32_t n_splits, int32_t D,
@@ -284,7 +470,8 @@ purekv_status purekv_decode_attention(const void* q, const void* k_cache, const 
   const int32_t G = n_q_heads / n_kv_heads;
   PK_REQUIRE((dtype == PUREKV_BF16 && head_dim == 128) || (dtype == PUREKV_FP32 && head_dim == 64), PUREKV_ERR_UNSUPPORTED,
              "purekv_decode_attention: rows must be 256 bytes (bf16 with head_dim 128, or fp32 with head_dim 64)");
-  PK_REQUIRE(G <= 8, PUREKV_ERR_UNSUPPORTED, "purekv_decode_attention: at most 8 query heads per KV head");
+  PK_REQUIRE(G <= (dtype == PUREKV_BF16 ? 16 : 8), PUREKV_ERR_UNSUPPORTED,
+             "purekv_decode_attention: at most 16 (bf16) or 8 (fp32) query heads per KV head");
   if (n_req == 0) return PUREKV_OK;
   int32_t max_kept = 0;
   PK_REQUIRE(h_cu_kept[0] == 0, PUREKV_ERR_INVALID_ARG, "purekv_decode_attention: cu_kept must start at 0");
@@ -317,7 +504,9 @@ purekv_status purekv_decode_attention(const void* q, const void* k_cache, const 
     default: launch_decode<T, 8>(grid, sm, q, k_cache, v_cache, cu_kept, n_q_heads, n_kv_heads, chunk, scale_log2, o, lse, part, n_splits); break; \
   }
   if (dtype == PUREKV_BF16) {
-    PK_DECODE(__nv_bfloat16)
+    decode_tc_kernel<<<grid, kDecThreads, 0, sm>>>((const uint4*)q, (const uint4*)k_cache, (const uint4*)v_cache, cu_kept,
+                                                  n_q_heads, n_kv_heads, chunk, scale_log2, (__nv_bfloat16*)o, lse, part,
+                                                  n_splits);
   } else {
     PK_DECODE(float)
   }

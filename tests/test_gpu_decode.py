@@ -56,7 +56,7 @@ def run_and_check(kept, H, Hkv, d, dtype, seed=0):
     return err
 
 
-@pytest.mark.parametrize("H,Hkv", [(4, 4), (8, 4), (32, 8), (28, 4), (8, 1), (3, 1)])
+@pytest.mark.parametrize("H,Hkv", [(4, 4), (8, 4), (32, 8), (28, 4), (8, 1), (3, 1), (16, 1), (12, 1)])
 def test_decode_group_sizes_bf16(H, Hkv):
     run_and_check([0, 1, 5, 64, 130, 700, 2000, 3], H, Hkv, 128, "bf16", seed=H)
 
@@ -130,9 +130,9 @@ def test_decode_at_keep_one_repeats_the_dense_prefill_last_row():
 def test_decode_rejects_unsupported_shapes():
     P = gc.pk()
     kb = Kept([4])
-    q = torch.zeros((1, 16, 128), dtype=torch.bfloat16, device="cuda")
+    q = torch.zeros((1, 17, 128), dtype=torch.bfloat16, device="cuda")
     kc = torch.zeros((4, 1, 128), dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(P.PureKVError):                      # 16 query heads per KV head
+    with pytest.raises(P.PureKVError):                      # 17 query heads per KV head
         P.purekv_decode_attention(q, kc, kc, kb)
     q = torch.zeros((1, 2, 64), dtype=torch.bfloat16, device="cuda")
     kc = torch.zeros((4, 1, 64), dtype=torch.bfloat16, device="cuda")
