@@ -403,24 +403,60 @@ __global__ void __launch_bounds__(kDecThreads) decode_tc_kernel(
   }
 }
 
-// grid (H, n_req), D threads: thread c merges column c of the splits' partial results.
+// grid (H, n_req), D threads (D = 64 or 128): merges the chunks' partial results of one (request, head).  The
+// chunks' weights 2^(m_s - m) are formed once, 128 chunks at a time, in shared memory; thread c then sums column c
+// with independent loads.
 template <typename T>
 __global__ void decode_merge_kernel(const float* __restrict__ part, int32_t n_q_heads, int32_t n_splits, int32_t D,
                                     T* __restrict__ o, float* __restrict__ lse) {
-  const int32_t hq = blockIdx.x, r = blockIdx.y, c = threadIdx.x;
+  __shared__ float s_w[128];
+  __shared__ float s_red[4];
+  __shared__ float s_m;
+  const int32_t hq = blockIdx.x, r = blockIdx.y, c = threadIdx.x, lane = c & 31, warp = c >> 5;
+  const int32_t n_warps = (int32_t)blockDim.x >> 5;
   const float* src = part + ((int64_t)r * n_q_heads + hq) * n_splits * (D + 2);
-  float m_all = -INFINITY;
-  for (int32_t s = 0; s < n_splits; ++s)
-    if (src[s * (D + 2) + D + 1] > 0.f) m_all = fmaxf(m_all, src[s * (D + 2) + D]);
-  float a = 0.f, l = 0.f;
-  for (int32_t s = 0; s < n_splits; ++s) {
-    const float ls = src[s * (D + 2) + D + 1];
-    if (ls > 0.f) {
-      const float wgt = dec_ex2(src[s * (D + 2) + D] - m_all);
-      a = fmaf(wgt, src[s * (D + 2) + c], a);
-      l = fmaf(wgt, ls, l);
-    }
+  // the largest chunk maximum among chunks that hold anything
+  float m = -INFINITY;
+  for (int32_t s = c; s < n_splits; s += (int32_t)blockDim.x)
+    if (src[(int64_t)s * (D + 2) + D + 1] > 0.f) m = fmaxf(m, src[(int64_t)s * (D + 2) + D]);
+#pragma unroll
+  for (int mask = 16; mask >= 1; mask >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, mask));
+  if (lane == 0) s_red[warp] = m;
+  __syncthreads();
+  if (c == 0) {
+    float mm = s_red[0];
+    for (int32_t w = 1; w < n_warps; ++w) mm = fmaxf(mm, s_red[w]);
+    s_m = mm;
   }
+  __syncthreads();
+  const float m_all = s_m;
+  float a = 0.f, l = 0.f;
+  for (int32_t s0 = 0; s0 < n_splits; s0 += 128) {
+    const int32_t ns = min(128, n_splits - s0);
+    __syncthreads();
+    for (int32_t i = c; i < ns; i += (int32_t)blockDim.x) {
+      const float ls = src[(int64_t)(s0 + i) * (D + 2) + D + 1];
+      const float wgt = ls > 0.f ? dec_ex2(src[(int64_t)(s0 + i) * (D + 2) + D] - m_all) : 0.f;
+      s_w[i] = wgt;
+      l = fmaf(wgt, ls, l);  // this thread's share of the row sum
+    }
+    __syncthreads();
+    const float* col = src + (int64_t)s0 * (D + 2) + c;
+    int32_t i = 0;
+    for (; i + 4 <= ns; i += 4) {
+      const float v0 = col[(int64_t)i * (D + 2)], v1 = col[(int64_t)(i + 1) * (D + 2)];
+      const float v2 = col[(int64_t)(i + 2) * (D + 2)], v3 = col[(int64_t)(i + 3) * (D + 2)];
+      a = fmaf(s_w[i], v0, a); a = fmaf(s_w[i + 1], v1, a); a = fmaf(s_w[i + 2], v2, a); a = fmaf(s_w[i + 3], v3, a);
+    }
+    for (; i < ns; ++i) a = fmaf(s_w[i], col[(int64_t)i * (D + 2)], a);
+  }
+#pragma unroll
+  for (int mask = 16; mask >= 1; mask >>= 1) l += __shfl_xor_sync(0xffffffffu, l, mask);
+  __syncthreads();
+  if (lane == 0) s_red[warp] = l;
+  __syncthreads();
+  l = 0.f;
+  for (int32_t w = 0; w < n_warps; ++w) l += s_red[w];
   o[((int64_t)r * n_q_heads + hq) * D + c] = (T)(l > 0.f ? a / l : 0.f);
   if (c == 0 && lse) lse[(int64_t)r * n_q_heads + hq] = l > 0.f ? (m_all + log2f(l)) * 0.6931471805599453f : -INFINITY;
 }
