@@ -89,6 +89,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_partial_kernel(
   __shared__ float s_m[GP], s_l[GP];
 
   const int32_t sp = blockIdx.x, g = blockIdx.y, r = blockIdx.z;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // the merge kernel may be placed meanwhile
   const int32_t G = n_q_heads / n_kv_heads;
   const int32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, hw = lane >> 4, ch = lane & 15;
   const int64_t j0 = (int64_t)cu_kept[r] + (int64_t)sp * chunk;
@@ -260,6 +261,7 @@ __global__ void __launch_bounds__(kDecThreads) decode_tc_kernel(
   __shared__ float s_ml[kDecThreads / 32][16][2];
 
   const int32_t sp = blockIdx.x, g = blockIdx.y, r = blockIdx.z;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // the merge kernel may be placed meanwhile
   const int32_t G = n_q_heads / n_kv_heads;
   const int32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, g8 = lane >> 2, t = lane & 3;
   const int64_t j0 = (int64_t)cu_kept[r] + (int64_t)sp * chunk;
@@ -414,6 +416,9 @@ __global__ void decode_merge_kernel(const float* __restrict__ part, int32_t n_q_
   __shared__ float s_m;
   const int32_t hq = blockIdx.x, r = blockIdx.y, c = threadIdx.x, lane = c & 31, warp = c >> 5;
   const int32_t n_warps = (int32_t)blockDim.x >> 5;
+  // launched with programmatic stream serialization: placed while the chunk kernel still runs, its partial results
+  // are complete and visible from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const float* src = part + ((int64_t)r * n_q_heads + hq) * n_splits * (D + 2);
   // the largest chunk maximum among chunks that hold anything
   float m = -INFINITY;
@@ -549,11 +554,21 @@ purekv_status purekv_decode_attention(const void* q, const void* k_cache, const 
 #undef PK_DECODE
   PK_CUDA(cudaGetLastError());
   if (n_splits > 1) {
-    dim3 g2((unsigned)n_q_heads, (unsigned)n_req);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_q_heads, (unsigned)n_req);
+    cfg.blockDim = dim3((unsigned)head_dim);
+    cfg.stream = sm;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol in the kernels
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float* part_c = part;
     if (dtype == PUREKV_BF16)
-      decode_merge_kernel<__nv_bfloat16><<<g2, head_dim, 0, sm>>>(part, n_q_heads, n_splits, head_dim, (__nv_bfloat16*)o, lse);
+      PK_CUDA(cudaLaunchKernelEx(&cfg, decode_merge_kernel<__nv_bfloat16>, part_c, n_q_heads, n_splits, head_dim,
+                                 (__nv_bfloat16*)o, lse));
     else
-      decode_merge_kernel<float><<<g2, head_dim, 0, sm>>>(part, n_q_heads, n_splits, head_dim, (float*)o, lse);
+      PK_CUDA(cudaLaunchKernelEx(&cfg, decode_merge_kernel<float>, part_c, n_q_heads, n_splits, head_dim, (float*)o, lse));
     PK_CUDA(cudaGetLastError());
   }
   return PUREKV_OK;
