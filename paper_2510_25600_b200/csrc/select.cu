@@ -98,6 +98,7 @@ __global__ void __launch_bounds__(256, 3) vnorm_score_kernel(const uint4* __rest
       s_out[((int64_t)layer * n_kv_heads + g) * n_tokens + t] = __ldg(c + (int64_t)g * n_tokens + t) * sqrtf(mine);
     }
   }
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // see select_kernel
 }
 
 __device__ __forceinline__ uint32_t order_key(float f) {
@@ -129,6 +130,10 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   __shared__ int32_t carry_gt, carry_eq;
 
   const int32_t r = blockIdx.x, g = blockIdx.y, layer = blockIdx.z;
+  // launched with programmatic stream serialization behind vnorm_score_kernel, which releases its dependents only
+  // when its own work is done: the launch latency overlaps that kernel's tail, and its scores are complete and
+  // visible from here on (no effect in an ordinary launch)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int32_t base = cu_seqlens[r];
   const int32_t len = cu_seqlens[r + 1] - base;
   const int32_t w = min(window, len);
@@ -372,9 +377,19 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
   const bool stage_keys = key_bytes <= 200 * 1024;
   if (stage_keys)
     PK_CUDA(cudaFuncSetAttribute(select_kernel<false, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
-  select_kernel<false, float><<<g2, kSelThreads, stage_keys ? key_bytes : 0, sm>>>(
-      s_buf, T, batch->cu_seqlens, cu_kept, keep, window, k_tot, n_kv_heads, idx_out, nullptr, 0, nullptr,
-      stage_keys ? s_buf : nullptr);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = g2;
+  cfg.blockDim = dim3(kSelThreads);
+  cfg.dynamicSmemBytes = stage_keys ? key_bytes : 0;
+  cfg.stream = sm;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see griddepcontrol in the two kernels
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  PK_CUDA(cudaLaunchKernelEx(&cfg, select_kernel<false, float>, (const float*)s_buf, T, batch->cu_seqlens, cu_kept, keep,
+                             window, k_tot, n_kv_heads, idx_out, (const uint4*)nullptr, (int64_t)0, (const float*)nullptr,
+                             stage_keys ? s_buf : (float*)nullptr));
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
 }
