@@ -187,11 +187,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       __syncwarp();
       const Unit u = unit_s[uo % kUnitRing];
       if (u.ent_count == 0) break;
-      // The next unit is drawn now and fetched once this unit's first tile is on its way, so that neither the
-      // counter's nor the list's latency falls between two units.
+      // The next unit is drawn as late as the latencies allow: when this unit's last tile goes out (the other roles
+      // still have about two tiles of it to work through, which covers the counter's and the list's round trips).
+      // Drawn at the start of a unit it would be reserved for as long as that unit runs, and the CTAs with the
+      // longest units would keep work from those that finish early.
       int32_t idx_next = 0;
-      Unit nxt = {};
-      if (lane == 0) idx_next = atomicAdd(sched, 1) + (int32_t)gridDim.x;
       const int32_t nt = u.ent_count;
       const int32_t g = u.pair / ppg, hq0 = g * G + 2 * (u.pair % ppg);
       const int32_t n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
@@ -215,6 +215,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
           e.x = __shfl_sync(0xffffffffu, e_l.x, n - n0);
           e.y = __shfl_sync(0xffffffffu, e_l.y, n - n0);
           if (lane == 0) {
+            if (n == nt - 1) idx_next = atomicAdd(sched, 1) + (int32_t)gridDim.x;  // used after the loop
             const uint32_t s = it % ST, par = ((it / ST) - 1u) & 1u, ms = it % MR;
             const int32_t tok = u.req_start + (e.x >> 4) * BK;
             const uint32_t hm = (uint32_t)(e.x >> 2) & 3u;  // which 64-key halves of the tile are present
@@ -255,13 +256,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
               }
               issued_v = (int32_t)it + 1;
             }
-            if (n == 0) nxt = fetch(idx_next);
           }
           ++it;
           ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
         }
       }
-      if (lane == 0 && ok) ok = publish(nxt, uo + 1u);
+      if (lane == 0 && ok) ok = publish(fetch(idx_next), uo + 1u);
     }
     if (lane == 0 && *abort_flag) {
       // drain: every issued copy must have landed before shared memory is released
