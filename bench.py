@@ -38,7 +38,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one ST-SpAttn launch of the tensor-core prefill
 # kernel, from the ncu capture summarised under profiles/.  It is reported only while the kernel and planner
 # sources are the ones the capture was taken from (sha1 of their text); otherwise the roofline's traffic is null.
-NCU_TRAFFIC = {"cfg1_videollama2": {"bytes_per_launch": 30.8e6, "source_sha1": "0672d8a16609d18596ba06b6f7dfa995e9fdd055"}}
+NCU_TRAFFIC = {"cfg1_videollama2": {"bytes_per_launch": 31.0e6, "source_sha1": "6c7e587a4c974b32291d8bee206eaa2ce03d012b"}}
 KERNEL_SOURCES = ("prefill_tc.cu", "tc_util.cuh", "plan.cu", "common.cuh", "prefill.cuh")
 
 
