@@ -227,3 +227,17 @@ def test_argument_errors():
     assert e.value.status == pk.ERR_UNSUPPORTED
     with pytest.raises(pk.PureKVError):
         pk.purekv_budget(-1, 4, 0.5)
+
+
+def test_decode_workspace_rule():
+    """The decode step needs a workspace exactly when a (request, KV head) is cut into several chunks: never for
+    512 kept rows or fewer with a large batch, always for one long request; its size is the chunks' partial results."""
+    assert pk.purekv_decode_ws_bytes(300, 512, 8, 2, 128) == 0            # 600 CTAs already, one chunk each
+    assert pk.purekv_decode_ws_bytes(300, 513, 8, 2, 128) > 0             # a chunk holds at most 512 rows
+    one = pk.purekv_decode_ws_bytes(1, 20000, 28, 4, 128)
+    assert one > 0 and (one - 256) % (28 * (128 + 2) * 4) == 0            # n_splits x heads x (d + 2) floats
+    n_splits = (one - 256) // (28 * (128 + 2) * 4)
+    assert 20000 / 512 <= n_splits <= 20000 / 64 + 1                      # chunks of 64 .. 512 rows
+    assert pk.purekv_decode_ws_bytes(1, 20000, 56, 8, 128) <= 2 * one + 256   # more KV heads: fewer chunks each
+    for bad in ((0, 10, 8, 2, 128), (4, 0, 8, 2, 128), (4, 10, 0, 2, 128)):
+        assert pk.purekv_decode_ws_bytes(*bad) == 0
