@@ -153,14 +153,18 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
     const int32_t lane = tid & 31, wrp = tid >> 5, half = lane >> 4, ch = lane & 15;
     const int32_t n_score = so ? len : nr;  // the window's scores are 0 by definition and only matter for s_out
     for (int32_t t0 = wrp * 32; t0 < n_score; t0 += (kSelThreads / 32) * 32) {
+      // as in vnorm_score_kernel: the 16 row loads of the trip are issued before the first is used
       float part[16];
+      uint4 buf[16];
 #pragma unroll
       for (int it = 0; it < 16; ++it) {
-        const int32_t t = t0 + it * 2 + half;
-        uint4 u = make_uint4(0, 0, 0, 0);
-        if (t < n_score) u = __ldg(vl + ((int64_t)(base + t) * n_kv_heads + g) * 16 + ch);
-        part[it] = Chunk<T>::sumsq(u);
+        const int32_t t = min(t0 + it * 2 + half, n_score - 1);  // rows past the end re-read the last one; never stored
+        const uint4* p = vl + ((int64_t)(base + t) * n_kv_heads + g) * 16 + ch;
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                     : "=r"(buf[it].x), "=r"(buf[it].y), "=r"(buf[it].z), "=r"(buf[it].w) : "l"(p));
       }
+#pragma unroll
+      for (int it = 0; it < 16; ++it) part[it] = Chunk<T>::sumsq(buf[it]);
       float mine = 0.f;
 #pragma unroll
       for (int it = 0; it < 16; ++it) {
