@@ -18,9 +18,12 @@
 //   pko_decode         one decoding step over the compacted cache (the stage Table 3 times as
 //                      decode latency): the new token's softmax attention, Eq. 1 for a single
 //                      row, over the keys its request kept; every kept key is visible.
-// Readings taken where the paper is silent (token order inside a frame, prefix
-// tokens always visible, text rows dense, mean over the query heads of a GQA
-// group, tie-break by position) are listed in the repository's design notes.
+// Readings taken where the paper is silent: visual tokens in raster order inside a frame;
+// prefix tokens visible to every query and text rows dense causal; the spatial and the
+// temporal path form one mask (their union); softmax rows of Eq. 1 normalised over the
+// whole causal row; C of a KV head is the mean over its group's query heads; V norms
+// per KV head; the budget counts the recent window; ties in the top-h cut go to the
+// lower position and the chosen positions are listed in ascending order.
 //
 // Parity pins: every function here is pinned by the CPU tests against brute
 // force, closed forms, invariants or library special cases.  Nothing numeric is
@@ -199,11 +202,17 @@ void pko_vnorm_scores(const double* c /* [H_kv,T] */, const float* v /* [T,H_kv,
 // in ascending position order, followed by the recent window l-w .. l-1.
 // s [H_kv, T]; idx_out [H_kv, K_tot], K_tot = cu_kept[n_req]; positions request-relative.
 // kth_out (nullable) [H_kv, n_req]: the h-th largest score (NaN when h == 0).
-void pko_select(const double* s, int32_t n_req, const int32_t* cu_seqlens, int32_t window,
-                const int32_t* h_keep, const int32_t* cu_kept, int32_t n_kv_heads,
-                int32_t* idx_out, double* kth_out) {
+int32_t pko_select(const double* s, int32_t n_req, const int32_t* cu_seqlens, int32_t window,
+                   const int32_t* h_keep, const int32_t* cu_kept, int32_t n_kv_heads,
+                   int32_t* idx_out, double* kth_out) {
   const int64_t T = cu_seqlens[n_req];
   const int64_t K_tot = cu_kept[n_req];
+  // a budget that asks for more non-recent keys than a request has, or whose kept count is not h + w, is refused
+  for (int32_t r = 0; r < n_req; ++r) {
+    const int32_t len = cu_seqlens[r + 1] - cu_seqlens[r];
+    const int32_t w = std::min(window, len);
+    if (h_keep[r] < 0 || h_keep[r] > len - w || cu_kept[r + 1] - cu_kept[r] != h_keep[r] + w) return 1;
+  }
   for (int32_t g = 0; g < n_kv_heads; ++g)
     for (int32_t r = 0; r < n_req; ++r) {
       const int64_t base = cu_seqlens[r];
@@ -223,6 +232,7 @@ void pko_select(const double* s, int32_t n_req, const int32_t* cu_seqlens, int32
       for (int32_t t = 0; t < w; ++t) o[h + t] = nr + t;
       if (kth_out) kth_out[(int64_t)g * n_req + r] = h > 0 ? sg[order[h - 1]] : std::nan("");
     }
+  return 0;
 }
 
 // Compacted cache of one layer: out[cu_kept[r]+t, g, :] = src[cu_seqlens[r] + idx[g, cu_kept[r]+t], g, :].
@@ -240,7 +250,6 @@ void pko_compact(const uint8_t* src /* [T,H_kv,row_bytes] */, const int32_t* idx
       }
 }
 
-// Budget: w <- min(w, l); k = max(w, floor(keep*l)) capped at l; h = k - w.
 // Decode step over the compacted cache (Sec. 3.1: later tokens attend to the compressed cache;
 // Table 3, decode column).  q [n_req, H, d]: one new query per request; kc, vc [K_tot, H_kv, d]:
 // the compact cache of one layer, request r owning rows cu_kept[r] .. cu_kept[r+1]-1; query
@@ -278,6 +287,7 @@ void pko_decode(const float* q, const float* kc, const float* vc, int32_t n_req,
   }
 }
 
+// Budget: w <- min(w, l); k = max(w, floor(keep*l)) capped at l; h = k - w.
 void pko_budget(int32_t len, int32_t window, double keep_ratio, int32_t* h_out, int32_t* k_out) {
   const int32_t w = std::min(window, len);
   int32_t k = (int32_t)std::floor(keep_ratio * (double)len);

@@ -42,6 +42,7 @@ def lib():
     if _lib is None:
         _lib = C.CDLL(build())
         _lib.pko_mask.restype = C.c_int32
+        _lib.pko_select.restype = C.c_int32
     return _lib
 
 
@@ -120,8 +121,10 @@ def select(s: np.ndarray, cu_seqlens, window: int, h_keep, cu_kept):
     n_req = len(cu) - 1
     idx = np.zeros((hkv, int(ck[-1])), dtype=np.int32)
     kth = np.zeros((hkv, n_req), dtype=np.float64)
-    lib().pko_select(_p(s, C.c_double), C.c_int32(n_req), _p(cu, C.c_int32), C.c_int32(window),
-                     _p(hk, C.c_int32), _p(ck, C.c_int32), C.c_int32(hkv), _p(idx, C.c_int32), _p(kth, C.c_double))
+    rc = lib().pko_select(_p(s, C.c_double), C.c_int32(n_req), _p(cu, C.c_int32), C.c_int32(window),
+                          _p(hk, C.c_int32), _p(ck, C.c_int32), C.c_int32(hkv), _p(idx, C.c_int32), _p(kth, C.c_double))
+    if rc != 0:
+        raise ValueError("select: a request's h is outside [0, l - w] or its kept count is not h + w")
     return idx, kth
 
 

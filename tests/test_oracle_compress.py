@@ -172,3 +172,14 @@ def test_keep_ratio_one_reproduces_dense_attention_for_the_last_query():
     for h in range(2):
         o, _, _ = matrix_attention(x["q"][l - 1:l, h], kc[:, 0], vc[:, 0], np.ones((1, l), dtype=bool), 1 / np.sqrt(8))
         np.testing.assert_allclose(o[0], out[l - 1, h], rtol=1e-12, atol=1e-14)
+
+
+def test_select_refuses_a_budget_that_does_not_fit_the_request():
+    """h beyond the non-recent keys, or a kept count other than h + w, is an error, not an out-of-range read."""
+    cu = np.array([0, 10], dtype=np.int32)
+    s = np.arange(10, dtype=np.float64)[None]
+    for hk, ck in (([7], [0, 11]), ([3], [0, 8]), ([-1], [0, 3])):        # w = 4: at most 6 non-recent keys
+        with pytest.raises(ValueError):
+            po.select(s, cu, 4, hk, ck)
+    idx, _ = po.select(s, cu, 4, [6], [0, 10])
+    assert np.array_equal(idx[0], np.arange(10))
