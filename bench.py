@@ -3,15 +3,18 @@
 
 A step = one pass of the whole hot path over one synthetic batch: planning, ST-SpAttn prefill
 of every layer (dense causal up to the CLIE layer), low-layer window scores, V-norm top-h
-selection and K/V compaction of the compressed layers.  Default workload: the
-VideoLLaMA2-shaped one (32 layers, 32/8 heads, head_dim 128, 2432 tokens, bf16).
+selection and K/V compaction of the compressed layers.  Default workload: the largest
+whole-pipeline one, Qwen2.5-VL-7B-shaped (28 layers, 28/4 heads, head_dim 128, 8320 tokens, bf16).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--cfg 1] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--cfg 2] [--impl reference] [--no-sub]
 
 Prints ONE JSON line (rank 0).  `value` = prefill tokens/s of the whole job with inputs
 resident in HBM; `e2e` = the same with inputs in pinned host memory and the compact cache read
 back; `roofline` describes the dominant kernel (tensor-core prefill); `cpu_baseline` is the
-fp64 oracle timed on this machine's host cores on a bounded sample.
+fp64 oracle timed on this machine's host cores on a bounded sample; `configs` (one GPU only) holds
+compact records of the other workloads -- the VideoLLaMA2-shaped pipeline, the long-video layer
+under masks of growing block density with its compression at three keep ratios, and the ragged
+serving batch -- each with the clocks sampled while it was timed.
 """
 from __future__ import annotations
 
@@ -33,6 +36,7 @@ if ROOT not in sys.path:
 METRIC = "st_spattn_prefill_tokens_per_s"
 UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 8000.0   # B200 dense bf16 and HBM3e figures, for context beside the measured peaks
 
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one ST-SpAttn launch of the tensor-core prefill
@@ -170,10 +174,51 @@ def job_throughput(tokens_per_rank: int, world: int, seconds_per_step_max: float
     return world * tokens_per_rank / seconds_per_step_max
 
 
-def oracle_sample(wl, layers_x, budget_s: float = 20.0):
-    """Times the oracle on a bounded sample of the step; returns (tokens/s extrapolated to the whole step,
-    cores, description).  Prefill: all heads of a row sample of one ST layer and of the dense layer; score,
-    selection and compaction of one layer in full."""
+def pick_tensor_peak(peaks, clocks):
+    """The bf16 peak a timed region is held against: the measured burst figure when the clocks sampled during
+    the region stayed at the maximum with no power-cap sample, the sustained one otherwise."""
+    burst = float(peaks["bf16_tflops"])
+    sustained = float(peaks.get("bf16_tflops_sustained", burst))
+    sm, smax = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    capped = "sw_power_cap" in clocks.get("reasons", [])
+    at_max = sm is not None and smax is not None and sm >= 0.97 * smax
+    if at_max and not capped:
+        return burst, "burst", "median SM clock %.0f of %.0f MHz, no power-cap sample" % (sm, smax)
+    why = "power-cap samples" if capped else ("clock query unavailable" if sm is None else "median SM clock %.0f of %.0f MHz" % (sm, smax))
+    return sustained, "sustained", why
+
+
+def tensor_fracs(tflops, peaks):
+    return {"of_measured_burst": tflops / float(peaks["bf16_tflops"]),
+            "of_measured_sustained": tflops / float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
+            "of_nominal_2250": tflops / NOMINAL_TFLOPS}
+
+
+def hbm_rec(ms, nbytes, peaks):
+    gbs = nbytes / ms / 1e6
+    return {"ms": ms, "bytes": nbytes, "GBps": gbs, "frac_hbm": gbs / float(peaks["hbm_gbs"]),
+            "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS}
+
+
+def config_dict(wl):
+    """The workload description both arms print (identical for `--impl purekv` and `--impl reference`)."""
+    b = wl.batch
+    esz = 2 if wl.dtype == "bf16" else 4
+    kv_layers = max(wl.n_layers, wl.compacted_layers[-1] + 1)
+    in_bytes = b.total_tokens * wl.head_dim * esz * (wl.n_layers * wl.n_q_heads + 2 * kv_layers * wl.n_kv_heads)
+    return {"workload": wl.name, "tokens": b.total_tokens, "requests": b.n_req, "layers": wl.n_layers,
+            "heads": [wl.n_q_heads, wl.n_kv_heads], "head_dim": wl.head_dim, "tile": wl.mask.tile, "window": wl.window,
+            "keep_ratio": wl.keep_ratio, "scored_layers": list(wl.scored_layers),
+            "compacted_layers": [wl.compacted_layers[0], wl.compacted_layers[-1]],
+            "l2": "inputs larger than L2 (each layer reads its own Q/K/V; %.0f MB per step)" % (in_bytes / 1e6),
+            "multi_gpu": "replicas only (the path has no exchange step)",
+            "step": "plan build + %d prefill layers + score + select + compact" % wl.n_layers}
+
+
+def oracle_sample(wl, layers_x, n_rows: int = 256):
+    """Times the oracle on a bounded sample of the step.  Prefill: all heads of a row sample of one ST layer and
+    of the dense layer; score, selection and compaction of one layer in full.  Returns a dict with the seconds the
+    sample took, the same extrapolated to the whole step, cores and a description."""
     from oracle import purekv_oracle as po
     b = wl.batch
     cu = b.cu_seqlens
@@ -183,8 +228,9 @@ def oracle_sample(wl, layers_x, budget_s: float = 20.0):
     x0 = layers_x[0]
     x1 = next((x for x in layers_x[1:] if "q" in x), x0)
     dense = type(wl.mask)(wl.mask.grid_h, wl.mask.grid_w, tile=wl.mask.tile, dense_causal=True)
-    n_rows = min(t_tot, 256)
+    n_rows = min(t_tot, n_rows)
     rows = np.sort(rng.choice(t_tot, size=n_rows, replace=False))
+    t_all = time.perf_counter()
     t = time.perf_counter()
     po.prefill(x1["q"], x1["k"], x1["v"], cu, b.n_prefix, b.n_frames, po.mask_params(wl.mask), rows=rows)
     t_st = (time.perf_counter() - t) * t_tot / n_rows
@@ -201,17 +247,20 @@ def oracle_sample(wl, layers_x, budget_s: float = 20.0):
     po.compact(x1["k"], idx, cu, ck)
     po.compact(x1["v"], idx, cu, ck)
     t_comp = time.perf_counter() - t
+    sample_s = time.perf_counter() - t_all
     n_dense = max(wl.scored_layers) + 1
     n_st = wl.n_layers - n_dense
     total = n_dense * t_dense + n_st * t_st + len(wl.scored_layers) * t_score + len(wl.compacted_layers) * t_comp
     desc = (f"{n_rows} seeded rows x all {wl.n_q_heads} heads of one ST layer and one dense layer, full score / select / "
             f"compact of one layer; extrapolated to {n_dense} dense + {n_st} ST layers, {len(wl.scored_layers)} scored, "
             f"{len(wl.compacted_layers)} compacted")
-    return t_tot / total, cores, desc, total
+    return {"tokens_per_s": t_tot / total, "cores": cores, "sample": desc, "sample_s": sample_s, "step_s_extrapolated": total}
 
 
 def run_reference(args, wl):
-    """--impl reference: the oracle as it stands, on host cores, bounded sample per step."""
+    """--impl reference: the oracle as it stands, on host cores; each step is a bounded sample of the workload.
+    `ms_per_step` is what a step really took (the sample); `value` extrapolates the sample to the whole step and
+    says so."""
     if rank_env()[1] != 0:
         return
     from oracle import purekv_oracle as po
@@ -219,35 +268,219 @@ def run_reference(args, wl):
     po.build()
     pool = ThreadPoolExecutor(len(os.sched_getaffinity(0)))
     layers_x = [inputs.make_qkv(wl, l, pool=pool) for l in range(min(2, wl.n_layers))]
-    vals, tot = [], 0.0
+    if wl.n_layers > 2:       # an ST layer above the scored ones
+        layers_x[1] = inputs.make_qkv(wl, max(wl.scored_layers) + 1, pool=pool) if max(wl.scored_layers) + 1 < wl.n_layers else layers_x[1]
+    recs = []
     for i in range(args.warmup + args.steps):
-        v, cores, desc, total = oracle_sample(wl, layers_x)
+        r = oracle_sample(wl, layers_x)
         if i >= args.warmup:
-            vals.append(v)
-            tot += total
-    value = float(np.mean(vals))
+            recs.append(r)
+    value = float(np.mean([r["tokens_per_s"] for r in recs]))
+    sample_s = float(np.mean([r["sample_s"] for r in recs]))
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / max(1, args.steps),
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sample_s,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": wl.name, "tokens": wl.batch.total_tokens, "layers": wl.n_layers},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "config": config_dict(wl), "extrapolated": True, "sample_s": sample_s,
+            "extrapolated_ms_per_step": 1e3 * float(np.mean([r["step_s_extrapolated"] for r in recs])),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": recs[0]["cores"], "kind": "oracle",
+                             "sample": recs[0]["sample"], "sample_s": sample_s, "extrapolated": True},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
 
 
-def run_sweep(args):
-    """--sweep: the long-video workload (cfg 3) under masks of growing block density, and its compression at
-    three keep ratios.  Prints one JSON line with a table; a companion to the default line, not a replacement."""
+# ---- timing helpers ---------------------------------------------------------------------------------------------
+class ColdTimer:
+    """CUDA-event timing of single calls with L2 flushed before each (a 256 MiB fill; L2 is 126 MB)."""
+
+    def __init__(self):
+        import torch
+        self.torch = torch
+        self.flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def __call__(self, fn, reps=5):
+        torch = self.torch
+        out = []
+        for _ in range(reps):
+            self.flush.zero_()
+            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            c.record()
+            torch.cuda.synchronize()
+            out.append(a.elapsed_time(c))
+        return float(np.median(out))
+
+
+def device_qkv(wl, layers_q, layers_kv, seed):
+    """Seeded N(0,1) tensors drawn on the device: the side records are timings (their workloads' parity is
+    covered by the tests), and the host generator would dominate the run."""
+    import torch
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    t = wl.batch.total_tokens
+    dt = torch.bfloat16
+    mk = lambda n, h: torch.randn((n, t, h, wl.head_dim), generator=g, device="cuda", dtype=torch.float32).to(dt) if n else None
+    q = torch.empty((layers_q, t, wl.n_q_heads, wl.head_dim), dtype=dt, device="cuda")
+    k = torch.empty((layers_kv, t, wl.n_kv_heads, wl.head_dim), dtype=dt, device="cuda")
+    v = torch.empty_like(k)
+    for l in range(layers_q):
+        q[l] = mk(1, wl.n_q_heads)[0]
+    for l in range(layers_kv):
+        k[l] = mk(1, wl.n_kv_heads)[0]
+        v[l] = mk(1, wl.n_kv_heads)[0]
+    return q, k, v
+
+
+def make_pipeline(wl):
+    import torch
+    from paper_2510_25600_b200.pipeline import PureKVPipeline
+    b = wl.batch
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    kv_layers = max(wl.n_layers, wl.compacted_layers[-1] + 1)
+    return PureKVPipeline(b.seq_lens, b.n_prefix, b.n_frames, wl.mask, wl.n_layers, wl.n_q_heads, wl.n_kv_heads,
+                          wl.head_dim, tdt, wl.scored_layers, wl.compacted_layers, wl.window, wl.keep_ratio, kv_layers), kv_layers
+
+
+def time_pipeline(pipe, wl, d_in, steps, warmup, local, world, peaks, sync_all):
+    """Times `steps` passes of the whole hot path with inputs resident in HBM.  Returns (ms per step on this
+    rank, clocks sampled during the region, roofline record of the prefill kernel)."""
+    import torch
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    # per-launch events only in the warm-up passes; in the timed region three events per step (start, after the
+    # dense layers, end), so consecutive launches still overlap their ramp and tail
+    events = [[(ev(), ev()) for _ in range(wl.n_layers)] for _ in range(warmup)]
+    marks = [(ev(), ev(), ev()) for _ in range(steps)]
+    for s in range(warmup):
+        pipe.run_device(*d_in, events=events[s])
+    pipe.check_status()
+    sampler = ClockSampler(local)
+    sampler.start()
+    sync_all()
+    e0, e1 = ev(), ev()
+    e0.record()
+    for s in range(steps):
+        pipe.run_device(*d_in, marks=marks[s])
+    e1.record()
+    sync_all()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    pipe.check_status()
+    info_d, info_s = pipe.plan_dense.info, pipe.plan_st.info
+    n_dense = pipe.clie + 1
+    n_st = wl.n_layers - n_dense
+    flops_tile = 4.0 * info_s.tile_q * info_s.tile_k * wl.head_dim * wl.n_q_heads
+    fl_dense, fl_st = flops_tile * n_dense * info_d.tiles_kept, flops_tile * n_st * info_s.tiles_kept
+    ms_dense = float(np.mean([m[0].elapsed_time(m[1]) for m in marks]))
+    ms_st = float(np.mean([m[1].elapsed_time(m[2]) for m in marks])) if n_st else 0.0
+    ms_prefill = ms_dense + ms_st
+    achieved = (fl_dense + fl_st) / (ms_prefill * 1e-3) / 1e12
+    peak, which, why = pick_tensor_peak(peaks, clocks)
+    k_ms = np.array([[p[0].elapsed_time(p[1]) for p in step] for step in events[1:]])     # [warm-up passes, layers]
+    part = lambda fl, ms: None if ms <= 0 else dict(ms_per_step=ms, TFLOPs=fl / ms / 1e9, frac=fl / ms / 1e9 / peak,
+                                                   **tensor_fracs(fl / ms / 1e9, peaks))
+    roofline = {"kernel": f"prefill_tc_kernel (128-key entries, skip granularity {info_s.tile_k})", "bound": "tensor",
+                "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "peak_kind": f"measured {which} cuBLAS bf16 ({why})" if "bf16_tflops_sustained" in peaks else f"fallback {which}",
+                **tensor_fracs(achieved, peaks), "traffic": ncu_traffic(wl.name),
+                "traffic_note": "ncu capture summarised in profiles/; null when the kernel sources changed since",
+                "algorithmic_bytes_per_launch": wl.batch.total_tokens * wl.head_dim * 2 * (2 * wl.n_q_heads + 2 * wl.n_kv_heads),
+                "flops_per_step": fl_dense + fl_st, "launches_per_step": wl.n_layers,
+                "avg_launch_ms": ms_prefill / wl.n_layers,
+                "st_layers": part(fl_st, ms_st), "dense_layers": part(fl_dense, ms_dense),
+                "st_layer_ms_isolated": float(k_ms[:, n_dense:].mean()) if n_st and len(k_ms) else None,
+                "dense_layer_ms_isolated": float(k_ms[:, :n_dense].mean()) if len(k_ms) else None,
+                "tiles_kept_st": info_s.tiles_kept, "tiles_causal": info_s.tiles_causal,
+                "useful_flops_per_step": 4.0 * wl.head_dim * wl.n_q_heads * (n_dense * info_d.pairs_kept + n_st * info_s.pairs_kept)}
+    return ms_total / steps, clocks, roofline
+
+
+def compression_detail(pipe, wl, d_in, peaks, timer):
+    """Score / select / compact (and a decode pass over the compact cache) timed one call at a time, cold L2."""
+    import torch
+    from paper_2510_25600_b200 import binding as P
+    b = wl.batch
+    tokens = b.total_tokens
+    q, k, v = d_in
+    esz = 2 if wl.dtype == "bf16" else 4
+    lo, hi = pipe.compacted[0], pipe.compacted[-1] + 1
+    nc = hi - lo
+    sl = pipe.scored[-1]
+    if pipe.one_pass_scores:          # as the pipeline runs it: from the log-sum-exp the scored layer's prefill left
+        t_score = timer(lambda: P.purekv_lowlayer_score_lse(q[sl], k[sl], pipe.lse[len(pipe.scored) - 1], pipe.batch,
+                                                            wl.window, c_out=pipe.c[0], status=pipe.status))
+    else:
+        t_score = timer(lambda: P.purekv_lowlayer_score(q[sl], k[sl], pipe.batch, wl.window, c_out=pipe.c[0],
+                                                        ws=pipe.score_ws))
+    t_select = timer(lambda: P.purekv_select_topk(pipe.c[len(pipe.scored) - 1], v[lo:hi], pipe.batch, pipe.budget,
+                                                  idx_out=pipe.idx, ws=pipe.select_ws))
+    t_compact = timer(lambda: P.purekv_compact_kv(k[lo:hi], v[lo:hi], pipe.idx, pipe.batch, pipe.budget,
+                                                  k_out=pipe.k_c, v_out=pipe.v_c))
+    row = wl.n_kv_heads * wl.head_dim * esz
+    kt = pipe.budget.total_kept
+    w_rows = sum(min(wl.window, int(l)) for l in b.seq_lens)
+    bytes_score = tokens * row + w_rows * wl.n_q_heads * wl.head_dim * esz + wl.n_kv_heads * tokens * 4
+    bytes_select = nc * (tokens * row + wl.n_kv_heads * tokens * 4 + wl.n_kv_heads * kt * 4)
+    bytes_compact = nc * (4 * kt * row + wl.n_kv_heads * kt * 4)
+    passes = 1 if pipe.one_pass_scores else 2
+    score_tf = passes * 2.0 * wl.n_q_heads * wl.head_dim * sum(min(wl.window, int(l)) * int(l) for l in b.seq_lens) / t_score / 1e9
+    detail = {"score": dict(hbm_rec(t_score, bytes_score, peaks), TFLOPs=score_tf,
+                            frac_tensor_burst=score_tf / float(peaks["bf16_tflops"]),
+                            kernel="one pass, tcgen05, from the prefill's log-sum-exp" if pipe.one_pass_scores else "two passes"),
+              "select": hbm_rec(t_select, bytes_select, peaks),
+              "compact": hbm_rec(t_compact, bytes_compact, peaks),
+              "hbm_peak_GBps": float(peaks["hbm_gbs"]), "timing": "cold L2 (256 MiB flush before each call), median of 5"}
+    # what the compact cache is for: one decode step (one new query per request) over all compacted layers,
+    # one call per layer; not part of the timed step or of `value`
+    g = wl.n_q_heads // wl.n_kv_heads
+    if g <= (16 if wl.dtype == "bf16" else 8) and wl.head_dim * esz == 256:
+        kept_max = int(np.diff(pipe.budget.h_cu_kept).max())
+        q_dec = torch.randn((b.n_req, wl.n_q_heads, wl.head_dim), device="cuda").to(q.dtype)
+        o_dec = torch.empty_like(q_dec)
+        dec_need = P.purekv_decode_ws_bytes(b.n_req, kept_max, wl.n_q_heads, wl.n_kv_heads, wl.head_dim)
+        dec_ws = torch.empty(max(16, dec_need), dtype=torch.uint8, device="cuda")
+
+        def decode_all_layers():
+            for layer in range(nc):
+                P.purekv_decode_attention(q_dec, pipe.k_c[layer], pipe.v_c[layer], pipe.budget, out=o_dec, ws=dec_ws)
+        t_decode = timer(decode_all_layers)
+        bytes_decode = nc * (2 * kt * row + 2 * b.n_req * wl.n_q_heads * wl.head_dim * esz)
+        detail["decode_step_after"] = dict(hbm_rec(t_decode, bytes_decode, peaks), launches=nc * (2 if dec_need else 1),
+                                           us_per_layer=1e3 * t_decode / nc,
+                                           note="one new query per request over the compact cache of every compacted layer, "
+                                                "one call per layer; outside the timed step")
+    return detail
+
+
+# ---- side records of the other workloads (one GPU only) ----------------------------------------------------------
+def sub_pipeline(cfg, steps, peaks, timer):
+    """A whole-pipeline workload (cfg 1) as a compact record: device-drawn inputs, its own clock samples."""
+    import torch
+    from paper_2510_25600_b200 import inputs
+    wl = inputs.workload(cfg)
+    pipe, kv_layers = make_pipeline(wl)
+    d_in = device_qkv(wl, wl.n_layers, kv_layers, wl.seed)
+    ms_step, clocks, roofline = time_pipeline(pipe, wl, d_in, steps, 3, torch.cuda.current_device(), 1, peaks,
+                                              torch.cuda.synchronize)
+    keep = ("achieved", "peak", "frac", "peak_kind", "of_measured_burst", "of_measured_sustained", "of_nominal_2250",
+            "avg_launch_ms", "st_layers", "dense_layers", "tiles_kept_st", "tiles_causal")
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    detail = compression_detail(pipe, wl, d_in, peaks, timer)
+    return {"config": config_dict(wl), "inputs": "N(0,1) bf16 drawn on the device (seeded); timing only",
+            "tokens_per_s": wl.batch.total_tokens / (ms_step * 1e-3), "ms_per_step": ms_step, "steps": steps, "clocks": clocks,
+            "roofline": {k: roofline[k] for k in keep}, "steps_detail": detail, "steps_detail_clocks": sampler.stop()}
+
+
+def sub_long_video(reps, peaks, timer):
+    """cfg 3: one layer of the long-video workload under masks of growing block density (the paper's mask and this
+    library's extended settings), and its compression at keep ratios 0.1 / 0.2 / 0.5."""
     import torch
     from paper_2510_25600_b200 import binding as P, inputs
     wl = inputs.workload(3)
     b = wl.batch
-    peaks, peak_kind = load_peaks()
-    pool = ThreadPoolExecutor(len(os.sched_getaffinity(0)))
-    x = inputs.make_qkv(wl, 0, pool=pool)
-    up = lambda n: torch.from_numpy(x[n + "_bits"].view(np.int16)).cuda().view(torch.bfloat16)
-    q, k, v = up("q"), up("k"), up("v")
+    qq, kk, vv = device_qkv(wl, 1, 1, wl.seed)
+    q, k, v = qq[0], kk[0], vv[0]
     db = P.Batch(b.seq_lens, b.n_prefix, b.n_frames)
     g = b.grid_h
     M = inputs.STMask
@@ -255,108 +488,173 @@ def run_sweep(args):
     masks += [(f"whole-frame links, depth {d}", M(g, g, 1, -1, d, 1, -1, tile=128)) for d in (1, 2, 4, 8, 16)]
     masks += [(f"same cell of all earlier frames at stride {st}", M(g, g, 1, -1, -1, st, 0, tile=128)) for st in (10, 5, 3)]
     masks += [("spatial radius 4", M(g, g, 1, 4, 1, 1, 0, tile=128)), ("dense causal", M(g, g, tile=128, dense_causal=True))]
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     o = torch.empty_like(q)
-
-    def timed(fn, reps):
-        out = []
-        for _ in range(reps):
-            flush.zero_()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            fn()
-            e1.record()
-            torch.cuda.synchronize()
-            out.append(e0.elapsed_time(e1))
-        return float(np.median(out))
-
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
     rows = []
-    peak = float(peaks["bf16_tflops"])
     for name, m in masks:
         plan = P.purekv_plan_build(db, P.st_params(m), P.BF16, wl.head_dim, wl.n_q_heads, wl.n_kv_heads)
         ws = torch.empty(max(16, plan.info.ws_bytes), dtype=torch.uint8, device="cuda")
         fn = lambda: P.purekv_st_sparse_prefill(q, k, v, db, plan, out=o, status=status, ws=ws)
         for _ in range(3):
             fn()
-        ms = timed(fn, max(3, min(args.steps, 10)))
+        ms = timer(fn, reps)
         info = plan.info
         tf = 4.0 * info.tile_q * info.tile_k * wl.head_dim * wl.n_q_heads * info.tiles_kept / ms / 1e9
         rows.append({"mask": name, "block_density": info.tiles_kept / info.tiles_causal, "ms": ms, "TFLOPs": tf,
-                     "frac_of_burst_peak": tf / peak, "tokens_per_s": b.total_tokens / (ms * 1e-3)})
+                     "tokens_per_s": b.total_tokens / (ms * 1e-3), **tensor_fracs(tf, peaks)})
     P.purekv_poll_status(status)
+    clocks_prefill = sampler.stop()
+    peak, which, why = pick_tensor_peak(peaks, clocks_prefill)
+    for r in rows:
+        r["frac"] = r["TFLOPs"] / peak
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
     comp = []
-    hbm = float(peaks["hbm_gbs"])
-    kk, vv = k[None].contiguous(), v[None].contiguous()
+    k4, v4 = k[None], v[None]
     row = wl.n_kv_heads * wl.head_dim * 2
-    for keep in (0.1, 0.2, 0.5):
-        bud = P.Budget(db, wl.window, keep)
-        c = P.purekv_lowlayer_score(q, k, db, wl.window)
-        idx = P.purekv_select_topk(c, vv, db, bud)
-        t_sel = timed(lambda: P.purekv_select_topk(c, vv, db, bud, idx_out=idx), 5)
-        kc, vc = P.purekv_compact_kv(kk, vv, idx, db, bud)
-        t_cmp = timed(lambda: P.purekv_compact_kv(kk, vv, idx, db, bud, k_out=kc, v_out=vc), 5)
-        by = 4 * bud.total_kept * row + wl.n_kv_heads * bud.total_kept * 4
-        # one decode step (one new query) over this layer's compact cache
-        q_dec = q[-1:].contiguous()
-        o_dec = torch.empty_like(q_dec)
-        ws_dec = torch.empty(max(16, P.purekv_decode_ws_bytes(1, bud.total_kept, wl.n_q_heads, wl.n_kv_heads, wl.head_dim)),
-                             dtype=torch.uint8, device="cuda")
-        t_dec = timed(lambda: P.purekv_decode_attention(q_dec, kc[0], vc[0], bud, out=o_dec, ws=ws_dec), 5)
-        comp.append({"keep_ratio": keep, "kept": bud.total_kept, "select_ms": t_sel, "compact_ms": t_cmp,
-                     "compact_GBps": by / t_cmp / 1e6, "compact_frac_hbm": by / t_cmp / 1e6 / hbm,
-                     "decode_ms": t_dec, "decode_GBps": 2 * bud.total_kept * row / t_dec / 1e6})
-    t_score = timed(lambda: P.purekv_lowlayer_score(q, k, db, wl.window, c_out=c), 5)
-    # the same scores in one pass from the dense layer's log-sum-exp (what the pipeline runs for this shape)
-    dense = inputs.STMask(b.grid_h, b.grid_w, tile=wl.mask.tile, dense_causal=True)
+    # scores as the pipeline takes them: one pass from the dense layer's log-sum-exp; and the two-pass form
+    dense = M(g, g, tile=128, dense_causal=True)
     plan_d = P.purekv_plan_build(db, P.st_params(dense), P.BF16, wl.head_dim, wl.n_q_heads, wl.n_kv_heads)
     ws_d = torch.empty(max(16, plan_d.info.ws_bytes), dtype=torch.uint8, device="cuda")
     lse = torch.empty((wl.n_q_heads, b.total_tokens), dtype=torch.float32, device="cuda")
     P.purekv_st_sparse_prefill(q, k, v, db, plan_d, out=o, lse=lse, status=status, ws=ws_d)
-    t_score_lse = timed(lambda: P.purekv_lowlayer_score_lse(q, k, lse, db, wl.window, c_out=c, status=status), 5)
+    c = P.purekv_lowlayer_score_lse(q, k, lse, db, wl.window, status=status)
+    t_score_lse = timer(lambda: P.purekv_lowlayer_score_lse(q, k, lse, db, wl.window, c_out=c, status=status))
+    t_score_2p = timer(lambda: P.purekv_lowlayer_score(q, k, db, wl.window, c_out=c))
+    score_fl = 2.0 * wl.n_q_heads * wl.head_dim * wl.window * b.total_tokens
+    bytes_score = b.total_tokens * row + wl.window * wl.n_q_heads * wl.head_dim * 2 + wl.n_kv_heads * b.total_tokens * 4
+    for keep in (0.1, 0.2, 0.5):
+        bud = P.Budget(db, wl.window, keep)
+        idx = P.purekv_select_topk(c, v4, db, bud)
+        t_sel = timer(lambda: P.purekv_select_topk(c, v4, db, bud, idx_out=idx))
+        kc, vc = P.purekv_compact_kv(k4, v4, idx, db, bud)
+        t_cmp = timer(lambda: P.purekv_compact_kv(k4, v4, idx, db, bud, k_out=kc, v_out=vc))
+        by = 4 * bud.total_kept * row + wl.n_kv_heads * bud.total_kept * 4
+        by_sel = b.total_tokens * row + wl.n_kv_heads * b.total_tokens * 4 + wl.n_kv_heads * bud.total_kept * 4
+        q_dec = q[-1:].contiguous()
+        o_dec = torch.empty_like(q_dec)
+        ws_dec = torch.empty(max(16, P.purekv_decode_ws_bytes(1, bud.total_kept, wl.n_q_heads, wl.n_kv_heads, wl.head_dim)),
+                             dtype=torch.uint8, device="cuda")
+        t_dec = timer(lambda: P.purekv_decode_attention(q_dec, kc[0], vc[0], bud, out=o_dec, ws=ws_dec))
+        comp.append({"keep_ratio": keep, "kept": bud.total_kept, "select": hbm_rec(t_sel, by_sel, peaks),
+                     "compact": hbm_rec(t_cmp, by, peaks), "decode_step": hbm_rec(t_dec, 2 * bud.total_kept * row, peaks)})
     P.purekv_poll_status(status)
-    # the decode step where it is bandwidth bound: many requests, each with a few thousand kept rows (synthetic cache)
-    n_big, kept_big = 128, 4096
+    return {"config": config_dict(wl), "inputs": "N(0,1) bf16 drawn on the device (seeded); timing only",
+            "prefill": rows, "prefill_peak": peak, "prefill_peak_kind": f"measured {which} ({why})", "prefill_clocks": clocks_prefill,
+            "score_one_pass": dict(hbm_rec(t_score_lse, bytes_score, peaks), TFLOPs=score_fl / t_score_lse / 1e9,
+                                   frac_tensor_burst=score_fl / t_score_lse / 1e9 / float(peaks["bf16_tflops"])),
+            "score_two_pass": dict(hbm_rec(t_score_2p, bytes_score, peaks), TFLOPs=2 * score_fl / t_score_2p / 1e9),
+            "compression": comp, "compression_clocks": sampler.stop(),
+            "note": "masks other than the paper mask are this library's extended settings; 38 MB of K+V per layer: "
+                    "the compression calls are latency dominated here",
+            "timing": "cold L2 (256 MiB fill before each call), median"}
+
+
+def sub_ragged(reps, peaks, timer):
+    """cfg 4: the ragged serving batch -- one prefill layer under both masks, then scores, selection and compaction
+    of all 27 compressed layers into the packed compact cache."""
+    import torch
+    from paper_2510_25600_b200 import binding as P, inputs
+    wl = inputs.workload(4)
+    b = wl.batch
+    nc = len(wl.compacted_layers)
+    qq, kk, vv = device_qkv(wl, 1, nc, wl.seed)
+    q = qq[0]
+    db = P.Batch(b.seq_lens, b.n_prefix, b.n_frames)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    o = torch.empty_like(q)
+    lse = torch.empty((wl.n_q_heads, b.total_tokens), dtype=torch.float32, device="cuda")
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    pre = []
+    for name, m in (("paper mask", wl.mask), ("dense causal", inputs.STMask(b.grid_h, b.grid_w, tile=128, dense_causal=True))):
+        plan = P.purekv_plan_build(db, P.st_params(m), P.BF16, wl.head_dim, wl.n_q_heads, wl.n_kv_heads)
+        ws = torch.empty(max(16, plan.info.ws_bytes), dtype=torch.uint8, device="cuda")
+        fn = lambda: P.purekv_st_sparse_prefill(q, kk[0], vv[0], db, plan, out=o, lse=lse, status=status, ws=ws)
+        for _ in range(3):
+            fn()
+        ms = timer(fn, reps)
+        info = plan.info
+        tf = 4.0 * info.tile_q * info.tile_k * wl.head_dim * wl.n_q_heads * info.tiles_kept / ms / 1e9
+        pre.append({"mask": name, "block_density": info.tiles_kept / info.tiles_causal, "ms": ms, "TFLOPs": tf,
+                    "tokens_per_s": b.total_tokens / (ms * 1e-3), **tensor_fracs(tf, peaks)})
+    clocks_prefill = sampler.stop()
+    peak, which, why = pick_tensor_peak(peaks, clocks_prefill)
+    for r in pre:
+        r["frac"] = r["TFLOPs"] / peak
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    row = wl.n_kv_heads * wl.head_dim * 2
+    tokens = b.total_tokens
+    one_pass = wl.window % 8 == 0 and all(l >= wl.window or l % 8 == 0 for l in b.seq_lens)
+    if one_pass:        # lse holds the dense layer's rows (the last prefill above)
+        c = P.purekv_lowlayer_score_lse(q, kk[0], lse, db, wl.window, status=status)
+        t_score = timer(lambda: P.purekv_lowlayer_score_lse(q, kk[0], lse, db, wl.window, c_out=c, status=status))
+    else:
+        c = P.purekv_lowlayer_score(q, kk[0], db, wl.window)
+        t_score = timer(lambda: P.purekv_lowlayer_score(q, kk[0], db, wl.window, c_out=c))
+    bud = P.Budget(db, wl.window, wl.keep_ratio)
+    ws_sel = torch.empty(P.purekv_select_ws_bytes(db, nc, wl.n_kv_heads), dtype=torch.uint8, device="cuda")
+    idx = P.purekv_select_topk(c, vv, db, bud, ws=ws_sel)
+    t_sel = timer(lambda: P.purekv_select_topk(c, vv, db, bud, idx_out=idx, ws=ws_sel))
+    kc, vc = P.purekv_compact_kv(kk, vv, idx, db, bud)
+    t_cmp = timer(lambda: P.purekv_compact_kv(kk, vv, idx, db, bud, k_out=kc, v_out=vc))
+    P.purekv_poll_status(status)
+    kt = bud.total_kept
+    w_rows = sum(min(wl.window, int(l)) for l in b.seq_lens)
+    score_fl = 2.0 * wl.n_q_heads * wl.head_dim * sum(min(wl.window, int(l)) * int(l) for l in b.seq_lens)
+    rec = {"config": config_dict(wl), "inputs": "N(0,1) bf16 drawn on the device (seeded); timing only",
+           "prefill": pre, "prefill_peak": peak, "prefill_peak_kind": f"measured {which} ({why})", "prefill_clocks": clocks_prefill,
+           "score": dict(hbm_rec(t_score, tokens * row + w_rows * wl.n_q_heads * wl.head_dim * 2 + wl.n_kv_heads * tokens * 4, peaks),
+                         TFLOPs=(1 if one_pass else 2) * score_fl / t_score / 1e9,
+                         kernel="one pass (tcgen05)" if one_pass else "two passes"),
+           "select": hbm_rec(t_sel, nc * (tokens * row + wl.n_kv_heads * tokens * 4 + wl.n_kv_heads * kt * 4), peaks),
+           "compact": hbm_rec(t_cmp, nc * (4 * kt * row + wl.n_kv_heads * kt * 4), peaks),
+           "compression_clocks": sampler.stop(), "timing": "cold L2 (256 MiB fill before each call), median"}
+    return rec
+
+
+def decode_large_batch(peaks, timer):
+    """The decode step where it is bandwidth bound: many requests, each with a few thousand kept rows."""
+    import torch
+    from paper_2510_25600_b200 import binding as P
+    n_big, kept_big, h, hkv, d = 128, 4096, 28, 4, 128
 
     class _Kept:
         h_cu_kept = np.arange(n_big + 1, dtype=np.int32) * kept_big
         cu_kept = torch.from_numpy(h_cu_kept.copy()).cuda()
-    kc_big = torch.randn((n_big * kept_big, wl.n_kv_heads, wl.head_dim), device="cuda").to(torch.bfloat16)
-    vc_big = torch.randn_like(kc_big)
-    q_big = torch.randn((n_big, wl.n_q_heads, wl.head_dim), device="cuda").to(torch.bfloat16)
-    o_big = torch.empty_like(q_big)
-    ws_big = torch.empty(max(16, P.purekv_decode_ws_bytes(n_big, kept_big, wl.n_q_heads, wl.n_kv_heads, wl.head_dim)),
-                         dtype=torch.uint8, device="cuda")
-    t_big = timed(lambda: P.purekv_decode_attention(q_big, kc_big, vc_big, _Kept, out=o_big, ws=ws_big), 5)
-    by_big = 2 * kc_big.numel() * 2 + 2 * q_big.numel() * 2
-    decode_big = {"requests": n_big, "kept_per_request": kept_big, "heads": [wl.n_q_heads, wl.n_kv_heads], "ms": t_big,
-                  "GBps": by_big / t_big / 1e6, "frac_hbm": by_big / t_big / 1e6 / hbm, "bytes": by_big}
-    print(json.dumps({"sweep": wl.name, "tokens": b.total_tokens, "peak_TFLOPs": peak, "peak_kind": peak_kind + " burst (kernel timed alone)",
-                      "prefill": rows, "score_ms": t_score, "score_one_pass_ms": t_score_lse,
-                      "compression": comp, "decode_large_batch": decode_big,
-                      "timing": "cold L2 (256 MiB fill before each call), median"}), flush=True)
+    kc = torch.randn((n_big * kept_big, hkv, d), device="cuda").to(torch.bfloat16)
+    vc = torch.randn_like(kc)
+    q = torch.randn((n_big, h, d), device="cuda").to(torch.bfloat16)
+    o = torch.empty_like(q)
+    ws = torch.empty(max(16, P.purekv_decode_ws_bytes(n_big, kept_big, h, hkv, d)), dtype=torch.uint8, device="cuda")
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    t = timer(lambda: P.purekv_decode_attention(q, kc, vc, _Kept, out=o, ws=ws))
+    return dict(hbm_rec(t, 2 * kc.numel() * 2 + 2 * q.numel() * 2, peaks), requests=n_big, kept_per_request=kept_big,
+                heads=[h, hkv], clocks=sampler.stop())
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--cfg", type=int, default=1)
+    ap.add_argument("--cfg", type=int, default=2)
     ap.add_argument("--impl", default="purekv")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sub", action="store_true", help="skip the side records of the other workloads (`configs`)")
+    ap.add_argument("--only-sub", default="", help="print only these side records (comma list of cfg1,cfg3,cfg4,decode) and exit")
     ap.add_argument("--print-kernel-hash", action="store_true", help="sha1 of the prefill kernel sources, then exit")
-    ap.add_argument("--sweep", action="store_true", help="long-video workload: TFLOP/s against block density, compaction")
     args = ap.parse_args()
     if args.print_kernel_hash:
         print(kernel_source_sha1())
         return
     args.warmup = max(args.warmup, 3) if args.impl != "reference" else args.warmup
 
-    if args.sweep:
-        run_sweep(args)
-        return
     from paper_2510_25600_b200 import inputs
     wl = inputs.workload(args.cfg)
     if args.impl == "reference":
@@ -365,24 +663,37 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2510_25600_b200 import binding as P
-    from paper_2510_25600_b200.pipeline import PureKVPipeline
+    from paper_2510_25600_b200 import binding as P   # noqa: F401  (raises if the CUDA library is missing)
 
     world, rank, local = rank_env()
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks, peak_kind = load_peaks()
+    timer = ColdTimer()
+
+    def side_records(which):
+        recs = {}
+        for name, fn in (("cfg1_videollama2", lambda: sub_pipeline(1, 20, peaks, timer)),
+                         ("cfg3_long_video", lambda: sub_long_video(5, peaks, timer)),
+                         ("cfg4_ragged_batch", lambda: sub_ragged(5, peaks, timer)),
+                         ("decode_large_batch", lambda: decode_large_batch(peaks, timer))):
+            if which is None or any(w and w in name for w in which):
+                recs[name] = fn()
+                torch.cuda.empty_cache()
+        return recs
+
+    if args.only_sub:
+        print(json.dumps({"configs": side_records(args.only_sub.split(",")), "peaks": peak_kind}), flush=True)
+        return
 
     # ---- inputs: generated on the host from the seed, then resident in HBM -------------------------------
     b = wl.batch
-    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
-    kv_layers = max(wl.n_layers, wl.compacted_layers[-1] + 1)
-    pipe = PureKVPipeline(b.seq_lens, b.n_prefix, b.n_frames, wl.mask, wl.n_layers, wl.n_q_heads, wl.n_kv_heads,
-                          wl.head_dim, tdt, wl.scored_layers, wl.compacted_layers, wl.window, wl.keep_ratio, kv_layers)
+    pipe, kv_layers = make_pipeline(wl)
     (hq, hk, hv), h_out = pipe.alloc_host_io()
     pool = ThreadPoolExecutor(len(os.sched_getaffinity(0)))
-    keep_for_oracle = []
+    keep_for_oracle = {}
+    st_layer = min(max(wl.scored_layers) + 1, wl.n_layers - 1)
     for layer in range(kv_layers):
         x = inputs.make_qkv(wl, layer, which="qkv" if layer < wl.n_layers else "kv", pool=pool)
         key = "_bits" if wl.dtype == "bf16" else ""
@@ -391,8 +702,8 @@ def main():
             hq[layer].copy_(view(x["q" + key]))
         hk[layer].copy_(view(x["k" + key]))
         hv[layer].copy_(view(x["v" + key]))
-        if layer < 2:
-            keep_for_oracle.append(x)
+        if layer in (0, st_layer):
+            keep_for_oracle[layer] = x
     d_in = tuple(t.cuda() for t in (hq, hk, hv))
     torch.cuda.synchronize()
 
@@ -403,118 +714,17 @@ def main():
             torch.cuda.synchronize()
 
     # ---- device-resident timing ---------------------------------------------------------------------------
-    # per-launch events only in the warm-up passes (they tell dense from ST layers); in the timed region one event pair
-    # per step spans the prefill launches, so consecutive launches still overlap their ramp and tail
-    ev = lambda: torch.cuda.Event(enable_timing=True)
-    events = [[(ev(), ev()) for _ in range(wl.n_layers)] for _ in range(args.warmup)]
-    spans = [(ev(), ev()) for _ in range(args.steps)]
-    for s in range(args.warmup):
-        pipe.run_device(*d_in, events=events[s])
-    pipe.check_status()
-    sampler = ClockSampler(local)
-    sampler.start()
-    sync_all()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for s in range(args.steps):
-        pipe.run_device(*d_in, span=spans[s])
-    e1.record()
-    sync_all()
-    ms_total = e0.elapsed_time(e1)
-    clocks = sampler.stop()
-    pipe.check_status()
-    ms_step = max_over_ranks(ms_total, "cuda") / args.steps
+    ms_rank, clocks, roofline = time_pipeline(pipe, wl, d_in, args.steps, args.warmup, local, world, peaks, sync_all)
+    ms_step = max_over_ranks(ms_rank, "cuda")
     tokens = b.total_tokens
     value = job_throughput(tokens, world, ms_step * 1e-3)
 
-    # ---- roofline of the dominant kernel (tensor-core prefill), from events around each launch -------------
-    info_d, info_s = pipe.plan_dense.info, pipe.plan_st.info
-    n_dense = pipe.clie + 1
-    flops_tile = 4.0 * info_s.tile_q * info_s.tile_k * wl.head_dim * wl.n_q_heads
-    flops_step = flops_tile * (n_dense * info_d.tiles_kept + (wl.n_layers - n_dense) * info_s.tiles_kept)
-    k_ms = np.array([[p[0].elapsed_time(p[1]) for p in step] for step in events[1:]])     # [warm-up passes, layers]
-    prefill_ms_step = float(np.mean([p[0].elapsed_time(p[1]) for p in spans]))          # timed region, all launches of a step
-    achieved = flops_step / (prefill_ms_step * 1e-3) / 1e12
-    peak = float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]))
-    roofline = {"kernel": f"prefill_tc_kernel (128-key entries, skip granularity {info_s.tile_k})", "bound": "tensor", "achieved": achieved, "peak": peak,
-                "unit": "TFLOP/s", "frac": achieved / peak, "traffic": ncu_traffic(wl.name),
-                "algorithmic_bytes_per_launch": b.total_tokens * wl.head_dim * 2 * (2 * wl.n_q_heads + 2 * wl.n_kv_heads),
-                "peak_kind": f"{peak_kind} sustained cuBLAS bf16 (burst {peaks['bf16_tflops']}, nominal dense 2250)",
-                "flops_per_step": flops_step, "launches_per_step": wl.n_layers, "avg_launch_ms": prefill_ms_step / wl.n_layers,
-                "st_layer_ms_isolated": float(k_ms[:, n_dense:].mean()) if wl.n_layers > n_dense else None,
-                "dense_layer_ms_isolated": float(k_ms[:, :n_dense].mean()),
-                "tiles_kept_st": info_s.tiles_kept, "tiles_causal": info_s.tiles_causal,
-                "useful_flops_per_step": 4.0 * wl.head_dim * wl.n_q_heads *
-                (n_dense * info_d.pairs_kept + (wl.n_layers - n_dense) * info_s.pairs_kept)}
-
-    # ---- per-step breakdown of the HBM-bound steps (separately timed, cold L2: inputs exceed L2) -----------
-    def time_call(fn, reps=5):
-        out = []
-        for _ in range(reps):
-            flush.zero_()
-            a, c = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            fn()
-            c.record()
-            torch.cuda.synchronize()
-            out.append(a.elapsed_time(c))
-        return float(np.median(out))
-
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    q, k, v = d_in
-    esz = 2 if wl.dtype == "bf16" else 4
-    lo, hi = pipe.compacted[0], pipe.compacted[-1] + 1
-    nc = hi - lo
-    sl = pipe.scored[-1]
-    if pipe.one_pass_scores:          # as the pipeline runs it: from the log-sum-exp the scored layer's prefill left
-        t_score = time_call(lambda: P.purekv_lowlayer_score_lse(q[sl], k[sl], pipe.lse[len(pipe.scored) - 1], pipe.batch,
-                                                                wl.window, c_out=pipe.c[0], status=pipe.status))
-    else:
-        t_score = time_call(lambda: P.purekv_lowlayer_score(q[sl], k[sl], pipe.batch, wl.window, c_out=pipe.c[0],
-                                                            ws=pipe.score_ws))
-    t_select = time_call(lambda: P.purekv_select_topk(pipe.c[len(pipe.scored) - 1], v[lo:hi], pipe.batch, pipe.budget,
-                                                      idx_out=pipe.idx, ws=pipe.select_ws))
-    t_compact = time_call(lambda: P.purekv_compact_kv(k[lo:hi], v[lo:hi], pipe.idx, pipe.batch, pipe.budget,
-                                                      k_out=pipe.k_c, v_out=pipe.v_c))
-    # what the compact cache is for: one decode step (one new query per request) over all compacted layers,
-    # one call per layer; not part of the timed step or of `value`
-    kept_max = int(np.diff(pipe.budget.h_cu_kept).max())
-    q_dec = torch.randn((b.n_req, wl.n_q_heads, wl.head_dim), device="cuda").to(q.dtype)
-    o_dec = torch.empty_like(q_dec)
-    dec_need = P.purekv_decode_ws_bytes(b.n_req, kept_max, wl.n_q_heads, wl.n_kv_heads, wl.head_dim)
-    dec_ws = torch.empty(max(16, dec_need), dtype=torch.uint8, device="cuda")
-
-    def decode_all_layers():
-        for layer in range(nc):
-            P.purekv_decode_attention(q_dec, pipe.k_c[layer], pipe.v_c[layer], pipe.budget, out=o_dec, ws=dec_ws)
-    decode_ok = wl.n_q_heads // wl.n_kv_heads <= 8 and wl.head_dim * (2 if wl.dtype == "bf16" else 4) == 256
-    t_decode = time_call(decode_all_layers) if decode_ok else None
+    # ---- per-step breakdown of the HBM-bound steps (separately timed, cold L2) ---------------------------------
+    steps_detail = compression_detail(pipe, wl, d_in, peaks, timer)
     t_plan = time.perf_counter()
     pipe.build_plans()
-    t_plan = (time.perf_counter() - t_plan) * 1e3
-    row = wl.n_kv_heads * wl.head_dim * esz
-    kt = pipe.budget.total_kept
-    bytes_score = tokens * row + min(wl.window, tokens) * wl.n_q_heads * wl.head_dim * esz * b.n_req + wl.n_kv_heads * tokens * 4
-    bytes_select = nc * (tokens * row + wl.n_kv_heads * tokens * 4 + wl.n_kv_heads * kt * 4)
-    bytes_compact = nc * (4 * kt * row + wl.n_kv_heads * kt * 4)
-    hbm = float(peaks["hbm_gbs"])
-    steps_detail = {
-        "plan_build_ms": t_plan,
-        "score": {"ms": t_score, "GBps": bytes_score / t_score / 1e6, "frac_hbm": bytes_score / t_score / 1e6 / hbm,
-                  "kernel": "one pass, tcgen05, from the prefill's log-sum-exp" if pipe.one_pass_scores else "two passes",
-                  "TFLOPs": (1 if pipe.one_pass_scores else 2) * 2.0 * wl.n_q_heads * min(wl.window, tokens) * tokens *
-                  wl.head_dim / t_score / 1e9},
-        "select": {"ms": t_select, "GBps": bytes_select / t_select / 1e6, "frac_hbm": bytes_select / t_select / 1e6 / hbm},
-        "compact": {"ms": t_compact, "GBps": bytes_compact / t_compact / 1e6, "frac_hbm": bytes_compact / t_compact / 1e6 / hbm},
-        "hbm_peak_GBps": hbm, "hbm_peak_kind": peak_kind, "timing": "cold L2 (256 MiB flush before each call), median of 5",
-    }
-    if t_decode is not None:
-        bytes_decode = nc * (2 * kt * row + 2 * b.n_req * wl.n_q_heads * wl.head_dim * esz)
-        steps_detail["decode_step_after"] = {
-            "ms": t_decode, "launches": nc * (2 if dec_need else 1), "us_per_layer": 1e3 * t_decode / nc,
-            "GBps": bytes_decode / t_decode / 1e6, "frac_hbm": bytes_decode / t_decode / 1e6 / hbm,
-            "note": "one new query per request over the compact cache of every compacted layer, one call per layer; "
-                    "outside the timed step"}
+    steps_detail["plan_build_ms"] = (time.perf_counter() - t_plan) * 1e3
+    steps_detail["hbm_peak_kind"] = peak_kind
 
     # ---- end to end: pinned host inputs, compact cache read back ---------------------------------------------
     e2e = None
@@ -533,27 +743,30 @@ def main():
         e2e = {"value": job_throughput(tokens, world, dt / n_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "steps": n_e2e, "ms_per_step": 1e3 * dt / n_e2e}
     pipe.check_status()
+    launches = pipe.launches_per_step * args.steps
 
     # ---- the oracle on this machine's host cores (rank 0, N = 1 only) ---------------------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import purekv_oracle as po
         po.build()
-        v_cpu, cores, desc, _ = oracle_sample(wl, keep_for_oracle)
-        cpu = {"value": v_cpu, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+        r = oracle_sample(wl, [keep_for_oracle[0], keep_for_oracle[st_layer]], n_rows=2048)   # 10-20 s of host work
+        cpu = {"value": r["tokens_per_s"], "unit": UNIT, "cores": r["cores"], "kind": "oracle", "sample": r["sample"],
+               "sample_s": r["sample_s"], "extrapolated": True}
+
+    # ---- the other workloads, each with its own clock samples (one GPU only) -----------------------------------
+    configs = None
+    if rank == 0 and world == 1 and not args.no_sub:
+        del d_in, pipe, hq, hk, hv, h_out
+        torch.cuda.empty_cache()
+        configs = side_records(None)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
-                "config": {"workload": wl.name, "tokens": tokens, "layers": wl.n_layers, "heads": [wl.n_q_heads, wl.n_kv_heads],
-                           "head_dim": wl.head_dim, "tile": wl.mask.tile, "window": wl.window, "keep_ratio": wl.keep_ratio,
-                           "l2": "inputs larger than L2 (each layer reads its own Q/K/V; %.0f MB per step)" %
-                                 (sum(t.numel() * t.element_size() for t in d_in) / 1e6),
-                           "multi_gpu": "replicas only (the path has no exchange step)",
-                           "step": "plan build + %d prefill layers + score + select + compact" % wl.n_layers},
-                "clocks": clocks, "e2e": e2e, "gpu_launches": pipe.launches_per_step * args.steps,
-                "roofline": roofline, "cpu_baseline": cpu, "steps_detail": steps_detail}
+                "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": config_dict(wl),
+                "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+                "roofline": roofline, "cpu_baseline": cpu, "steps_detail": steps_detail, "configs": configs}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -98,22 +98,24 @@ class PureKVPipeline:
         P.purekv_st_sparse_prefill(q, k, v, self.batch, plan, out=self.o[layer], lse=lse, status=self.status,
                                    ws=self.prefill_ws)
 
-    def run_device(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, events=None, span=None) -> None:
+    def run_device(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, events=None, marks=None) -> None:
         """q [n_layers,T,H,d], k,v [kv_layers,T,H_kv,d] on the GPU.  Results in self.o / idx / k_c / v_c.
         `events`, if given, is a list of (start, end) torch.cuda.Event pairs, one per prefill launch (an event
-        between two launches keeps the second from starting under the first's tail); `span`, if given, is one
-        (start, end) pair around all prefill launches."""
+        between two launches keeps the second from starting under the first's tail); `marks`, if given, is three
+        events recorded before the first prefill launch, after the last dense-causal one and after the last one."""
         self.build_plans()
-        if span is not None:
-            span[0].record()
+        if marks is not None:
+            marks[0].record()
         for layer in range(self.n_layers):
             if events is not None:
                 events[layer][0].record()
             self.prefill_layer(layer, q[layer], k[layer], v[layer])
             if events is not None:
                 events[layer][1].record()
-        if span is not None:
-            span[1].record()
+            if marks is not None and layer == self.clie:
+                marks[1].record()
+        if marks is not None:
+            marks[2].record()
         for n, layer in enumerate(self.scored):
             if self.one_pass_scores:
                 P.purekv_lowlayer_score_lse(q[layer], k[layer], self.lse[n], self.batch, self.window, c_out=self.c[n],
