@@ -38,7 +38,8 @@ typedef enum {
   PUREKV_ERR_UNSUPPORTED = 2, /* head_dim / dtype / tile combination without a kernel    */
   PUREKV_ERR_WORKSPACE = 3,   /* plan or workspace buffer too small                      */
   PUREKV_ERR_CUDA = 4,        /* a CUDA call failed; text in purekv_last_error           */
-  PUREKV_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (purekv_poll_status) */
+  PUREKV_ERR_TIMEOUT = 5,     /* a bounded device-side wait expired (purekv_poll_status) */
+  PUREKV_ERR_BAD_PLAN = 6     /* a kernel found the plan it was handed inconsistent and did not use it (purekv_poll_status) */
 } purekv_status;
 
 typedef enum { PUREKV_BF16 = 0, PUREKV_FP32 = 1 } purekv_dtype;
@@ -178,10 +179,12 @@ purekv_status purekv_lowlayer_score_lse(const void *q, const void *k, const floa
  * allocate at all.  For them this entry point keeps its scratch (the window rows' log-sum-exp values)
  * in an array inside the library's device image instead of a caller-provided workspace.  It calls no
  * cudaMalloc / cudaFree and no allocating library routine; inputs and c_out are still the caller's.
- *  - Limit: the problem's workspace need, purekv_score_ws_bytes(batch, window, n_q_heads), must not exceed
- *    PUREKV_NOALLOC_SCORE_MAX_ROWS (65536) values, i.e. n_req * n_q_heads * window * (1 + 2 * ceil(longest
- *    request / 64)) <= 65536 -- 256 KiB that every GPU loading the library holds until the process exits.
- *    Larger problems return PUREKV_ERR_WORKSPACE and leave c_out untouched; use purekv_lowlayer_score.
+ *  - Limit: the problem's workspace need in fp32 values -- with rows = n_req * n_q_heads * max(window, 1):
+ *    rows rounded up to a multiple of 64, plus 2 * rows * ceil(longest request / 64) -- must not exceed
+ *    PUREKV_NOALLOC_SCORE_MAX_ROWS (262144) values: 1 MiB that every GPU loading the library holds until the
+ *    process exits (a 2432-token prompt with 32 query heads and a window of 64 needs 157 696).  Larger problems
+ *    return PUREKV_ERR_WORKSPACE and leave c_out untouched; use purekv_lowlayer_score.  An empty batch returns
+ *    PUREKV_OK whatever the other arguments are.
  *  - The first call on each device looks up the array's device address (with that device current).
  *    Make that first call before any stream capture on that device.
  *  - All calls on a device share the one array, and it keeps the previous call's contents.  Nothing in
@@ -189,7 +192,7 @@ purekv_status purekv_lowlayer_score_lse(const void *q, const void *k, const floa
  *    kernels overlap on the GPU -- different streams, or different host threads -- race on it.
  *    Serialise them, e.g. by issuing them on one stream.
  * Results are those of purekv_lowlayer_score. */
-#define PUREKV_NOALLOC_SCORE_MAX_ROWS 65536
+#define PUREKV_NOALLOC_SCORE_MAX_ROWS 262144
 purekv_status purekv_lowlayer_score_noalloc(const void *q, const void *k, float *c_out,
                                             const purekv_batch *batch, int32_t window, int32_t n_q_heads,
                                             int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
@@ -242,8 +245,22 @@ purekv_status purekv_decode_attention(const void *q, const void *k_cache, const 
                                       int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
                                       float softmax_scale, void *ws, size_t ws_bytes, void *stream);
 
-/* Synchronises `stream`, copies the device status word to *h_status_out and returns
- * PUREKV_ERR_TIMEOUT if it is non-zero, PUREKV_ERR_CUDA if the stream reported an error. */
+/* Failure detection (no counterpart in the paper).  Every wait inside the tensor-core kernels -- on a copy, on a
+ * product, on another role of the CTA -- is bounded: when the limit passes the CTA raises the status word to
+ * PUREKV_ERR_TIMEOUT, lets its copies and products in flight finish, frees its tensor memory and returns, so the
+ * context stays usable.  The limit is process-wide, 1 s by default; ns == 0 restores the default.  The tensor-core
+ * prefill also checks the plan before using it (header, section offsets against the plan's size, every unit's and
+ * entry's indices against the header's counts): on a mismatch nothing is read through the bad field, the status
+ * word becomes PUREKV_ERR_BAD_PLAN and the output is undefined (untouched when the header itself fails).  After either code the plan's scheduling counters are
+ * undefined: build the plan again before the next launch. */
+void purekv_set_wait_limit_ns(uint64_t ns);
+
+/* Synchronises `stream`, copies the device status word to *h_status_out and returns the code it holds
+ * (PUREKV_ERR_TIMEOUT or PUREKV_ERR_BAD_PLAN) if it is non-zero, PUREKV_ERR_CUDA if the stream reported an error.
+ * status == NULL polls the word inside the library that calls made with a NULL status use (one per
+ * device, shared by all such calls) and clears it if it was raised.  A raised word makes every later
+ * call that uses it return without computing -- the caller's own word stays raised until the caller
+ * clears it, the library's until it is polled this way -- so poll after the calls whose results matter. */
 purekv_status purekv_poll_status(const int32_t *status, int32_t *h_status_out, void *stream);
 
 #ifdef __cplusplus

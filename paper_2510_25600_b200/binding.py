@@ -20,7 +20,7 @@ if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2510_25600_b200.build`")
 _lib = C.CDLL(LIB_PATH)
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_PLAN = range(7)
 BF16, FP32 = 0, 1
 FLAG_DENSE_CAUSAL = 1
 
@@ -29,7 +29,7 @@ EXPORTS = ("purekv_version", "purekv_last_error", "purekv_budget", "purekv_plan_
            "purekv_st_sparse_prefill", "purekv_score_ws_bytes", "purekv_lowlayer_score", "purekv_lowlayer_score_lse", "purekv_lowlayer_score_noalloc",
            "purekv_select_ws_bytes",
            "purekv_select_topk", "purekv_compact_kv", "purekv_decode_ws_bytes", "purekv_decode_attention",
-           "purekv_poll_status")
+           "purekv_poll_status", "purekv_set_wait_limit_ns")
 
 _i32p = C.POINTER(C.c_int32)
 
@@ -54,7 +54,22 @@ class PlanInfo(C.Structure):
                 ("max_chunks", C.c_int32), ("ws_bytes", C.c_int64)]
 
 
+class PlanHeaderView(C.Structure):
+    """The first bytes of a plan buffer, field by field (tooling and tests that inspect or edit a host copy)."""
+    _fields_ = [("magic", C.c_uint32), ("tile_q", C.c_int32), ("tile_k", C.c_int32), ("n_qtiles", C.c_int32),
+                ("total_tokens", C.c_int64), ("n_entries", C.c_int64), ("n_mask_words", C.c_int64),
+                ("off_qtiles", C.c_int64), ("off_order", C.c_int64), ("off_entries", C.c_int64), ("off_masks", C.c_int64),
+                ("words_per_row", C.c_int32), ("n_ctas", C.c_int32), ("n_units", C.c_int32), ("n_counters", C.c_int32),
+                ("off_units", C.c_int64), ("off_counters", C.c_int64), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("part_slots", C.c_int64), ("test_flags", C.c_uint32), ("pad_flags", C.c_uint32)]
+
+
+UNIT_INT32S = 12        # a work unit of the tensor-core plan: q_start, q_rows, req_start, ent_begin, ent_count, pair,
+                        # chunk, n_chunks, part_base, counter_base, 2 x padding
+
 _lib.purekv_version.restype = C.c_char_p
+_lib.purekv_set_wait_limit_ns.restype = None
+_lib.purekv_set_wait_limit_ns.argtypes = [C.c_uint64]
 _lib.purekv_plan_bytes.restype = C.c_size_t
 _lib.purekv_score_ws_bytes.restype = C.c_size_t
 _lib.purekv_select_ws_bytes.restype = C.c_size_t
@@ -269,7 +284,7 @@ def purekv_lowlayer_score_lse(q: torch.Tensor, k: torch.Tensor, lse: torch.Tenso
     return c_out
 
 
-NOALLOC_SCORE_MAX_ROWS = 65536
+NOALLOC_SCORE_MAX_ROWS = 262144
 
 
 def purekv_lowlayer_score_noalloc(q: torch.Tensor, k: torch.Tensor, batch: Batch, window: int, c_out: torch.Tensor,
@@ -347,6 +362,11 @@ def purekv_decode_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: tor
                                         ws.numel() * ws.element_size() if ws is not None else 0, _stream()),
            "purekv_decode_attention")
     return out
+
+
+def purekv_set_wait_limit_ns(ns: int) -> None:
+    """Limit of every device-side wait of the tensor-core kernels, process-wide; 0 restores the default (1 s)."""
+    _lib.purekv_set_wait_limit_ns(int(ns))
 
 
 def purekv_poll_status(status: Optional[torch.Tensor]) -> int:

@@ -17,7 +17,7 @@ namespace purekv {
 
 // Scratch of purekv_lowlayer_score_noalloc: the window rows' log-sum-exp values and their per-key-block
 // parts, i.e. what purekv_lowlayer_score keeps in its workspace.  It lives in the library's device image, so every GPU that
-// loads the library holds these 256 KiB until the process exits.  Host code may not pass this name to
+// loads the library holds this 1 MiB until the process exits.  Host code may not pass this name to
 // a kernel (on the host it is only a stand-in for the symbol); the device address comes from
 // cudaGetSymbolAddress, looked up once per device.
 constexpr size_t kNoallocScoreFloats = PUREKV_NOALLOC_SCORE_MAX_ROWS;
@@ -496,8 +496,16 @@ static purekv_status launch_score_mma(const void* q, const void* k, float* c_out
   // the pairs start on a 256-byte boundary behind the log-sum-exp values
   float2* partial = reinterpret_cast<float2*>(ws_f + (((int64_t)b->n_req * H * window + 63) & ~(int64_t)63));  // [n_req][Hkv][n_kb][rows_max]
   const size_t smem = (size_t)(kCtaKeys + 2 * kMmaRows) * (d + 8) * sizeof(__nv_bfloat16);  // K block + two Q blocks
-  PK_CUDA(cudaFuncSetAttribute(score_mma_partial_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  PK_CUDA(cudaFuncSetAttribute(score_mma_colsum_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  {
+    static std::atomic<uint64_t> smem_allowed{0};
+    const purekv_status st_smem = allow_max_dynamic_smem(score_mma_partial_kernel, smem_allowed);
+    if (st_smem != PUREKV_OK) return st_smem;
+  }
+  {
+    static std::atomic<uint64_t> smem_allowed{0};
+    const purekv_status st_smem = allow_max_dynamic_smem(score_mma_colsum_kernel, smem_allowed);
+    if (st_smem != PUREKV_OK) return st_smem;
+  }
   const float scale_log2 = scale * 1.4426950408889634f;
   dim3 grid((unsigned)((ml + kCtaKeys - 1) / kCtaKeys), (unsigned)Hkv, (unsigned)b->n_req);
   score_mma_partial_kernel<<<grid, kMmaThreads, smem, sm>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, b->cu_seqlens,
@@ -520,8 +528,16 @@ static purekv_status launch_score(const void* q, const void* k, float* c_out, co
   const int32_t w = std::min(window, ml);
   const int32_t G = H / Hkv;
   const size_t smem = (size_t)(kRB + kKB) * (d + 4) * sizeof(float);
-  PK_CUDA(cudaFuncSetAttribute(score_lse_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  PK_CUDA(cudaFuncSetAttribute(score_colsum_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  {
+    static std::atomic<uint64_t> smem_allowed{0};
+    const purekv_status st_smem = allow_max_dynamic_smem(score_lse_kernel<T>, smem_allowed);
+    if (st_smem != PUREKV_OK) return st_smem;
+  }
+  {
+    static std::atomic<uint64_t> smem_allowed{0};
+    const purekv_status st_smem = allow_max_dynamic_smem(score_colsum_kernel<T>, smem_allowed);
+    if (st_smem != PUREKV_OK) return st_smem;
+  }
   const float scale_log2 = scale * 1.4426950408889634f;
   dim3 g1((unsigned)((G * w + kRB - 1) / kRB), (unsigned)Hkv, (unsigned)b->n_req);
   score_lse_kernel<T><<<g1, kThreads, smem, sm>>>((const T*)q, (const T*)k, b->cu_seqlens, window, H, Hkv, d, scale_log2,
@@ -599,6 +615,7 @@ extern "C" purekv_status purekv_lowlayer_score_noalloc(const void* q, const void
                                                        float softmax_scale, void* stream) {
   purekv_status st = check_batch(batch, true);
   if (st != PUREKV_OK) return st;
+  if (batch->total_tokens == 0 || batch->n_req == 0) return PUREKV_OK;  // empty batch: nothing to do
   PK_REQUIRE(window >= 1 && n_q_heads >= 1, PUREKV_ERR_INVALID_ARG, "window and n_q_heads must be >= 1");
   const size_t need = (purekv_score_ws_bytes(batch, window, n_q_heads) - 256) / sizeof(float);
   PK_REQUIRE(need <= kNoallocScoreFloats, PUREKV_ERR_WORKSPACE,
