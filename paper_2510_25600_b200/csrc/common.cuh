@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdarg>
 #include <cstdint>
 #include <cstdio>
@@ -34,6 +35,29 @@ void set_error(const char* fmt, ...);
   } while (0)
 
 purekv_status check_batch(const purekv_batch* b, bool need_device);
+uint64_t wait_limit_ns();  // the process-wide limit of device-side waits (purekv_set_wait_limit_ns)
+
+// The status word a call uses when the caller passes none: one word per device inside the library, read and
+// cleared by purekv_poll_status(NULL, ...).  Its device address is looked up once per device.
+purekv_status default_status_word(int32_t** out);
+
+// Raises a kernel's dynamic shared-memory limit to what the device's opt-in maximum leaves, once per (kernel, device): `done`
+// is a bit mask over device ordinals that the call site keeps in a function-local static.  Launches then pass
+// whatever size they need; setting the attribute on every call would cost a driver call per launch.
+template <typename Kernel>
+purekv_status allow_max_dynamic_smem(Kernel kernel, std::atomic<uint64_t>& done) {
+  int dev = -1;
+  PK_CUDA(cudaGetDevice(&dev));
+  PK_REQUIRE(dev >= 0 && dev < 64, PUREKV_ERR_UNSUPPORTED, "device ordinal %d is beyond 63", dev);
+  if (done.load(std::memory_order_acquire) & (1ull << dev)) return PUREKV_OK;
+  int max_optin = 0;
+  PK_CUDA(cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+  cudaFuncAttributes fa;
+  PK_CUDA(cudaFuncGetAttributes(&fa, kernel));  // the opt-in maximum covers the kernel's static shared memory too
+  PK_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, max_optin - (int)fa.sharedSizeBytes));
+  done.fetch_or(1ull << dev, std::memory_order_release);
+  return PUREKV_OK;
+}
 
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
@@ -42,7 +66,7 @@ __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162flo
 // [PlanHeader][QTile x n_qtiles][order int32 x n_qtiles][entries int2 x n_entries][masks uint32 x n_mask_words]
 // [Unit x n_units][merge counters int32 x n_counters][scheduling counters int32 x 2]
 // all sections 16-byte aligned.  The last three sections exist only in plans for the tensor-core kernel.
-constexpr uint32_t kPlanMagic = 0x504B5634u;  // "PKV4"
+constexpr uint32_t kPlanMagic = 0x504B5635u;  // "PKV5"
 
 enum TileClass : int32_t { kTileFull = 0, kTileDiag = 1, kTileGeneral = 2 };
 
@@ -59,6 +83,9 @@ struct PlanHeader {
   int64_t off_units, off_counters;
   int32_t n_q_heads, n_kv_heads;
   int64_t part_slots;  // partial-result slots of the workspace (split chunks x query heads)
+  uint32_t test_flags;  // 0 in every plan the planner writes; bit 0 (set by a test in a host copy of a plan): the
+                        // producer withholds the first K copy, so that the bounded waits can be seen to expire
+  uint32_t pad_flags;
 };
 
 struct QTile {

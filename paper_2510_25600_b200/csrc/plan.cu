@@ -9,6 +9,7 @@
 // bits from the same intervals.  The kernels therefore never evaluate the mask's definition.
 #include <algorithm>
 #include <cstring>
+#include <mutex>
 #include <string>
 #include <queue>
 #include <vector>
@@ -18,6 +19,9 @@
 namespace purekv {
 
 static thread_local char g_err[512] = "";
+static std::atomic<uint64_t> g_wait_limit_ns{1000ull * 1000ull * 1000ull};
+
+uint64_t wait_limit_ns() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
 
 void set_error(const char* fmt, ...) {
   va_list ap;
@@ -76,13 +80,39 @@ static purekv_status check_params(const purekv_batch* b, const purekv_st_params*
 
 struct Span { int32_t a, b; };  // inclusive request-relative positions
 
+// The status word of calls made without one.  In host code this name is only a stand-in for the symbol: the device
+// address comes from cudaGetSymbolAddress, once per device.
+static __device__ int32_t g_default_status;
+
+purekv_status default_status_word(int32_t** out) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static int32_t* ptrs[kMaxDevices] = {};
+  int dev = -1;
+  PK_CUDA(cudaGetDevice(&dev));
+  PK_REQUIRE(dev >= 0 && dev < kMaxDevices, PUREKV_ERR_UNSUPPORTED, "device ordinal %d is beyond %d", dev, kMaxDevices);
+  std::lock_guard<std::mutex> lock(mu);
+  if (!ptrs[dev]) {
+    int32_t* p = nullptr;
+    PK_CUDA(cudaGetSymbolAddress((void**)&p, g_default_status));
+    PK_REQUIRE(p != nullptr, PUREKV_ERR_CUDA, "cudaGetSymbolAddress returned a null status address");
+    ptrs[dev] = p;
+  }
+  *out = ptrs[dev];
+  return PUREKV_OK;
+}
+
 }  // namespace purekv
 
 using namespace purekv;
 
 extern "C" {
 
-const char* purekv_version(void) { return "purekv-b200 0.1.0 (sm_100a)"; }
+const char* purekv_version(void) { return "purekv-b200 0.2.0 (sm_100a)"; }
+
+void purekv_set_wait_limit_ns(uint64_t ns) {
+  g_wait_limit_ns.store(ns ? ns : 1000ull * 1000ull * 1000ull, std::memory_order_relaxed);
+}
 
 void purekv_last_error(char* buf, size_t n) {
   if (!buf || n == 0) return;
@@ -455,8 +485,20 @@ purekv_status purekv_poll_status(const int32_t* status, int32_t* h_out, void* st
   cudaStream_t s = (cudaStream_t)stream;
   PK_CUDA(cudaStreamSynchronize(s));
   int32_t v = 0;
-  if (status) PK_CUDA(cudaMemcpy(&v, status, sizeof(v), cudaMemcpyDeviceToHost));
+  if (status) {
+    PK_CUDA(cudaMemcpy(&v, status, sizeof(v), cudaMemcpyDeviceToHost));
+  } else {
+    // the library's own word, used by calls made with status == NULL: report it and clear it, so that one expired
+    // wait does not block every later call of that kind
+    int32_t* own = nullptr;
+    purekv_status st = default_status_word(&own);
+    if (st != PUREKV_OK) return st;
+    PK_CUDA(cudaMemcpy(&v, own, sizeof(v), cudaMemcpyDeviceToHost));
+    if (v != 0) PK_CUDA(cudaMemset(own, 0, sizeof(v)));
+  }
   if (h_out) *h_out = v;
+  PK_REQUIRE(v != (int32_t)PUREKV_ERR_BAD_PLAN, PUREKV_ERR_BAD_PLAN,
+             "device status word is %d: a kernel refused the plan it was handed", v);
   PK_REQUIRE(v == 0, PUREKV_ERR_TIMEOUT, "device status word is %d: a bounded device-side wait expired", v);
   return PUREKV_OK;
 }

@@ -144,7 +144,11 @@ static purekv_status launch(const PrefillArgs& a) {
                        (size_t)kSimtWarps * a.info->tile_k) * sizeof(float);
   PK_REQUIRE(smem <= 227 * 1024, PUREKV_ERR_UNSUPPORTED,
              "head_dim %d with tile %d needs %zu bytes of shared memory", D, a.info->tile_k, smem);
-  PK_CUDA(cudaFuncSetAttribute(prefill_simt_kernel<T, DPL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  {
+    static std::atomic<uint64_t> smem_allowed{0};
+    const purekv_status st_smem = allow_max_dynamic_smem(prefill_simt_kernel<T, DPL>, smem_allowed);
+    if (st_smem != PUREKV_OK) return st_smem;
+  }
   dim3 grid((unsigned)a.info->n_qtiles, (unsigned)a.n_q_heads);
   prefill_simt_kernel<T, DPL><<<grid, kSimtThreads, smem, a.stream>>>(
       (const T*)a.q, (const T*)a.k, (const T*)a.v, (T*)a.o, a.lse, (const uint8_t*)a.plan, a.n_q_heads, a.n_kv_heads,

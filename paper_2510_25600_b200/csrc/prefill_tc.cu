@@ -71,7 +71,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_k64,
     const __grid_constant__ CUtensorMap tm_v64, __nv_bfloat16* __restrict__ o, float* __restrict__ lse,
     uint8_t* __restrict__ plan, float* __restrict__ ws, int32_t n_q_heads, int32_t n_kv_heads, float scale_log2,
-    int32_t* __restrict__ status) {
+    int32_t* __restrict__ status, uint64_t wait_ns, int64_t plan_bytes, int64_t ws_floats) {
   constexpr int ST = Cfg<BK>::kStages, SB = Cfg<BK>::kSBuf, MR = Cfg<BK>::kMeta;
   constexpr uint32_t kPanelQ = kBQ * 128;  // bytes of one 64-column panel of a Q tile
   constexpr uint32_t kTileQ = 2 * kPanelQ;
@@ -84,6 +84,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
   __shared__ Unit unit_s[kUnitRing];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
+  __shared__ int abort_code_s;  // what the status word becomes if the CTA gives up: an expired wait unless set otherwise
   __shared__ int merge_s[2];
 
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -130,23 +131,53 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     tmem_relinquish();
   }
   asm volatile("griddepcontrol.wait;" ::: "memory");  // the stream's earlier work is complete and visible from here on
-  if (tid == 0) abort_s = *reinterpret_cast<volatile int32_t*>(status) != 0;  // an earlier CTA or launch already failed
+  if (tid == 0) {
+    abort_s = *reinterpret_cast<volatile int32_t*>(status) != 0;  // an earlier CTA or launch already failed
+    abort_code_s = (int)PUREKV_ERR_TIMEOUT;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
   const PlanHeader* hdr = reinterpret_cast<const PlanHeader*>(plan);
-  const int2* entries = reinterpret_cast<const int2*>(plan + hdr->off_entries);
-  const uint32_t* masks = reinterpret_cast<const uint32_t*>(plan + hdr->off_masks);
-  const Unit* units = reinterpret_cast<const Unit*>(plan + hdr->off_units);
-  int32_t* counters = reinterpret_cast<int32_t*>(plan + hdr->off_counters);
+  // The plan is checked before anything is read through it: the header's own fields here (by every thread, on the
+  // same values, so the decision is uniform), each unit and each list entry by the producer before it publishes or
+  // uses them.  A plan that fails is not used: the status word becomes PUREKV_ERR_BAD_PLAN and the CTA leaves.
+  bool plan_ok = plan_bytes >= (int64_t)sizeof(PlanHeader);
+  if (plan_ok) {
+    const int64_t G_ = n_kv_heads > 0 ? n_q_heads / n_kv_heads : 0;
+    auto section = [&](int64_t off, int64_t count, int64_t elem) {
+      return off >= (int64_t)sizeof(PlanHeader) && (off & 15) == 0 && count >= 0 && count <= plan_bytes / elem &&
+             off <= plan_bytes - count * elem;
+    };
+    plan_ok = hdr->magic == kPlanMagic && hdr->tile_q == kBQ && hdr->tile_k == BK && hdr->words_per_row == BK / 32 &&
+              hdr->n_q_heads == n_q_heads && hdr->n_kv_heads == n_kv_heads && G_ >= 1 &&
+              hdr->n_ctas == (int32_t)gridDim.x && hdr->n_units >= 1 && hdr->n_counters >= 0 &&
+              section(hdr->off_entries, hdr->n_entries, 8) && section(hdr->off_masks, hdr->n_mask_words, 4) &&
+              section(hdr->off_units, hdr->n_units, (int64_t)sizeof(Unit)) &&
+              section(hdr->off_counters, (int64_t)hdr->n_counters + 2, 4) && hdr->part_slots >= 0 &&
+              hdr->part_slots <= ws_floats / kPartFloats && hdr->total_tokens >= 0;
+  }
+  if (!plan_ok) {
+    if (tid == 0 && abort_s == 0) atomicExch(status, (int32_t)PUREKV_ERR_BAD_PLAN);
+    hdr = nullptr;
+  }
+  const int2* entries = reinterpret_cast<const int2*>(plan + (plan_ok ? hdr->off_entries : 0));
+  const uint32_t* masks = reinterpret_cast<const uint32_t*>(plan + (plan_ok ? hdr->off_masks : 0));
+  const Unit* units = reinterpret_cast<const Unit*>(plan + (plan_ok ? hdr->off_units : 0));
+  int32_t* counters = reinterpret_cast<int32_t*>(plan + (plan_ok ? hdr->off_counters : 0));
   const int32_t G = n_q_heads / n_kv_heads, ppg = (G + 1) >> 1;
   // Units are handed out at run time: CTA c starts with unit c of the list (sorted by decreasing cost) and draws
   // every further one from a counter behind the merge counters, so the CTAs finish within one small unit of one
   // another whatever the units really cost.  The producer draws and publishes; the other roles follow unit_s[].
-  const int32_t n_units = hdr->n_units;
-  int32_t* sched = counters + hdr->n_counters;  // [0] units drawn beyond the first round, [1] CTAs that drew their last
-  const bool start_ok = abort_s == 0;
+  const int32_t n_units = plan_ok ? hdr->n_units : 0;
+  int32_t* sched = counters + (plan_ok ? hdr->n_counters : 0);  // [0] units drawn beyond the first round, [1] CTAs that drew their last
+  const int64_t n_entries = plan_ok ? hdr->n_entries : 0, n_mask_words = plan_ok ? hdr->n_mask_words : 0;
+  const int64_t total_tokens = plan_ok ? hdr->total_tokens : 0;
+  const int32_t n_counters = plan_ok ? hdr->n_counters : 0;
+  const int64_t part_slots = plan_ok ? hdr->part_slots : 0;
+  const bool withhold_first_k = plan_ok && (hdr->test_flags & 1u) != 0u;
+  const bool start_ok = abort_s == 0 && plan_ok;
   // the two softmax warpgroups take registers from the warpgroup of the producer and MMA warps
 
   if (warp >= 8) {
@@ -157,15 +188,33 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     int32_t issued_k = 0, issued_v = 0;
     bool ok = true;
     // unit idx of the list, or the end mark (ent_count 0) past its end
+    // Also checks the unit: a unit whose fields point outside the plan's sections, the batch or the workspace is not
+    // published; the CTA gives up with PUREKV_ERR_BAD_PLAN instead.
     auto fetch = [&](int32_t idx) -> Unit {
       Unit uu = {};
-      if (idx < n_units) uu = units[idx];
+      if (idx < n_units) {
+        uu = units[idx];
+        const int32_t n_pairs = n_kv_heads * ppg;
+        const bool split = uu.n_chunks > 1;
+        const bool good = uu.ent_count >= 1 && uu.ent_begin >= 0 && (int64_t)uu.ent_begin + uu.ent_count <= n_entries &&
+                          uu.q_rows >= 1 && uu.q_rows <= kBQ && uu.req_start >= 0 && uu.q_start >= uu.req_start &&
+                          (int64_t)uu.q_start + uu.q_rows <= total_tokens && uu.pair >= 0 && uu.pair < n_pairs &&
+                          uu.n_chunks >= 1 && uu.chunk >= 0 && uu.chunk < uu.n_chunks &&
+                          (!split || (uu.part_base >= 0 && ((int64_t)uu.part_base + uu.n_chunks) * n_q_heads <= part_slots &&
+                                      uu.counter_base >= 0 && (int64_t)uu.counter_base + n_q_heads <= n_counters));
+        if (!good) {
+          abort_code_s = (int)PUREKV_ERR_BAD_PLAN;
+          *abort_flag = 1;
+          uu = Unit{};
+        }
+      }
       return uu;
     };
     // lane 0: put a fetched unit into the ring as the CTA's unit number uo
     auto publish = [&](const Unit& uu, uint32_t uo) -> bool {
+      if (*abort_flag) return false;
       const uint32_t us = uo % kUnitRing;
-      if (uo >= (uint32_t)kUnitRing && !mbar_wait(smem_u32(&bars.u_empty[us]), ((uo / kUnitRing) - 1u) & 1u, abort_flag))
+      if (uo >= (uint32_t)kUnitRing && !mbar_wait(smem_u32(&bars.u_empty[us]), ((uo / kUnitRing) - 1u) & 1u, abort_flag, wait_ns))
         return false;
       unit_s[us] = uu;
       mbar_arrive(smem_u32(&bars.u_full[us]));
@@ -196,7 +245,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       const int32_t g = u.pair / ppg, hq0 = g * G + 2 * (u.pair % ppg);
       const int32_t n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
       if (lane == 0) {
-        if (uo > 0) ok = mbar_wait(smem_u32(&bars.q_empty), (uo - 1u) & 1u, abort_flag);
+        if (uo > 0) ok = mbar_wait(smem_u32(&bars.q_empty), (uo - 1u) & 1u, abort_flag, wait_ns);
         if (ok) {
           mbar_expect_tx(smem_u32(&bars.q_full), n_slots * kTileQ);
           for (int sl = 0; sl < n_slots; ++sl) {
@@ -219,7 +268,14 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
             const uint32_t s = it % ST, par = ((it / ST) - 1u) & 1u, ms = it % MR;
             const int32_t tok = u.req_start + (e.x >> 4) * BK;
             const uint32_t hm = (uint32_t)(e.x >> 2) & 3u;  // which 64-key halves of the tile are present
-            if (it >= (uint32_t)ST) ok = mbar_wait(smem_u32(&bars.k_empty[s]), par, abort_flag);
+            // the entry is checked before its mask offset or key-tile index is used for a copy
+            if (e.x < 0 || hm == 0u || (e.x & 3) > kTileGeneral || (int64_t)tok >= total_tokens ||
+                ((e.x & 3) == kTileGeneral && (e.y < 0 || (int64_t)e.y + (int64_t)(kMaskBytes / 4) > n_mask_words || (e.y & 3) != 0))) {
+              abort_code_s = (int)PUREKV_ERR_BAD_PLAN;
+              *abort_flag = 1;
+              ok = false;
+            }
+            if (ok && it >= (uint32_t)ST) ok = mbar_wait(smem_u32(&bars.k_empty[s]), par, abort_flag, wait_ns);
             if (ok) {
               meta_s[ms] = e;
               if ((e.x & 3) == kTileGeneral) {
@@ -228,7 +284,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
               } else {
                 mbar_arrive(smem_u32(&bars.m_full[ms]));
               }
-              if (hm == 3u) {
+              if (withhold_first_k && it == 0u) {
+                // test plans only: this tile's K is never asked for, so whoever waits for it runs into the limit
+              } else if (hm == 3u) {
                 mbar_expect_tx(smem_u32(&bars.k_full[s]), kTileKV);
                 tma_load_3d(sK + s * kTileKV, &tm_k, smem_u32(&bars.k_full[s]), 0, g, tok);
                 tma_load_3d(sK + s * kTileKV + kPanelKV, &tm_k, smem_u32(&bars.k_full[s]), 64, g, tok);
@@ -239,8 +297,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
                 tma_load_3d(sK + s * kTileKV + kPanelKV + off, &tm_k64, smem_u32(&bars.k_full[s]), 64, g,
                             tok + 64 * (int32_t)hh);
               }
-              issued_k = (int32_t)it + 1;
-              if (it >= (uint32_t)ST) ok = mbar_wait(smem_u32(&bars.v_empty[s]), par, abort_flag);
+              if (!(withhold_first_k && it == 0u)) issued_k = (int32_t)it + 1;
+              if (it >= (uint32_t)ST) ok = mbar_wait(smem_u32(&bars.v_empty[s]), par, abort_flag, wait_ns);
             }
             if (ok) {
               if (hm == 3u) {
@@ -267,11 +325,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       // drain: every issued copy must have landed before shared memory is released
       const uint64_t t0 = global_ns();
       for (int32_t n = max(0, issued_k - ST); n < issued_k; ++n)
-        while (!mbar_try_wait(smem_u32(&bars.k_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(smem_u32(&bars.k_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < wait_ns) {}
       for (int32_t n = max(0, issued_v - ST); n < issued_v; ++n)
-        while (!mbar_try_wait(smem_u32(&bars.v_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(smem_u32(&bars.v_full[n % ST]), (n / ST) & 1) && global_ns() - t0 < wait_ns) {}
       for (int32_t n = max(0, issued_k - MR); n < issued_k; ++n)
-        while (!mbar_try_wait(smem_u32(&bars.m_full[n % MR]), (n / MR) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(smem_u32(&bars.m_full[n % MR]), (n / MR) & 1) && global_ns() - t0 < wait_ns) {}
       __nanosleep(20000);  // a Q tile possibly still in flight (its barrier's phase is not known here)
     }
   } else if (start_ok && warp == kWarpMma) {
@@ -284,6 +342,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       uint32_t tq[2] = {0, 0};         // S products issued per slot, over all units
       uint32_t tp[2] = {0, 0};         // P.V products issued per slot, over all units
       int32_t nt = 0, n_slots = 0;
+      int32_t pend_v = -1;             // V stage whose release is due behind the next S product
       // Descriptor words.  High word: stride between 8-row groups 1024 B, descriptor version 1, 128-byte swizzle.
       // Low word: start address / 16 and the leading-dimension offset / 16 (used by the MN-major V operand only).
       constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
@@ -296,7 +355,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         const uint32_t it = it_base + (uint32_t)n;
         const uint32_t s = it % ST, b = tq[sl] % SB;
         // the stage was already awaited for slot 0 of the same tile
-        if (sl == 0 && !mbar_wait(smem_u32(&bars.k_full[s]), (it / ST) & 1u, abort_flag)) return false;
+        if (sl == 0 && !mbar_wait(smem_u32(&bars.k_full[s]), (it / ST) & 1u, abort_flag, wait_ns)) return false;
         tc_fence_after();
         const uint32_t hm = (uint32_t)(meta_s[it % MR].x >> 2) & 3u;  // written before the stage's barrier was armed
         const uint32_t q_lo = q_lo0 + (uint32_t)sl * (kTileQ >> 4);
@@ -315,11 +374,18 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
             mma_ss_lh(d_addr, q_lo + (ks >> 2) * (kPanelQ >> 4) + (ks & 3) * 2, kDescHi,
                       k_lo + (ks >> 2) * (kPanelKV >> 4) + (ks & 3) * 2, kDescHi, idesc_qk_half, ks > 0 ? 1u : 0u);
         }
+        // A commit costs the issuing thread about as long as a product and the slot's rows are waiting for S, so S
+        // is announced first; the releases behind it (and the V release a preceding P.V left pending) cover the
+        // same products and only reach the producer a little later.
+        tc_commit(smem_u32(&bars.s_full[sl][b]));
+        if (pend_v >= 0) {
+          tc_commit(smem_u32(&bars.v_empty[pend_v]));
+          pend_v = -1;
+        }
         if (sl == n_slots - 1) {
           tc_commit(smem_u32(&bars.k_empty[s]));
           if (n == nt - 1) tc_commit(smem_u32(&bars.q_empty));  // the unit's last read of Q
         }
-        tc_commit(smem_u32(&bars.s_full[sl][b]));
         ++tq[sl];
         return true;
       };
@@ -328,9 +394,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         constexpr int sl = decltype(sl_c)::value;
         const uint32_t it = it_base + (uint32_t)n;
         const uint32_t s = it % ST, b = tp[sl] % SB;
-        if (sl == 0 && !mbar_wait(smem_u32(&bars.v_full[s]), (it / ST) & 1u, abort_flag)) return false;
+        if (sl == 0 && !mbar_wait(smem_u32(&bars.v_full[s]), (it / ST) & 1u, abort_flag, wait_ns)) return false;
         // P of the unit's first tile also implies that the previous unit's output has left TMEM
-        if (!mbar_wait(smem_u32(&bars.p_full[sl][b]), (tp[sl] / SB) & 1u, abort_flag)) return false;
+        if (!mbar_wait(smem_u32(&bars.p_full[sl][b]), (tp[sl] / SB) & 1u, abort_flag, wait_ns)) return false;
         tc_fence_after();
         const uint32_t p_addr = tmem + sl * 128 + b * BK, o_addr = tmem + kColO + sl * 128;
         // B = V tile, MN-major: per K step 16 key rows (2 groups of 8, 1024 B apart) x 128 dims (2 panels)
@@ -347,22 +413,26 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
           for (int ks = 0; ks < BK / 32; ++ks)
             mma_ts_lh(o_addr, p_addr + (k0 + ks) * 8, v_lo + (k0 + ks) * (2048 >> 4), kDescHi, idesc_pv, ks > 0 ? 1u : acc0);
         }
-        if (sl == n_slots - 1) tc_commit(smem_u32(&bars.v_empty[s]));
         if (SB > 1) tc_commit(smem_u32(&bars.o_done[sl]));
         if (n == nt - 1) tc_commit(smem_u32(&bars.o_final[sl]));
+        if (sl == n_slots - 1) {
+          // the V stage is released behind the S product that follows, if one does (see issue_qk)
+          if (n + SB < nt) pend_v = (int32_t)s;
+          else tc_commit(smem_u32(&bars.v_empty[s]));
+        }
         ++tp[sl];
         return true;
       };
       bool ok = true;
       for (uint32_t uo = 0; ok; ++uo) {
         const uint32_t us = uo % kUnitRing;
-        if (!mbar_wait(smem_u32(&bars.u_full[us]), (uo / kUnitRing) & 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(smem_u32(&bars.u_full[us]), (uo / kUnitRing) & 1u, abort_flag, wait_ns)) { ok = false; break; }
         const Unit u = unit_s[us];
         mbar_arrive(smem_u32(&bars.u_empty[us]));
         if (u.ent_count == 0) break;
         nt = u.ent_count;
         n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
-        ok = mbar_wait(smem_u32(&bars.q_full), uo & 1u, abort_flag);
+        ok = mbar_wait(smem_u32(&bars.q_full), uo & 1u, abort_flag, wait_ns);
         constexpr std::integral_constant<int, 0> s0{};
         constexpr std::integral_constant<int, 1> s1{};
         for (int32_t n = 0; ok && n < SB && n < nt; ++n) {
@@ -383,7 +453,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         // leaving early: let every issued MMA finish before TMEM is released
         tc_commit(smem_u32(&bars.drain));
         const uint64_t t0 = global_ns();
-        while (!mbar_try_wait(smem_u32(&bars.drain), 0) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(smem_u32(&bars.drain), 0) && global_ns() - t0 < wait_ns) {}
       }
     }
   }
@@ -397,7 +467,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
     // waits are made warp-uniform: the TMEM loads/stores below need the whole warp
     auto wait_w = [&](uint32_t bar, uint32_t parity) -> bool {
-      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, wait_ns) ? 1 : 0) != 0;
     };
     uint32_t it_base = 0;     // key tiles of earlier units (both slots)
     uint32_t t = 0;           // tiles this slot has processed, over all units
@@ -617,7 +687,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
           }
         }
         if (lse && row_valid)
-          lse[(int64_t)hq * hdr->total_tokens + u.q_start + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+          lse[(int64_t)hq * total_tokens + u.q_start + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
       } else {
         // one chunk of a split list: leave the unnormalised result for whoever arrives last
         float* part = ws + ((int64_t)(u.part_base + u.chunk) * n_q_heads + hq) * kPartFloats;
@@ -693,7 +763,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
             }
           }
           if (lse && row_valid)
-            lse[(int64_t)hq * hdr->total_tokens + u.q_start + row] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+            lse[(int64_t)hq * total_tokens + u.q_start + row] = (m_all + log2f(l_all)) * 0.6931471805599453f;
         }
       }
       release_unit();
@@ -707,25 +777,29 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
-  if (tid == 0 && abort_s && start_ok) atomicExch(status, (int32_t)PUREKV_ERR_TIMEOUT);
+  if (tid == 0 && abort_s && start_ok) atomicCAS(status, 0, (int32_t)abort_code_s);  // the first code raised stays
 }
-
-__device__ int32_t g_default_status;
 
 static purekv_status launch(const PrefillArgs& a, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                             const CUtensorMap& mk64, const CUtensorMap& mv64, int32_t* status) {
   constexpr int BK = 128;
   const size_t smem = 1024 + 2 * 2 * (size_t)kBQ * 128 + 2 * (size_t)Cfg<BK>::kStages * 2 * BK * 128 +
                       (size_t)Cfg<BK>::kMeta * Cfg<BK>::kMaskBytes;
-  static int launch_regs = 0;
-  if (launch_regs == 0) {
+  static std::atomic<int> launch_regs{0};  // the compiled register count: the same on every device, read once
+  int regs = launch_regs.load(std::memory_order_relaxed);
+  if (regs == 0) {
     cudaFuncAttributes fa;
     PK_CUDA(cudaFuncGetAttributes(&fa, prefill_tc_kernel<BK>));
-    launch_regs = fa.numRegs;
+    regs = fa.numRegs;
+    launch_regs.store(regs, std::memory_order_relaxed);
   }
-  PK_REQUIRE(256 * kRegsSoftmax + 128 * kRegsOther <= kThreads * launch_regs, PUREKV_ERR_UNSUPPORTED,
-             "prefill kernel was compiled with %d registers per thread, too few for its register hand-over", launch_regs);
-  PK_CUDA(cudaFuncSetAttribute(prefill_tc_kernel<BK>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  PK_REQUIRE(256 * kRegsSoftmax + 128 * kRegsOther <= kThreads * regs, PUREKV_ERR_UNSUPPORTED,
+             "prefill kernel was compiled with %d registers per thread, too few for its register hand-over", regs);
+  {
+    static std::atomic<uint64_t> smem_allowed{0};
+    const purekv_status st_smem = allow_max_dynamic_smem(prefill_tc_kernel<BK>, smem_allowed);
+    if (st_smem != PUREKV_OK) return st_smem;
+  }
   dim3 grid((unsigned)a.info->n_ctas);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
@@ -739,7 +813,8 @@ static purekv_status launch(const PrefillArgs& a, const CUtensorMap& mq, const C
   cfg.numAttrs = 1;
   PK_CUDA(cudaLaunchKernelEx(&cfg, prefill_tc_kernel<BK>, mq, mk, mv, mk64, mv64, (__nv_bfloat16*)a.o, a.lse,
                              (uint8_t*)a.plan, (float*)a.ws, a.n_q_heads, a.n_kv_heads,
-                             a.scale * 1.4426950408889634f, status));
+                             a.scale * 1.4426950408889634f, status, wait_limit_ns(), (int64_t)a.info->bytes_used,
+                             (int64_t)(a.ws_bytes / sizeof(float))));
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
 }
@@ -761,7 +836,10 @@ purekv_status launch_prefill_tc(const PrefillArgs& a) {
   if ((st = make_map(&mk64, a.k, T, a.n_kv_heads, 64)) != PUREKV_OK) return st;
   if ((st = make_map(&mv64, a.v, T, a.n_kv_heads, 64)) != PUREKV_OK) return st;
   int32_t* status = a.status;
-  if (!status) PK_CUDA(cudaGetSymbolAddress((void**)&status, g_default_status));
+  if (!status) {
+    const purekv_status st_w = default_status_word(&status);
+    if (st_w != PUREKV_OK) return st_w;
+  }
   return launch(a, mq, mk, mv, mk64, mv64, status);
 }
 

@@ -35,7 +35,7 @@ struct __align__(8) Barriers {
 __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
     const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q8, const float* __restrict__ lse,
     float* __restrict__ c_out, const int32_t* __restrict__ cu_seqlens, int32_t window, int32_t n_q_heads,
-    int32_t n_kv_heads, float scale_log2, int64_t n_tokens, int32_t* __restrict__ status) {
+    int32_t n_kv_heads, float scale_log2, int64_t n_tokens, int32_t* __restrict__ status, uint64_t wait_ns) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ Barriers bars;
   __shared__ uint32_t tmem_base_s;
@@ -92,7 +92,7 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
       int32_t issued = 0;
       for (int32_t t = 0; t < n_blocks; ++t) {
         const int32_t s = t % kStages;
-        if (t >= kStages && !mbar_wait(smem_u32(&bars.q_empty[s]), ((t / kStages) - 1) & 1, abort_flag)) break;
+        if (t >= kStages && !mbar_wait(smem_u32(&bars.q_empty[s]), ((t / kStages) - 1) & 1, abort_flag, wait_ns)) break;
         mbar_expect_tx(smem_u32(&bars.q_full[s]), kTile);
         for (int32_t grp = 0; grp < kRows / 8; ++grp) {
           const int32_t row = t * kRows + 8 * grp;
@@ -110,9 +110,9 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
       }
       if (*abort_flag) {  // every issued copy must have landed before shared memory is released
         const uint64_t t0 = global_ns();
-        while (!mbar_try_wait(smem_u32(&bars.k_full), 0) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(smem_u32(&bars.k_full), 0) && global_ns() - t0 < wait_ns) {}
         for (int32_t t = max(0, issued - kStages); t < issued; ++t)
-          while (!mbar_try_wait(smem_u32(&bars.q_full[t % kStages]), (t / kStages) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+          while (!mbar_try_wait(smem_u32(&bars.q_full[t % kStages]), (t / kStages) & 1) && global_ns() - t0 < wait_ns) {}
       }
     }
   } else if (start_ok && warp == 1) {
@@ -122,11 +122,11 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
       constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
       const uint32_t k_lo0 = ((sK & 0x3FFFFu) >> 4) | (1u << 16);
       const uint32_t q_lo0 = ((sQ & 0x3FFFFu) >> 4) | (1u << 16);
-      bool ok = mbar_wait(smem_u32(&bars.k_full), 0, abort_flag);
+      bool ok = mbar_wait(smem_u32(&bars.k_full), 0, abort_flag, wait_ns);
       for (int32_t t = 0; ok && t < n_blocks; ++t) {
         const int32_t s = t % kStages, b = t & 1;
-        ok = mbar_wait(smem_u32(&bars.q_full[s]), (t / kStages) & 1, abort_flag);
-        if (ok && t >= 2) ok = mbar_wait(smem_u32(&bars.d_empty[b]), ((t >> 1) - 1) & 1, abort_flag);
+        ok = mbar_wait(smem_u32(&bars.q_full[s]), (t / kStages) & 1, abort_flag, wait_ns);
+        if (ok && t >= 2) ok = mbar_wait(smem_u32(&bars.d_empty[b]), ((t >> 1) - 1) & 1, abort_flag, wait_ns);
         if (!ok) break;
         tc_fence_after();
         const uint32_t q_lo = q_lo0 + s * (kTile >> 4);
@@ -140,7 +140,7 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
       if (!ok) {  // leaving early: let every issued MMA finish before TMEM is released
         tc_commit(smem_u32(&bars.drain));
         const uint64_t t0 = global_ns();
-        while (!mbar_try_wait(smem_u32(&bars.drain), 0) && global_ns() - t0 < kWaitLimitNs) {}
+        while (!mbar_try_wait(smem_u32(&bars.drain), 0) && global_ns() - t0 < wait_ns) {}
       }
     }
   } else if (start_ok && warp >= 2) {
@@ -162,7 +162,7 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
         if (row < n_rows)
           lv[c] = __ldg(lse + (int64_t)(g * G + row / w) * n_tokens + base + len - w + row % w) * kLog2e;
       }
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.d_full[b]), (t >> 1) & 1, abort_flag) ? 1 : 0) != 0;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.d_full[b]), (t >> 1) & 1, abort_flag, wait_ns) ? 1 : 0) != 0;
       if (!ok) break;
       tc_fence_after();
 #pragma unroll
@@ -195,7 +195,6 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
   if (tid == 0 && abort_s && start_ok) atomicExch(status, (int32_t)PUREKV_ERR_TIMEOUT);
 }
 
-__device__ int32_t g_score_status;
 
 }  // namespace sc
 }  // namespace purekv
@@ -231,13 +230,20 @@ extern "C" purekv_status purekv_lowlayer_score_lse(const void* q, const void* k,
   CUtensorMap mk, mq8;
   if ((st = make_map(&mk, k, T, n_kv_heads, kKeys)) != PUREKV_OK) return st;
   if ((st = make_map(&mq8, q, T, n_q_heads, 8)) != PUREKV_OK) return st;
-  if (!status) PK_CUDA(cudaGetSymbolAddress((void**)&status, g_score_status));
+  if (!status) {
+    const purekv_status st_w = default_status_word(&status);
+    if (st_w != PUREKV_OK) return st_w;
+  }
   const size_t smem = 1024 + (size_t)(1 + kStages) * kTile;
-  PK_CUDA(cudaFuncSetAttribute(score_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  {
+    static std::atomic<uint64_t> smem_allowed{0};
+    const purekv_status st_smem = allow_max_dynamic_smem(score_tc_kernel, smem_allowed);
+    if (st_smem != PUREKV_OK) return st_smem;
+  }
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
   dim3 grid((unsigned)((ml + kKeys - 1) / kKeys), (unsigned)n_kv_heads, (unsigned)batch->n_req);
   score_tc_kernel<<<grid, kThreads, smem, (cudaStream_t)stream>>>(mk, mq8, lse, c_out, batch->cu_seqlens, window, n_q_heads,
-                                                                   n_kv_heads, scale * 1.4426950408889634f, T, status);
+                                                                   n_kv_heads, scale * 1.4426950408889634f, T, status, wait_limit_ns());
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
 }

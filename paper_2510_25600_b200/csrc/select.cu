@@ -350,12 +350,20 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
   const int64_t segments = (int64_t)batch->n_req * n_kv_heads * n_layers;
   if (cpr == 16 && key_bytes <= 200 * 1024 && segments >= 2 * 148) {
     if (dtype == PUREKV_BF16) {
-      PK_CUDA(cudaFuncSetAttribute(select_kernel<true, __nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
+      {
+        static std::atomic<uint64_t> smem_allowed{0};
+        const purekv_status st_smem = allow_max_dynamic_smem(select_kernel<true, __nv_bfloat16>, smem_allowed);
+        if (st_smem != PUREKV_OK) return st_smem;
+      }
       select_kernel<true, __nv_bfloat16><<<g2, kSelThreads, key_bytes, sm>>>(
           nullptr, T, batch->cu_seqlens, cu_kept, keep, window, k_tot, n_kv_heads, idx_out, (const uint4*)v,
           v_layer_stride * esz / 16, c, s_out);
     } else {
-      PK_CUDA(cudaFuncSetAttribute(select_kernel<true, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
+      {
+        static std::atomic<uint64_t> smem_allowed{0};
+        const purekv_status st_smem = allow_max_dynamic_smem(select_kernel<true, float>, smem_allowed);
+        if (st_smem != PUREKV_OK) return st_smem;
+      }
       select_kernel<true, float><<<g2, kSelThreads, key_bytes, sm>>>(nullptr, T, batch->cu_seqlens, cu_kept, keep, window,
                                                                      k_tot, n_kv_heads, idx_out, (const uint4*)v,
                                                                      v_layer_stride * esz / 16, c, s_out);
@@ -380,7 +388,11 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
   PK_CUDA(cudaGetLastError());
   const bool stage_keys = key_bytes <= 200 * 1024;
   if (stage_keys)
-    PK_CUDA(cudaFuncSetAttribute(select_kernel<false, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)key_bytes));
+    {
+      static std::atomic<uint64_t> smem_allowed{0};
+      const purekv_status st_smem = allow_max_dynamic_smem(select_kernel<false, float>, smem_allowed);
+      if (st_smem != PUREKV_OK) return st_smem;
+    }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = g2;
   cfg.blockDim = dim3(kSelThreads);

@@ -9,7 +9,6 @@ namespace purekv {
 namespace tc {
 
 constexpr int kD = 128;                                          // head dimension of the tensor-core kernels
-constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
 constexpr int kPolyOf8 = 0;  // of every 8 pairs of exponentials in the prefill, how many go to the FMA pipe
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -33,6 +32,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// Non-blocking test of a barrier phase (try_wait may suspend the thread for a while before it answers).
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ uint64_t global_ns() {
   uint64_t t;
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
@@ -40,7 +49,7 @@ __device__ __forceinline__ uint64_t global_ns() {
 }
 // Bounded wait: false if the abort flag is up or the time limit passed (then raises the flag).
 // The wall-clock timer is slow to read, so it is consulted only every 1024 failed polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_ns) {
   uint64_t t0 = 0;
   uint32_t it = 0;
   while (true) {
@@ -50,7 +59,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       const uint64_t now = global_ns();
       if (t0 == 0) {
         t0 = now;
-      } else if (now - t0 > kWaitLimitNs) {
+      } else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         return false;
       }

@@ -36,7 +36,7 @@ def parse_plan(buf: np.ndarray):
     raw = buf.tobytes()
     (magic, tq, tk, nq, T, ne, nm, oq, oo, oe, om, wpr, n_ctas, n_units, n_counters, o_units, o_counters, H, Hkv,
      part_slots) = struct.unpack_from("<Iiiiqqqqqqqiiiiqqiiq", raw, 0)
-    assert magic == 0x504B5634
+    assert magic == 0x504B5635
     qt = np.frombuffer(raw, dtype=np.int32, count=nq * 8, offset=oq).reshape(nq, 8)
     order = np.frombuffer(raw, dtype=np.int32, count=nq, offset=oo)
     entries = np.frombuffer(raw, dtype=np.int32, count=2 * ne, offset=oe).reshape(ne, 2)
