@@ -6,7 +6,9 @@
 // What each function follows:
 //   pko_mask           ST-SpAttn mask, Sec. 3.2 (spatial path: first frame + current
 //                      frame; temporal path: corresponding token of the previous frame
-//                      + first frame), under causal attention (Sec. 3.1/3.2).
+//                      + first frame), under causal attention (Sec. 3.1/3.2); the comparison
+//                      masks of App. A.3 / Table 7 (spatial only, temporal only, local,
+//                      atrous) and a block-level widening of any of them.
 //   pko_prefill        masked softmax attention; the softmax is Eq. 1 restricted to the
 //                      kept keys of each row.
 //   pko_lowlayer_score Eq. 1 (dense causal softmax rows) and Eq. 2 (sum of the recent
@@ -47,12 +49,17 @@ struct pko_mask_params {
   int32_t temporal_stride;  // linked frames are f-s, f-2s, ... (paper: 1)
   int32_t temporal_radius;  // 0: same grid cell only (paper); -1: whole linked frame
   int32_t dense_causal;     // nonzero: plain causal attention
+  // The comparison masks of App. A.3 / Table 7 (the paper names them and shows them only in a figure that the text
+  // does not reproduce; the readings are the usual meanings of the names):
+  int32_t local_window;     // > 0: Local Attention -- a visual query also sees the local_window most recent positions
+  int32_t atrous_dilation;  // > 0: Atrous Attention -- a visual query also sees every atrous_dilation-th earlier position
+  int32_t coarse_block;     // > 0: the mask is widened to blocks of this many positions (a block pair is kept whole,
+                            //      under causality, as soon as it holds one kept pair): block-sparse reading of the mask
 };
 
-// Sec. 3.2.  Positions are relative to the request; len = n_prefix + n_frames*N + n_suffix.
-// Returns 1 when query i may attend key j.
-int32_t pko_mask(const pko_mask_params* p, int32_t len, int32_t n_prefix, int32_t n_frames,
-                 int32_t i, int32_t j) {
+// The token-level predicate.  Sec. 3.2 for the spatial and temporal paths; App. A.3 names the other two.
+static int32_t mask_token(const pko_mask_params* p, int32_t len, int32_t n_prefix, int32_t n_frames, int32_t i,
+                          int32_t j) {
   if (i < 0 || j < 0 || i >= len || j >= len) return 0;
   if (j > i) return 0;                           // causal attention
   if (p->dense_causal) return 1;
@@ -77,6 +84,24 @@ int32_t pko_mask(const pko_mask_params* p, int32_t len, int32_t n_prefix, int32_
       (p->temporal_depth < 0 || df <= (int64_t)p->temporal_depth * p->temporal_stride) &&
       (p->temporal_radius < 0 || rho <= p->temporal_radius))
     return 1;
+  // (4) Local Attention: the most recent positions, whatever frame they belong to
+  if (p->local_window > 0 && i - j < p->local_window) return 1;
+  // (5) Atrous Attention: every dilation-th position counted back from the query
+  if (p->atrous_dilation > 0 && (i - j) % p->atrous_dilation == 0) return 1;
+  return 0;
+}
+
+// Positions are relative to the request; len = n_prefix + n_frames*N + n_suffix.
+// Returns 1 when query i may attend key j.
+int32_t pko_mask(const pko_mask_params* p, int32_t len, int32_t n_prefix, int32_t n_frames,
+                 int32_t i, int32_t j) {
+  if (p->coarse_block <= 0 || p->dense_causal) return mask_token(p, len, n_prefix, n_frames, i, j);
+  if (i < 0 || j < 0 || i >= len || j > i) return 0;
+  // block-level reading: (i, j) is kept if its block pair holds any kept pair of the token-level mask
+  const int32_t B = p->coarse_block, i0 = (i / B) * B, j0 = (j / B) * B;
+  for (int32_t ii = i0; ii < std::min(len, i0 + B); ++ii)
+    for (int32_t jj = j0; jj < std::min(len, j0 + B); ++jj)
+      if (mask_token(p, len, n_prefix, n_frames, ii, jj)) return 1;
   return 0;
 }
 

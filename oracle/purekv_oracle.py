@@ -28,13 +28,15 @@ def build(force: bool = False) -> str:
 class MaskParams(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("grid_h", "grid_w", "anchor_frames", "spatial_radius",
                                          "temporal_depth", "temporal_stride", "temporal_radius",
-                                         "dense_causal")]
+                                         "dense_causal", "local_window", "atrous_dilation", "coarse_block")]
 
 
 def mask_params(m) -> MaskParams:
     """From an inputs.STMask-like object (attribute access only)."""
     return MaskParams(m.grid_h, m.grid_w, m.anchor_frames, m.spatial_radius, m.temporal_depth,
-                      m.temporal_stride, m.temporal_radius, 1 if m.dense_causal else 0)
+                      m.temporal_stride, m.temporal_radius, 1 if m.dense_causal else 0,
+                      getattr(m, "local_window", 0), getattr(m, "atrous_dilation", 0),
+                      m.tile if getattr(m, "coarse", False) else 0)
 
 
 def lib():

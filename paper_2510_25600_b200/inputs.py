@@ -91,6 +91,30 @@ class STMask:
     temporal_radius: int = 0
     tile: int = 128
     dense_causal: bool = False
+    local_window: int = 0        # > 0: also the most recent positions (Local Attention of App. A.3)
+    atrous_dilation: int = 0     # > 0: also every n-th earlier position (Atrous Attention of App. A.3)
+    coarse: bool = False         # widen the mask to whole tile x tile blocks (block-sparse reading)
+
+
+def mask_variant(name: str, grid_h: int, grid_w: int, tile: int = 128, coarse: bool = False, local_window: int = 64,
+                 atrous_dilation: int = 4) -> STMask:
+    """The sparse-attention variants the paper compares (App. A.3, Table 7), as parameter settings:
+    "st" the paper's mask; "spatial" its spatial path alone (first frame + current frame); "temporal" its temporal
+    path alone (first frame + the same cell of the previous frame, and the token itself); "local" the most recent
+    `local_window` positions; "atrous" every `atrous_dilation`-th earlier position.  Prefix tokens stay visible and
+    text rows dense in all of them."""
+    kw = dict(tile=tile, coarse=coarse)
+    if name == "st":
+        return STMask(grid_h, grid_w, **kw)
+    if name == "spatial":
+        return STMask(grid_h, grid_w, 1, -1, 0, 1, 0, **kw)
+    if name == "temporal":
+        return STMask(grid_h, grid_w, 1, 0, 1, 1, 0, **kw)
+    if name == "local":
+        return STMask(grid_h, grid_w, 0, 0, 0, 1, 0, local_window=local_window, **kw)
+    if name == "atrous":
+        return STMask(grid_h, grid_w, 0, 0, 0, 1, 0, atrous_dilation=atrous_dilation, **kw)
+    raise ValueError(f"no mask variant {name!r}")
 
 
 @dataclasses.dataclass(frozen=True)

@@ -136,3 +136,100 @@ def test_budget_rule():
     assert po.budget(100, 32, 0.1) == (0, 32)        # budget below the window: window only
     assert po.budget(10, 32, 0.5) == (0, 10)         # window clipped to the sequence
     assert po.budget(50, 8, 1.0) == (42, 50)         # keep everything
+
+
+# ---- the comparison masks of App. A.3 / Table 7, each from its own sentence ------------------------------------------
+def variant_sentence_mask(name, n_prefix, n_frames, gh, gw, n_suffix, local_window=0, dilation=0):
+    """A second construction, by loops over (frame, cell): what each name keeps for a visual query; prefix keys
+    stay visible and text rows dense causal as in the paper's mask; everything causal."""
+    n = gh * gw
+    l = n_prefix + n_frames * n + n_suffix
+    m = np.zeros((l, l), dtype=bool)
+    pos = lambda f, c: n_prefix + f * n + c
+    for i in range(n_prefix):
+        m[i, :i + 1] = True
+    for f in range(n_frames):
+        for c in range(n):
+            i = pos(f, c)
+            m[i, :n_prefix] = True
+            m[i, i] = True
+            if name in ("spatial", "temporal"):
+                for c2 in range(n):
+                    m[i, pos(0, c2)] = True                    # the first frame anchors both paths
+            if name == "spatial":
+                for c2 in range(n):
+                    m[i, pos(f, c2)] = True                    # the current frame
+            if name == "temporal" and f >= 1:
+                m[i, pos(f - 1, c)] = True                     # the corresponding token of the previous frame
+            if name == "local":
+                for j in range(max(n_prefix, i - local_window + 1), i + 1):
+                    m[i, j] = True                             # the most recent positions
+            if name == "atrous":
+                for j in range(i, n_prefix - 1, -dilation):
+                    m[i, j] = True                             # every dilation-th position counted back
+    for i in range(n_prefix + n_frames * n, l):
+        m[i, :] = True
+    return m & np.tril(np.ones((l, l), dtype=bool))
+
+
+def variant_pairs(name, ns, F, N, nt, local_window=0, dilation=0):
+    """Kept pairs of a variant in closed form (prefix rows, visual rows frame by frame, suffix rows)."""
+    tri = lambda a: a * (a + 1) // 2
+    tot = tri(ns) + nt * (ns + F * N) + tri(nt)
+    for f in range(F):
+        if name == "spatial":        # prefix + first frame + causal part of the own frame (frame 0: the two coincide)
+            tot += N * ns + tri(N) + (N * N if f >= 1 else 0)
+        elif name == "temporal":     # prefix + first frame + previous cell + self (they coincide for f = 0 and f = 1)
+            tot += N * ns + (tri(N) if f == 0 else N * N + N * (1 if f == 1 else 2))
+        elif name == "local":        # prefix + the window clipped at the first visual position
+            tot += sum(ns + min(local_window, f * N + c + 1) for c in range(N))
+        elif name == "atrous":       # prefix + every dilation-th position back to the first visual one
+            tot += sum(ns + (f * N + c) // dilation + 1 for c in range(N))
+    return tot
+
+
+VARIANT_SHAPES = [(4, 5, 3, 4, 6), (0, 3, 2, 3, 5), (3, 1, 4, 4, 2), (2, 6, 1, 1, 0)]
+
+
+@pytest.mark.parametrize("ns,F,gh,gw,nt", VARIANT_SHAPES)
+@pytest.mark.parametrize("name,kw", [("spatial", {}), ("temporal", {}), ("local", dict(local_window=7)),
+                                     ("local", dict(local_window=1)), ("atrous", dict(atrous_dilation=3)),
+                                     ("atrous", dict(atrous_dilation=1))])
+def test_named_variants_match_their_sentences_and_pair_counts(name, kw, ns, F, gh, gw, nt):
+    m = inputs.mask_variant(name, gh, gw, **kw)
+    l = ns + F * gh * gw + nt
+    got = po.mask_matrix(po.mask_params(m), l, ns, F)
+    lw, dil = kw.get("local_window", 0), kw.get("atrous_dilation", 0)
+    assert np.array_equal(got, variant_sentence_mask(name, ns, F, gh, gw, nt, lw, dil))
+    assert int(got.sum()) == variant_pairs(name, ns, F, gh * gw, nt, lw, dil)
+    assert got.diagonal().all()
+
+
+def test_variants_relate_to_the_paper_mask_and_to_dense_attention():
+    ns, F, gh, gw, nt = 3, 5, 3, 4, 4
+    l = ns + F * gh * gw + nt
+    mat = lambda m: po.mask_matrix(po.mask_params(m), l, ns, F)
+    st, sp, tp = (mat(inputs.mask_variant(n, gh, gw)) for n in ("st", "spatial", "temporal"))
+    assert np.array_equal(st, sp | tp)                    # the paper's mask is the union of its two paths
+    tril = np.tril(np.ones((l, l), dtype=bool))
+    assert np.array_equal(mat(inputs.mask_variant("local", gh, gw, local_window=l)), tril)
+    assert np.array_equal(mat(inputs.mask_variant("atrous", gh, gw, atrous_dilation=1)), tril)
+    assert np.array_equal(mat(inputs.mask_variant("st", gh, gw)), mat(inputs.STMask(gh, gw)))
+
+
+@pytest.mark.parametrize("name,kw", [("st", {}), ("temporal", {}), ("local", dict(local_window=5)),
+                                     ("atrous", dict(atrous_dilation=7))])
+@pytest.mark.parametrize("block", [4, 16])
+def test_block_level_widening_keeps_whole_blocks_under_causality(name, kw, block):
+    """coarse: a block pair is kept whole (its causal part) exactly when the token-level mask keeps any pair in it."""
+    ns, F, gh, gw, nt = 5, 4, 3, 3, 7
+    l = ns + F * gh * gw + nt
+    fine = po.mask_matrix(po.mask_params(inputs.mask_variant(name, gh, gw, tile=block, **kw)), l, ns, F)
+    got = po.mask_matrix(po.mask_params(inputs.mask_variant(name, gh, gw, tile=block, coarse=True, **kw)), l, ns, F)
+    nb = (l + block - 1) // block
+    pad = np.zeros((nb * block, nb * block), dtype=bool)
+    pad[:l, :l] = fine
+    blocks = pad.reshape(nb, block, nb, block).any(axis=(1, 3))
+    want = np.repeat(np.repeat(blocks, block, axis=0), block, axis=1)[:l, :l] & np.tril(np.ones((l, l), dtype=bool))
+    assert np.array_equal(got, want)
+    assert (got | ~fine).all()                            # widening never drops a pair
