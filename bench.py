@@ -453,6 +453,38 @@ def compression_detail(pipe, wl, d_in, peaks, timer):
 
 
 # ---- side records of the other workloads (one GPU only) ----------------------------------------------------------
+def variant_rows(wl, q, k, v, db, names, reps, peaks, timer):
+    """One prefill layer under the sparse-attention variants the paper compares (App. A.3 / Table 7) and under
+    the block-level widening of the paper's mask: block density, time, TFLOP/s on issued blocks."""
+    import torch
+    from paper_2510_25600_b200 import binding as P, inputs
+    g = wl.batch.grid_h
+    tile = wl.mask.tile
+    spec = {"ST-SpAttn (paper)": ("st", {}), "ST-SpAttn widened to blocks": ("st", dict(coarse=True)),
+            "Spatial Sparse Attention": ("spatial", {}), "Temporal Sparse Attention": ("temporal", {}),
+            "Local Attention (256 positions)": ("local", dict(local_window=256)),
+            "Atrous Attention (every 4th position)": ("atrous", dict(atrous_dilation=4))}
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    o = torch.empty_like(q)
+    rows = []
+    for label in names:
+        name, kw = spec[label]
+        m = inputs.mask_variant(name, g, g, tile=tile, **kw)
+        plan = P.purekv_plan_build(db, P.st_params(m), P.BF16, wl.head_dim, wl.n_q_heads, wl.n_kv_heads)
+        ws = torch.empty(max(16, plan.info.ws_bytes), dtype=torch.uint8, device="cuda")
+        fn = lambda: P.purekv_st_sparse_prefill(q, k, v, db, plan, out=o, status=status, ws=ws)
+        for _ in range(3):
+            fn()
+        ms = timer(fn, reps)
+        info = plan.info
+        tf = 4.0 * info.tile_q * info.tile_k * wl.head_dim * wl.n_q_heads * info.tiles_kept / ms / 1e9
+        rows.append({"mask": label, "block_density": info.tiles_kept / info.tiles_causal,
+                     "pair_density": info.pairs_kept / (sum(int(l) * (int(l) + 1) // 2 for l in wl.batch.seq_lens)),
+                     "ms": ms, "TFLOPs": tf, "tokens_per_s": wl.batch.total_tokens / (ms * 1e-3), **tensor_fracs(tf, peaks)})
+    P.purekv_poll_status(status)
+    return rows
+
+
 def sub_pipeline(cfg, steps, peaks, timer):
     """A whole-pipeline workload (cfg 1) as a compact record: device-drawn inputs, its own clock samples."""
     import torch
@@ -467,7 +499,12 @@ def sub_pipeline(cfg, steps, peaks, timer):
     sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
     detail = compression_detail(pipe, wl, d_in, peaks, timer)
+    variants = variant_rows(wl, d_in[0][1], d_in[1][1], d_in[2][1], pipe.batch,
+                            ["ST-SpAttn (paper)", "ST-SpAttn widened to blocks", "Spatial Sparse Attention",
+                             "Temporal Sparse Attention", "Local Attention (256 positions)",
+                             "Atrous Attention (every 4th position)"], 5, peaks, timer)
     return {"config": config_dict(wl), "inputs": "N(0,1) bf16 drawn on the device (seeded); timing only",
+            "mask_variants": variants, "mask_variants_note": "one layer, kernel timed alone with cold L2; fractions in each row",
             "tokens_per_s": wl.batch.total_tokens / (ms_step * 1e-3), "ms_per_step": ms_step, "steps": steps, "clocks": clocks,
             "roofline": {k: roofline[k] for k in keep}, "steps_detail": detail, "steps_detail_clocks": sampler.stop()}
 
@@ -505,9 +542,11 @@ def sub_long_video(reps, peaks, timer):
         rows.append({"mask": name, "block_density": info.tiles_kept / info.tiles_causal, "ms": ms, "TFLOPs": tf,
                      "tokens_per_s": b.total_tokens / (ms * 1e-3), **tensor_fracs(tf, peaks)})
     P.purekv_poll_status(status)
+    variants = variant_rows(wl, q, k, v, db, ["ST-SpAttn widened to blocks", "Spatial Sparse Attention",
+                                              "Temporal Sparse Attention", "Local Attention (256 positions)"], reps, peaks, timer)
     clocks_prefill = sampler.stop()
     peak, which, why = pick_tensor_peak(peaks, clocks_prefill)
-    for r in rows:
+    for r in rows + variants:
         r["frac"] = r["TFLOPs"] / peak
     sampler = ClockSampler(torch.cuda.current_device())
     sampler.start()
@@ -542,7 +581,8 @@ def sub_long_video(reps, peaks, timer):
                      "compact": hbm_rec(t_cmp, by, peaks), "decode_step": hbm_rec(t_dec, 2 * bud.total_kept * row, peaks)})
     P.purekv_poll_status(status)
     return {"config": config_dict(wl), "inputs": "N(0,1) bf16 drawn on the device (seeded); timing only",
-            "prefill": rows, "prefill_peak": peak, "prefill_peak_kind": f"measured {which} ({why})", "prefill_clocks": clocks_prefill,
+            "prefill": rows, "mask_variants": variants, "prefill_peak": peak, "prefill_peak_kind": f"measured {which} ({why})",
+            "prefill_clocks": clocks_prefill,
             "score_one_pass": dict(hbm_rec(t_score_lse, bytes_score, peaks), TFLOPs=score_fl / t_score_lse / 1e9,
                                    frac_tensor_burst=score_fl / t_score_lse / 1e9 / float(peaks["bf16_tflops"])),
             "score_two_pass": dict(hbm_rec(t_score_2p, bytes_score, peaks), TFLOPs=2 * score_fl / t_score_2p / 1e9),

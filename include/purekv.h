@@ -45,13 +45,24 @@ typedef enum {
 typedef enum { PUREKV_BF16 = 0, PUREKV_FP32 = 1 } purekv_dtype;
 
 #define PUREKV_FLAG_DENSE_CAUSAL 1u
+#define PUREKV_FLAG_COARSE_BLOCKS 2u
 
 /* The ST-SpAttn mask (Sec. 3.2).  The paper's mask is {anchor_frames 1, spatial_radius -1,
  * temporal_depth 1, temporal_stride 1, temporal_radius 0}: a visual query attends the first
  * frame, its own frame, and its own grid cell in the previous frame, all under causality.
  * Other values are this library's extension.  Text queries are dense causal and prefix keys
  * are visible to every query.  The mask is token-exact; `tile` only sets the granularity at
- * which fully masked key blocks are skipped. */
+ * which fully masked key blocks are skipped -- unless PUREKV_FLAG_COARSE_BLOCKS is set: then the
+ * mask is widened to tile x tile blocks of request positions (a block pair is kept whole, under
+ * causality, as soon as it holds one kept pair), the block-sparse reading of the same mask.
+ * The sparse-attention variants the paper compares with (App. A.3, Table 7; the paper names
+ * them and shows them in a figure only, so the settings are the usual meanings of the names):
+ *   Spatial Sparse Attention   {1, -1, 0, 1, 0}: the spatial path alone, first frame + own frame;
+ *   Temporal Sparse Attention  {1,  0, 1, 1, 0}: the temporal path alone, first frame + own cell
+ *                              of the previous frame (+ the token itself);
+ *   Local Attention            {0,  0, 0, 1, 0} with local_window = L: the L most recent positions;
+ *   Atrous Attention           {0,  0, 0, 1, 0} with atrous_dilation = D: every D-th earlier position.
+ * A visual query sees the union of whatever terms are switched on. */
 typedef struct {
   int32_t grid_h, grid_w;  /* per-frame token grid                                         */
   int32_t anchor_frames;   /* first frames every visual query sees                         */
@@ -60,7 +71,10 @@ typedef struct {
   int32_t temporal_stride; /* linked frames are f-s, f-2s, ... (>= 1)                      */
   int32_t temporal_radius; /* 0: same grid cell; r: Chebyshev radius; -1: whole frame      */
   int32_t tile;            /* key-block size for skipping: 16, 32, 64 or 128               */
-  uint32_t flags;          /* PUREKV_FLAG_DENSE_CAUSAL: plain causal attention             */
+  uint32_t flags;          /* PUREKV_FLAG_DENSE_CAUSAL: plain causal attention;
+                              PUREKV_FLAG_COARSE_BLOCKS: widen the mask to whole blocks   */
+  int32_t local_window;    /* > 0: also the local_window most recent positions (0: off)    */
+  int32_t atrous_dilation; /* > 0: also positions i - D, i - 2D, ... (0: off)              */
 } purekv_st_params;
 
 /* Packed batch.  Device arrays feed kernels; host mirrors feed planning and launch sizing.

@@ -23,6 +23,7 @@ _lib = C.CDLL(LIB_PATH)
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT, ERR_BAD_PLAN = range(7)
 BF16, FP32 = 0, 1
 FLAG_DENSE_CAUSAL = 1
+FLAG_COARSE_BLOCKS = 2
 
 EXPORTS = ("purekv_version", "purekv_last_error", "purekv_budget", "purekv_plan_bytes", "purekv_plan_build",
            "purekv_plan_build_host",
@@ -37,7 +38,8 @@ _i32p = C.POINTER(C.c_int32)
 class StParams(C.Structure):
     _fields_ = [("grid_h", C.c_int32), ("grid_w", C.c_int32), ("anchor_frames", C.c_int32),
                 ("spatial_radius", C.c_int32), ("temporal_depth", C.c_int32), ("temporal_stride", C.c_int32),
-                ("temporal_radius", C.c_int32), ("tile", C.c_int32), ("flags", C.c_uint32)]
+                ("temporal_radius", C.c_int32), ("tile", C.c_int32), ("flags", C.c_uint32),
+                ("local_window", C.c_int32), ("atrous_dilation", C.c_int32)]
 
 
 class CBatch(C.Structure):
@@ -184,7 +186,8 @@ def st_params(mask, tile: Optional[int] = None) -> StParams:
     """From an object with the STMask attributes."""
     return StParams(mask.grid_h, mask.grid_w, mask.anchor_frames, mask.spatial_radius, mask.temporal_depth,
                     mask.temporal_stride, mask.temporal_radius, tile if tile is not None else mask.tile,
-                    FLAG_DENSE_CAUSAL if mask.dense_causal else 0)
+                    (FLAG_DENSE_CAUSAL if mask.dense_causal else 0) | (FLAG_COARSE_BLOCKS if getattr(mask, "coarse", False) else 0),
+                    getattr(mask, "local_window", 0), getattr(mask, "atrous_dilation", 0))
 
 
 class Plan:

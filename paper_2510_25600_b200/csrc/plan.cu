@@ -60,7 +60,7 @@ static purekv_status check_params(const purekv_batch* b, const purekv_st_params*
              "tile %d not in {16,32,64,128}", p->tile);
   PK_REQUIRE(p->anchor_frames >= 0 && p->spatial_radius >= -1 && p->temporal_depth >= -1 &&
                  p->temporal_radius >= -1 && p->temporal_stride >= 1 && p->temporal_stride <= 32767 &&
-                 p->temporal_depth <= 32767,
+                 p->temporal_depth <= 32767 && p->local_window >= 0 && p->atrous_dilation >= 0,
              PUREKV_ERR_INVALID_ARG, "mask parameter out of range");
   PK_REQUIRE(dtype == PUREKV_BF16 || dtype == PUREKV_FP32, PUREKV_ERR_INVALID_ARG, "unknown dtype");
   const int64_t n = (int64_t)p->grid_h * p->grid_w;
@@ -249,7 +249,9 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
   memset(info, 0, sizeof(*info));
 
   std::vector<int64_t> cnt, diff, cg;  // kept pairs per gk-key block of the current query tile
-  std::vector<Span> spans, row_spans;
+  std::vector<Span> spans, row_spans, merged;
+  std::vector<char> blk_kept;
+  const bool coarse = (p->flags & PUREKV_FLAG_COARSE_BLOCKS) != 0 && !dense;
   std::vector<int32_t> row_off;
   for (int r = 0; r < b->n_req; ++r) {
     const int32_t base = b->h_cu_seqlens[r];
@@ -261,6 +263,51 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
     diff.assign((size_t)nkt + 3, 0);
     cg.assign((size_t)nkt + 3, 0);
     const int32_t anchor_end = (int32_t)std::min<int64_t>(vis_end, npre + (int64_t)p->anchor_frames * n);  // exclusive
+    // the token-level mask of row i as disjoint ascending spans of kept key positions
+    auto token_spans = [&](int32_t i, std::vector<Span>& out) {
+      out.clear();
+      const bool visual = i >= npre && i < vis_end;
+      if (dense || !visual) {
+        out.push_back({0, i});  // text rows and the dense mask: plain causal
+        return;
+      }
+      spans.clear();
+      if (anchor_end > 0) spans.push_back({0, std::min(i, anchor_end - 1)});  // prefix + first frame(s)
+      const int32_t f = (i - npre) / n, c = (i - npre) % n, y = c / gw, x = c % gw;
+      const int32_t fs = npre + f * n;
+      if (p->spatial_radius < 0) {
+        spans.push_back({fs, i});  // the current frame, causal
+      } else {
+        const int32_t rr = p->spatial_radius;
+        for (int32_t yy = std::max(0, y - rr); yy <= y; ++yy) {
+          const int32_t xa = std::max(0, x - rr), xb = yy == y ? x : std::min(gw - 1, x + rr);
+          spans.push_back({fs + yy * gw + xa, fs + yy * gw + xb});
+        }
+      }
+      for (int32_t m = 1;; ++m) {  // linked earlier frames: the corresponding cell (or a window / the frame)
+        const int64_t fj = (int64_t)f - (int64_t)m * p->temporal_stride;
+        if (fj < 0 || (p->temporal_depth >= 0 && m > p->temporal_depth)) break;
+        const int32_t fjs = npre + (int32_t)fj * n;
+        if (p->temporal_radius < 0) {
+          spans.push_back({fjs, fjs + n - 1});
+        } else {
+          const int32_t rr = p->temporal_radius;
+          for (int32_t yy = std::max(0, y - rr); yy <= std::min(gh - 1, y + rr); ++yy)
+            spans.push_back({fjs + yy * gw + std::max(0, x - rr), fjs + yy * gw + std::min(gw - 1, x + rr)});
+        }
+      }
+      if (p->local_window > 0) spans.push_back({std::max(npre, i - p->local_window + 1), i});  // the most recent positions
+      if (p->atrous_dilation > 0)                                                             // every D-th position back
+        for (int32_t j = i; j >= npre; j -= p->atrous_dilation) spans.push_back({j, j});
+      std::sort(spans.begin(), spans.end(), [](const Span& u, const Span& v) { return u.a < v.a; });
+      int32_t ca = spans[0].a, cb = spans[0].b;
+      for (size_t s = 1; s < spans.size(); ++s) {
+        if (spans[s].a <= cb + 1) cb = std::max(cb, spans[s].b);
+        else { out.push_back({ca, cb}); ca = spans[s].a; cb = spans[s].b; }
+      }
+      out.push_back({ca, cb});
+    };
+    int32_t cached_rb = -1;          // block of rows whose kept key blocks are in blk_kept (coarse masks)
     for (int32_t q0 = 0; q0 < len; q0 += tq) {
       const int32_t q1 = std::min(len, q0 + tq);  // exclusive
       const int32_t kt_hi = (q1 - 1) / tk;        // last list entry a causal mask reaches
@@ -278,44 +325,32 @@ static purekv_status build_plan(const purekv_batch* b, const purekv_st_params* p
         diff[ta + 1] += gk;
         diff[tb] -= gk;
       };
-      // each row's kept keys as disjoint ascending spans (Sec. 3.2)
+      // each row's kept keys as disjoint ascending spans (Sec. 3.2; App. A.3 for the local and atrous terms)
       for (int32_t i = q0; i < q1; ++i) {
-        const bool visual = i >= npre && i < vis_end;
-        if (dense || !visual) {
-          add_span(0, i);  // text rows and the dense mask: plain causal
+        if (!coarse) {
+          token_spans(i, merged);
+          for (const Span& sp : merged) add_span(sp.a, sp.b);
         } else {
-          spans.clear();
-          if (anchor_end > 0) spans.push_back({0, std::min(i, anchor_end - 1)});  // prefix + first frame(s)
-          const int32_t f = (i - npre) / n, c = (i - npre) % n, y = c / gw, x = c % gw;
-          const int32_t fs = npre + f * n;
-          if (p->spatial_radius < 0) {
-            spans.push_back({fs, i});  // the current frame, causal
-          } else {
-            const int32_t rr = p->spatial_radius;
-            for (int32_t yy = std::max(0, y - rr); yy <= y; ++yy) {
-              const int32_t xa = std::max(0, x - rr), xb = yy == y ? x : std::min(gw - 1, x + rr);
-              spans.push_back({fs + yy * gw + xa, fs + yy * gw + xb});
+          // block-level widening: the key blocks in which any row of this row's block keeps a pair (found once per
+          // block of rows), each taken whole up to the diagonal
+          const int32_t rb = i / gk;
+          if (rb != cached_rb) {
+            cached_rb = rb;
+            const int32_t r_hi = std::min(len, rb * gk + gk);
+            blk_kept.assign((size_t)(r_hi - 1) / gk + 1, 0);
+            for (int32_t ii = rb * gk; ii < r_hi; ++ii) {
+              token_spans(ii, merged);
+              for (const Span& sp : merged)
+                for (int32_t kb = sp.a / gk; kb <= sp.b / gk; ++kb) blk_kept[kb] = 1;
             }
           }
-          for (int32_t m = 1;; ++m) {  // linked earlier frames: the corresponding cell (or a window / the frame)
-            const int64_t fj = (int64_t)f - (int64_t)m * p->temporal_stride;
-            if (fj < 0 || (p->temporal_depth >= 0 && m > p->temporal_depth)) break;
-            const int32_t fjs = npre + (int32_t)fj * n;
-            if (p->temporal_radius < 0) {
-              spans.push_back({fjs, fjs + n - 1});
-            } else {
-              const int32_t rr = p->temporal_radius;
-              for (int32_t yy = std::max(0, y - rr); yy <= std::min(gh - 1, y + rr); ++yy)
-                spans.push_back({fjs + yy * gw + std::max(0, x - rr), fjs + yy * gw + std::min(gw - 1, x + rr)});
-            }
+          for (int32_t kb = 0; kb <= i / gk; ++kb) {
+            if (!blk_kept[kb]) continue;
+            int32_t ke = kb;
+            while (ke + 1 <= i / gk && blk_kept[ke + 1]) ++ke;
+            add_span(kb * gk, std::min(ke * gk + gk - 1, i));
+            kb = ke;
           }
-          std::sort(spans.begin(), spans.end(), [](const Span& u, const Span& v) { return u.a < v.a; });
-          int32_t ca = spans[0].a, cb = spans[0].b;
-          for (size_t s = 1; s < spans.size(); ++s) {
-            if (spans[s].a <= cb + 1) cb = std::max(cb, spans[s].b);
-            else { add_span(ca, cb); ca = spans[s].a; cb = spans[s].b; }
-          }
-          add_span(ca, cb);
         }
         row_off.push_back((int32_t)row_spans.size());
       }

@@ -37,6 +37,22 @@ def test_prefill_tensor_core_kernel(tile, mask_kw):
     gc.check_prefill(wl, inputs.make_qkv(wl, 0))
 
 
+VARIANTS = [("spatial", {}), ("temporal", {}), ("local", dict(local_window=40)), ("atrous", dict(atrous_dilation=3))]
+
+
+@pytest.mark.parametrize("coarse", [False, True])
+@pytest.mark.parametrize("name,kw", VARIANTS + [("st", {})])
+def test_prefill_named_mask_variants(name, kw, coarse):
+    """The sparse-attention variants of App. A.3 / Table 7 and their block-level widening, on both kernels."""
+    if name == "st" and not coarse:
+        pytest.skip("the paper's token-exact mask is covered by the tests above")
+    for dtype, d, tile in (("bf16", 128, 64), ("bf16", 128, 128), ("fp32", 64, 16)):
+        batch = inputs.make_batch([37, 0, 5], [5, 3, 1], [29, 140, 0], 9, 11)
+        wl = inputs.Workload("t", 19, dtype, 4, 2, d, 1, (0,), (0,), batch,
+                             inputs.mask_variant(name, 9, 11, tile=tile, coarse=coarse, **kw), 8, 0.3)
+        gc.check_prefill(wl, inputs.make_qkv(wl, 0))
+
+
 @pytest.mark.parametrize("tile", [64, 128])
 @pytest.mark.parametrize("H,Hkv,n_ctas", [(3, 1, 0), (7, 1, 5), (4, 2, 600), (5, 1, 300), (2, 2, 1)])
 def test_prefill_tensor_core_schedules(tile, H, Hkv, n_ctas):

@@ -131,3 +131,15 @@ def test_workload_long_video_sweep():
             assert plan.info.pairs_kept == 41042944                             # closed form of the paper's mask
     for keep in (0.1, 0.5):
         check_scores_selection_compaction(inputs.workload(3, keep_ratio=keep), x0, [x0], groups=[1])
+
+
+def test_workload_named_mask_variants_at_full_size():
+    """App. A.3 / Table 7: each named variant on the VideoLLaMA2-shaped prompt (sampled rows against the oracle)."""
+    wl = inputs.workload(1)
+    rng = np.random.default_rng(wl.seed + 1)
+    x0 = inputs.make_qkv(wl, 0, pool=POOL)
+    rows = sample_rows(wl, 32, rng)
+    g = wl.mask.grid_h
+    for name, kw in (("spatial", {}), ("temporal", {}), ("local", dict(local_window=256)), ("atrous", dict(atrous_dilation=4))):
+        plan = check_prefill_sampled(wl, x0, inputs.mask_variant(name, g, g, tile=64, **kw), rows)
+        assert 0 < plan.info.tiles_kept <= plan.info.tiles_causal

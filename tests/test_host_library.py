@@ -187,6 +187,19 @@ def test_plan_matches_oracle_mask(tile, mask_kw):
     check_plan(batch, inputs.STMask(5, 7, tile=tile, **mask_kw), pk.FP32, 64)
 
 
+@pytest.mark.parametrize("tile", [16, 64])
+@pytest.mark.parametrize("coarse", [False, True])
+@pytest.mark.parametrize("name,kw", [("st", {}), ("spatial", {}), ("temporal", {}), ("local", dict(local_window=9)),
+                                     ("atrous", dict(atrous_dilation=5))])
+def test_plan_matches_oracle_for_the_named_variants_and_their_block_level_widening(name, kw, coarse, tile):
+    """App. A.3 / Table 7 variants: lists, classes and bit masks of the plan against the oracle's mask matrix, for
+    the CUDA-core planner shapes and (tile 64) the tensor-core ones."""
+    batch = inputs.make_batch([5, 0, 20], [6, 3, 0], [9, 40, 3], 5, 7)
+    check_plan(batch, inputs.mask_variant(name, 5, 7, tile=tile, coarse=coarse, **kw), pk.FP32, 64)
+    if tile == 64:
+        check_plan(batch, inputs.mask_variant(name, 5, 7, tile=tile, coarse=coarse, **kw), pk.BF16, 128, 4, 2, 7)
+
+
 def test_plan_for_tensor_core_shapes_and_workload_counts():
     batch = inputs.make_batch([64, 3], [5, 2], [64, 130], 12, 12)
     for tile in (64, 128):
