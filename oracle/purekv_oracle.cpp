@@ -13,6 +13,10 @@
 //                      kept keys of each row.
 //   pko_lowlayer_score Eq. 1 (dense causal softmax rows) and Eq. 2 (sum of the recent
 //                      window's rows over the non-recent keys).
+//   pko_lowlayer_score_ex  the same with the other reductions of App. A.1 / Table 6's policies
+//                      (accumulation over all rows, an observation window, pooling along keys).
+//   pko_select_sink_recent  the score-free policy of App. A.1 / Table 6 (first keys + window).
+//   pko_spearman       Eq. 7, the rank correlation of Sec. 3.3 (validation tool, CPU only).
 //   pko_vnorm_scores   Eq. 3 / Eq. 4 (C weighted by the L2 norm of each key's V vector).
 //   pko_select         Sec. 3.1: keep the recent window w plus the top-h non-recent keys.
 //   pko_compact        the compacted cache implied by that selection.
@@ -209,6 +213,98 @@ void pko_lowlayer_score(const float* q, const float* k,
       for (int32_t j = 0; j < nr; ++j) c_out[(int64_t)g * T + base + j] = acc[j] / (double)G;
     }
   }
+}
+
+// The score reductions of the policies the paper combines its estimator with (App. A.1, Table 6), as variations of
+// Eq. 2 (the paper cites them by name; the forms below are the usual ones of those methods):
+//   accumulated attention (Sec. 3.1: "most existing methods rely on accumulated attention scores", which the
+//     lower-triangular matrix biases toward early tokens): every row of A is summed, obs_rows < 0 or >= l;
+//   an observation window of obs_rows last rows (obs_rows = window is Eq. 2 itself);
+//   pooling along the key axis: pool > 1 replaces each non-recent key's sum by the mean over the pool positions
+//     centred on it, positions outside the non-recent segment counting as 0 (pool odd).
+// A row contributes to the keys it can see (j <= i) only.  Rows, normalisation, GQA mean and output layout as in
+// pko_lowlayer_score.
+void pko_lowlayer_score_ex(const float* q, const float* k, int32_t n_req, const int32_t* cu_seqlens, int32_t window,
+                           int32_t obs_rows, int32_t pool, int32_t n_q_heads, int32_t n_kv_heads, int32_t d,
+                           double scale, double* c_out) {
+  const int64_t T = cu_seqlens[n_req];
+  if (scale <= 0.0) scale = 1.0 / std::sqrt((double)d);
+  const int32_t G = n_q_heads / n_kv_heads;
+  for (int64_t x = 0; x < (int64_t)n_kv_heads * T; ++x) c_out[x] = 0.0;
+  for (int32_t r = 0; r < n_req; ++r) {
+    const int64_t base = cu_seqlens[r];
+    const int32_t len = cu_seqlens[r + 1] - cu_seqlens[r];
+    const int32_t w = std::min(window, len);
+    const int32_t nr = len - w;
+    const int32_t wo = (obs_rows < 0 || obs_rows > len) ? len : obs_rows;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int32_t g = 0; g < n_kv_heads; ++g) {
+      std::vector<double> s(len), acc(std::max(nr, 1), 0.0);
+      for (int32_t hq = g * G; hq < (g + 1) * G; ++hq)
+        for (int32_t i = len - wo; i < len; ++i) {
+          const float* qi = q + ((base + i) * n_q_heads + hq) * d;
+          double m = -std::numeric_limits<double>::infinity();
+          for (int32_t j = 0; j <= i; ++j) {
+            s[j] = scale * dot_fd(qi, k + ((base + j) * n_kv_heads + g) * d, d);
+            m = std::max(m, s[j]);
+          }
+          double z = 0.0;
+          for (int32_t j = 0; j <= i; ++j) { s[j] = std::exp(s[j] - m); z += s[j]; }
+          for (int32_t j = 0; j < nr && j <= i; ++j) acc[j] += s[j] / z;
+        }
+      for (int32_t j = 0; j < nr; ++j) {
+        double v = 0.0;
+        const int32_t half = pool > 1 ? pool / 2 : 0;
+        for (int32_t jj = j - half; jj <= j + half; ++jj)
+          if (jj >= 0 && jj < nr) v += acc[jj];
+        c_out[(int64_t)g * T + base + j] = v / (double)(2 * half + 1) / (double)G;
+      }
+    }
+  }
+}
+
+// The selection of a policy that uses no scores (attention sinks + recent window, App. A.1 / Table 6): of the
+// non-recent keys the first h_keep[r] positions are kept, then the recent window, for every KV head.
+int32_t pko_select_sink_recent(int32_t n_req, const int32_t* cu_seqlens, int32_t window, const int32_t* h_keep,
+                               const int32_t* cu_kept, int32_t n_kv_heads, int32_t* idx_out) {
+  const int64_t K_tot = cu_kept[n_req];
+  for (int32_t r = 0; r < n_req; ++r) {
+    const int32_t len = cu_seqlens[r + 1] - cu_seqlens[r];
+    const int32_t w = std::min(window, len), h = h_keep[r];
+    if (h < 0 || h > len - w || cu_kept[r + 1] - cu_kept[r] != h + w) return 1;
+    for (int32_t g = 0; g < n_kv_heads; ++g) {
+      int32_t* o = idx_out + (int64_t)g * K_tot + cu_kept[r];
+      for (int32_t t = 0; t < h; ++t) o[t] = t;
+      for (int32_t t = 0; t < w; ++t) o[h + t] = len - w + t;
+    }
+  }
+  return 0;
+}
+
+// Spearman's rank correlation of two score vectors (Sec. 3.3, Eq. 7): rho = 1 - 6 sum_j d_j^2 / (n (n^2 - 1)), d_j the
+// difference of the two ranks of element j.  The printed upper limit of the sum (j = 0 .. n) has one term too many
+// for n elements: the sum runs over the n elements.  Ranks are 1 .. n by descending value; equal values share the
+// mean of the ranks they span (the formula is exact only without ties).  n < 2 gives NaN.
+double pko_spearman(const double* a, const double* b, int64_t n) {
+  if (n < 2) return std::nan("");
+  auto ranks = [n](const double* x) {
+    std::vector<int64_t> order(n);
+    std::iota(order.begin(), order.end(), (int64_t)0);
+    std::stable_sort(order.begin(), order.end(), [x](int64_t u, int64_t v) { return x[u] > x[v]; });
+    std::vector<double> rk(n);
+    for (int64_t p = 0; p < n;) {
+      int64_t e = p;
+      while (e + 1 < n && x[order[e + 1]] == x[order[p]]) ++e;
+      const double mean_rank = 0.5 * (double)(p + e) + 1.0;
+      for (int64_t t = p; t <= e; ++t) rk[order[t]] = mean_rank;
+      p = e + 1;
+    }
+    return rk;
+  };
+  const std::vector<double> ra = ranks(a), rb = ranks(b);
+  double sum = 0.0;
+  for (int64_t j = 0; j < n; ++j) sum += (ra[j] - rb[j]) * (ra[j] - rb[j]);
+  return 1.0 - 6.0 * sum / ((double)n * ((double)n * (double)n - 1.0));
 }
 
 // Eq. 3 / Eq. 4 for one layer: S[g, t] = C[g, t] * ||V[t, g, :]||_2.

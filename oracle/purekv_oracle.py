@@ -45,6 +45,8 @@ def lib():
         _lib = C.CDLL(build())
         _lib.pko_mask.restype = C.c_int32
         _lib.pko_select.restype = C.c_int32
+        _lib.pko_select_sink_recent.restype = C.c_int32
+        _lib.pko_spearman.restype = C.c_double
     return _lib
 
 
@@ -102,6 +104,55 @@ def lowlayer_score(q, k, cu_seqlens, window: int, scale: float = 0.0) -> np.ndar
                              C.c_int32(window), C.c_int32(h), C.c_int32(hkv), C.c_int32(d),
                              C.c_double(scale), _p(c, C.c_double))
     return c
+
+
+def lowlayer_score_ex(q, k, cu_seqlens, window: int, obs_rows: int = -1, pool: int = 1, scale: float = 0.0) -> np.ndarray:
+    """C [H_kv, T] float64 under another reduction (App. A.1 / Table 6): the last obs_rows rows of each request are
+    accumulated (all rows if negative), then averaged over `pool` neighbouring keys."""
+    q = np.ascontiguousarray(q, dtype=np.float32)
+    k = np.ascontiguousarray(k, dtype=np.float32)
+    t_tot, h, d = q.shape
+    hkv = k.shape[1]
+    cu = _i32(cu_seqlens)
+    c = np.zeros((hkv, t_tot), dtype=np.float64)
+    lib().pko_lowlayer_score_ex(_p(q, C.c_float), _p(k, C.c_float), C.c_int32(len(cu) - 1), _p(cu, C.c_int32),
+                                C.c_int32(window), C.c_int32(obs_rows), C.c_int32(pool), C.c_int32(h), C.c_int32(hkv),
+                                C.c_int32(d), C.c_double(scale), _p(c, C.c_double))
+    return c
+
+
+def select_sink_recent(cu_seqlens, window: int, h_keep, cu_kept, n_kv_heads: int) -> np.ndarray:
+    """idx [H_kv, K_tot] of the score-free policy: the first h positions of each request, then its window."""
+    cu, hk, ck = _i32(cu_seqlens), _i32(h_keep), _i32(cu_kept)
+    idx = np.zeros((n_kv_heads, int(ck[-1])), dtype=np.int32)
+    if lib().pko_select_sink_recent(C.c_int32(len(cu) - 1), _p(cu, C.c_int32), C.c_int32(window), _p(hk, C.c_int32),
+                                    _p(ck, C.c_int32), C.c_int32(n_kv_heads), _p(idx, C.c_int32)) != 0:
+        raise ValueError("select_sink_recent: a request's h is outside [0, l - w] or its kept count is not h + w")
+    return idx
+
+
+def spearman(a, b) -> float:
+    """Eq. 7 on two equally long score vectors."""
+    a = np.ascontiguousarray(a, dtype=np.float64).ravel()
+    b = np.ascontiguousarray(b, dtype=np.float64).ravel()
+    assert a.shape == b.shape
+    return float(lib().pko_spearman(_p(a, C.c_double), _p(b, C.c_double), C.c_int64(a.size)))
+
+
+def clie_rank_agreement(q_low, k_low, q_high, k_high, v_high, cu_seqlens, window: int) -> np.ndarray:
+    """The validation study of Sec. 3.3 for one (low layer, high layer) pair: Spearman's rho between the estimate
+    S_hat = C_low * ||V_high|| (Eq. 4) and S_high = C_high * ||V_high|| (Eq. 6) over each request's non-recent keys.
+    Returns rho [H_kv, n_req].  CPU only; on synthetic inputs it checks the plumbing, not the paper's hypothesis."""
+    cu = _i32(cu_seqlens)
+    s_hat = vnorm_scores(lowlayer_score(q_low, k_low, cu, window), v_high)
+    s_high = vnorm_scores(lowlayer_score(q_high, k_high, cu, window), v_high)
+    out = np.full((s_hat.shape[0], len(cu) - 1), np.nan)
+    for r in range(len(cu) - 1):
+        nr = int(cu[r + 1] - cu[r]) - min(window, int(cu[r + 1] - cu[r]))
+        for g in range(s_hat.shape[0]):
+            if nr >= 2:
+                out[g, r] = spearman(s_hat[g, cu[r]:cu[r] + nr], s_high[g, cu[r]:cu[r] + nr])
+    return out
 
 
 def vnorm_scores(c: np.ndarray, v: np.ndarray) -> np.ndarray:
