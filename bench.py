@@ -503,8 +503,19 @@ def sub_pipeline(cfg, steps, peaks, timer):
                             ["ST-SpAttn (paper)", "ST-SpAttn widened to blocks", "Spatial Sparse Attention",
                              "Temporal Sparse Attention", "Local Attention (256 positions)",
                              "Atrous Attention (every 4th position)"], 5, peaks, timer)
+    # the score reductions of the other eviction policies (App. A.1 / Table 6) on the scored layer, two-pass kernels
+    from paper_2510_25600_b200 import binding as P
+    reductions = []
+    for label, obs, pool in (("window rows (Eq. 2)", wl.window, 1), ("observation window 32 + pooling 7", 32, 7),
+                             ("accumulated attention, all rows", -1, 1)):
+        ws_r = torch.empty(P.purekv_score_ex_ws_bytes(pipe.batch, obs, pool, wl.n_q_heads, wl.n_kv_heads), dtype=torch.uint8, device="cuda")
+        c_r = torch.empty_like(pipe.c[0])
+        t_r = timer(lambda: P.purekv_lowlayer_score_ex(d_in[0][0], d_in[1][0], pipe.batch, wl.window, obs, pool, c_out=c_r, ws=ws_r))
+        rows_acc = wl.batch.total_tokens if obs < 0 else min(obs, wl.batch.total_tokens)
+        reductions.append({"reduction": label, "ms": t_r, "workspace_MB": ws_r.numel() / 1e6,
+                           "TFLOPs": 2 * 2.0 * wl.n_q_heads * wl.head_dim * rows_acc * wl.batch.total_tokens / t_r / 1e9})
     return {"config": config_dict(wl), "inputs": "N(0,1) bf16 drawn on the device (seeded); timing only",
-            "mask_variants": variants, "mask_variants_note": "one layer, kernel timed alone with cold L2; fractions in each row",
+            "score_reductions": reductions, "mask_variants": variants, "mask_variants_note": "one layer, kernel timed alone with cold L2; fractions in each row",
             "tokens_per_s": wl.batch.total_tokens / (ms_step * 1e-3), "ms_per_step": ms_step, "steps": steps, "clocks": clocks,
             "roofline": {k: roofline[k] for k in keep}, "steps_detail": detail, "steps_detail_clocks": sampler.stop()}
 

@@ -185,6 +185,31 @@ purekv_status purekv_lowlayer_score_lse(const void *q, const void *k, const floa
                                         int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
                                         float softmax_scale, int32_t *status, void *stream);
 
+/* ---- the score reductions of other eviction policies (App. A.1, Table 6: the paper drives H2O-, SnapKV- and
+ * StreamingLLM-style policies with its estimator and ST-SpAttn; it cites the policies by name, so the forms here are
+ * the usual ones of those methods) ------------------------------------------------------------
+ * purekv_lowlayer_score_ex is purekv_lowlayer_score with two more parameters:
+ *   obs_rows  how many of a request's last rows are accumulated.  obs_rows = window is Eq. 2 itself; a negative
+ *             value (or one beyond the request) accumulates every row of A -- the "accumulated attention scores"
+ *             of Sec. 3.1, biased toward early keys by the lower-triangular matrix; a small value is the
+ *             observation window of SnapKV-style policies.  A row counts only for the keys it can see (j <= i).
+ *   pool      odd, >= 1: each non-recent key's sum is replaced by the mean over `pool` positions centred on it,
+ *             positions outside the non-recent segment counting as zero (1: no pooling).
+ * c_out as in purekv_lowlayer_score (the recent `window` keys get 0), so Eq. 3 / Eq. 4 and the selection apply
+ * unchanged.  ws: purekv_score_ex_ws_bytes.  Accumulating all rows costs two passes over the whole causal matrix.
+ * purekv_select_sink_recent is the score-free policy (attention sinks + recent window): for every layer and KV
+ * head the first h_keep[r] positions of request r, then its window; idx_out as purekv_select_topk writes it. */
+size_t purekv_score_ex_ws_bytes(const purekv_batch *batch, int32_t obs_rows, int32_t pool, int32_t n_q_heads,
+                                int32_t n_kv_heads);
+purekv_status purekv_lowlayer_score_ex(const void *q, const void *k, float *c_out, const purekv_batch *batch,
+                                       int32_t window, int32_t obs_rows, int32_t pool, int32_t n_q_heads,
+                                       int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                       float softmax_scale, void *ws, size_t ws_bytes, void *stream);
+purekv_status purekv_select_sink_recent(const purekv_batch *batch, int32_t window, const int32_t *keep /* device */,
+                                        const int32_t *h_keep, const int32_t *cu_kept /* device */,
+                                        const int32_t *h_cu_kept, int32_t n_layers, int32_t n_kv_heads,
+                                        int32_t *idx_out, void *stream);
+
 /* ---- the same scores for callers that cannot hand over a workspace ---------------------------
  * (The paper has no counterpart: this is a packaging variant of purekv_lowlayer_score.)
  * Some callers cannot obtain device memory at the moment they need the scores: a serving engine that

@@ -30,7 +30,8 @@ EXPORTS = ("purekv_version", "purekv_last_error", "purekv_budget", "purekv_plan_
            "purekv_st_sparse_prefill", "purekv_score_ws_bytes", "purekv_lowlayer_score", "purekv_lowlayer_score_lse", "purekv_lowlayer_score_noalloc",
            "purekv_select_ws_bytes",
            "purekv_select_topk", "purekv_compact_kv", "purekv_decode_ws_bytes", "purekv_decode_attention",
-           "purekv_poll_status", "purekv_set_wait_limit_ns")
+           "purekv_poll_status", "purekv_set_wait_limit_ns", "purekv_score_ex_ws_bytes", "purekv_lowlayer_score_ex",
+           "purekv_select_sink_recent")
 
 _i32p = C.POINTER(C.c_int32)
 
@@ -87,6 +88,13 @@ _lib.purekv_st_sparse_prefill.argtypes = [C.c_void_p] * 5 + [C.POINTER(CBatch), 
 _lib.purekv_score_ws_bytes.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_int32]
 _lib.purekv_lowlayer_score.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32, C.c_int32,
                                        C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.purekv_score_ex_ws_bytes.restype = C.c_size_t
+_lib.purekv_score_ex_ws_bytes.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_int32, C.c_int32, C.c_int32]
+_lib.purekv_lowlayer_score_ex.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32, C.c_int32,
+                                          C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p,
+                                          C.c_size_t, C.c_void_p]
+_lib.purekv_select_sink_recent.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_void_p, _i32p, C.c_void_p, _i32p, C.c_int32,
+                                           C.c_int32, C.c_void_p, C.c_void_p]
 _lib.purekv_lowlayer_score_lse.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32,
                                            C.c_int32, C.c_int32, C.c_int32, C.c_int, C.c_float, C.c_void_p, C.c_void_p]
 _lib.purekv_lowlayer_score_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(CBatch), C.c_int32,
@@ -285,6 +293,40 @@ def purekv_lowlayer_score_lse(q: torch.Tensor, k: torch.Tensor, lse: torch.Tenso
                                           window, h, hkv, d, _dtype_code(q), softmax_scale, _ptr(status), _stream()),
            "purekv_lowlayer_score_lse")
     return c_out
+
+
+def purekv_score_ex_ws_bytes(batch: Batch, obs_rows: int, pool: int, n_q_heads: int, n_kv_heads: int) -> int:
+    return int(_lib.purekv_score_ex_ws_bytes(C.byref(batch.c), obs_rows, pool, n_q_heads, n_kv_heads))
+
+
+def purekv_lowlayer_score_ex(q: torch.Tensor, k: torch.Tensor, batch: Batch, window: int, obs_rows: int = -1,
+                             pool: int = 1, c_out: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
+                             softmax_scale: float = 0.0) -> torch.Tensor:
+    """C [H_kv, T] fp32 with the last `obs_rows` rows accumulated (all rows if negative) and averaged over `pool`
+    neighbouring keys: the score reductions of the other eviction policies of App. A.1 / Table 6."""
+    assert q.is_contiguous() and k.is_contiguous()
+    t, h, d = q.shape
+    hkv = k.shape[1]
+    if c_out is None:
+        c_out = torch.empty((hkv, t), dtype=torch.float32, device=q.device)
+    if ws is None:
+        ws = torch.empty(purekv_score_ex_ws_bytes(batch, obs_rows, pool, h, hkv), dtype=torch.uint8, device=q.device)
+    _check(_lib.purekv_lowlayer_score_ex(q.data_ptr(), k.data_ptr(), c_out.data_ptr(), C.byref(batch.c), window, obs_rows,
+                                         pool, h, hkv, d, _dtype_code(q), softmax_scale, ws.data_ptr(), ws.numel(),
+                                         _stream()), "purekv_lowlayer_score_ex")
+    return c_out
+
+
+def purekv_select_sink_recent(batch: Batch, budget: "Budget", n_layers: int, n_kv_heads: int,
+                              idx_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """idx [L, H_kv, K_tot] of the score-free policy: the first h positions of each request, then its window."""
+    if idx_out is None:
+        idx_out = torch.empty((n_layers, n_kv_heads, budget.total_kept), dtype=torch.int32, device="cuda")
+    _check(_lib.purekv_select_sink_recent(C.byref(batch.c), budget.window, budget.keep.data_ptr(),
+                                          budget.h_keep.ctypes.data_as(_i32p), budget.cu_kept.data_ptr(),
+                                          budget.h_cu_kept.ctypes.data_as(_i32p), n_layers, n_kv_heads,
+                                          idx_out.data_ptr(), _stream()), "purekv_select_sink_recent")
+    return idx_out
 
 
 NOALLOC_SCORE_MAX_ROWS = 262144

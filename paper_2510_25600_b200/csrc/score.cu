@@ -151,7 +151,7 @@ __global__ void __launch_bounds__(kThreads) score_lse_kernel(const T* __restrict
 template <typename T>
 __global__ void __launch_bounds__(kThreads) score_colsum_kernel(const T* __restrict__ q, const T* __restrict__ k,
                                                                 const int32_t* __restrict__ cu_seqlens,
-                                                                int32_t window, int32_t n_q_heads,
+                                                                int32_t window, int32_t obs, int32_t n_q_heads,
                                                                 int32_t n_kv_heads, int32_t d, float scale_log2,
                                                                 const float* __restrict__ lse2, int64_t n_tokens,
                                                                 float* __restrict__ c_out) {
@@ -165,6 +165,7 @@ __global__ void __launch_bounds__(kThreads) score_colsum_kernel(const T* __restr
   const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
   const int32_t w = min(window, len);
   const int32_t nr = len - w;  // non-recent keys
+  const int32_t wo = min(obs, len);  // rows that are accumulated: the last wo of the request (Eq. 2: wo = w)
   const int32_t j0 = blockIdx.x * kKB;
   if (j0 >= len) return;
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
@@ -180,7 +181,7 @@ __global__ void __launch_bounds__(kThreads) score_colsum_kernel(const T* __restr
     if (j < len) load_row_f32(dst, k + ((int64_t)(base + j) * n_kv_heads + g) * d, d, tid & 7, 8);
     else for (int c = tid & 7; c < d; c += 8) dst[c] = 0.f;
   }
-  const int32_t n_rows = G * w;
+  const int32_t n_rows = G * wo;
   float col[4] = {0.f, 0.f, 0.f, 0.f};
   for (int32_t row0 = 0; row0 < n_rows; row0 += kRB) {
     __syncthreads();
@@ -188,7 +189,7 @@ __global__ void __launch_bounds__(kThreads) score_colsum_kernel(const T* __restr
       const int32_t row = row0 + rr;
       float* dst = qs + rr * ld;
       if (row < n_rows) {
-        const int32_t hq = g * G + row / w, i = len - w + row % w;
+        const int32_t hq = g * G + row / wo, i = len - wo + row % wo;
         load_row_f32(dst, q + ((int64_t)(base + i) * n_q_heads + hq) * d, d, tid & 7, 8);
       } else {
         for (int c = tid & 7; c < d; c += 8) dst[c] = 0.f;
@@ -201,10 +202,13 @@ __global__ void __launch_bounds__(kThreads) score_colsum_kernel(const T* __restr
     for (int a = 0; a < 2; ++a) {
       const int32_t row = row0 + 2 * ty + a;
       if (row < n_rows) {
-        const float lse = __ldg(lse2 + ((int64_t)r * n_q_heads + g * G + row / w) * window + row % w);
-        // every non-recent key precedes every window row, so causality holds for all of them
+        const float lse = __ldg(lse2 + ((int64_t)r * n_q_heads + g * G + row / wo) * obs + row % wo);
+        // with wo = w every non-recent key precedes every accumulated row; a longer observation reaches rows that
+        // lie before some of the block's keys, and a row only counts for the keys it can see
+        const int32_t i = len - wo + row % wo;
 #pragma unroll
-        for (int b = 0; b < 4; ++b) col[b] += exp2f(s[a][b] * scale_log2 - lse);
+        for (int b = 0; b < 4; ++b)
+          if (j0 + tx + 16 * b <= i) col[b] += exp2f(s[a][b] * scale_log2 - lse);
       }
     }
   }
@@ -412,8 +416,8 @@ __global__ void __launch_bounds__(256) score_lse_merge_kernel(const float2* __re
 // Pass 2 (Eq. 2).  C[g, j] = (1/G) * sum over the stacked rows of exp2(s - lse) for the non-recent keys of the CTA's block.
 __global__ void __launch_bounds__(kMmaThreads) score_mma_colsum_kernel(
     const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k, const int32_t* __restrict__ cu_seqlens,
-    int32_t window, int32_t n_q_heads, int32_t n_kv_heads, int32_t d, float scale_log2, const float* __restrict__ lse2,
-    int64_t n_tokens, float* __restrict__ c_out) {
+    int32_t window, int32_t obs, int32_t n_q_heads, int32_t n_kv_heads, int32_t d, float scale_log2,
+    const float* __restrict__ lse2, int64_t n_tokens, float* __restrict__ c_out) {
   extern __shared__ __align__(16) uint8_t smem_mma[];
   __shared__ float red[4][kCtaKeys];  // per row group of warps
   __nv_bfloat16* ks = reinterpret_cast<__nv_bfloat16*>(smem_mma);
@@ -421,7 +425,8 @@ __global__ void __launch_bounds__(kMmaThreads) score_mma_colsum_kernel(
   const int32_t r = blockIdx.z, g = blockIdx.y, j0 = blockIdx.x * kCtaKeys;
   const int32_t G = n_q_heads / n_kv_heads;
   const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
-  const int32_t w = min(window, len), nr = len - w, n_rows = G * w;
+  const int32_t w = min(window, len), nr = len - w;
+  const int32_t wo = min(obs, len), n_rows = G * wo;  // accumulated rows: the last wo of the request (Eq. 2: wo = w)
   if (j0 >= len) return;
   float* cg = c_out + (int64_t)g * n_tokens + base;
   if (j0 >= nr) {  // block inside the window: defined as 0
@@ -437,7 +442,7 @@ __global__ void __launch_bounds__(kMmaThreads) score_mma_colsum_kernel(
 #pragma unroll
   for (int nb = 0; nb < 8; ++nb) col[nb][0] = col[nb][1] = 0.f;
   auto q_row = [&](int32_t row) -> int64_t {
-    return row < n_rows ? ((int64_t)(base + len - w + row % w) * n_q_heads + g * G + row / w) * d : -1;
+    return row < n_rows ? ((int64_t)(base + len - wo + row % wo) * n_q_heads + g * G + row / wo) * d : -1;
   };
   __nv_bfloat16* qbuf[2] = {qs, qs + kMmaRows * (d + 8)};
   stage_rows_bf16_async(qbuf[0], q, kMmaRows, d, [&](int rr) { return q_row(rr); });
@@ -459,12 +464,22 @@ __global__ void __launch_bounds__(kMmaThreads) score_mma_colsum_kernel(
       for (int h = 0; h < 2; ++h) {
         const int32_t row = row0 + 32 * wr + 16 * mb + (lane >> 2) + 8 * h;
         if (row < n_rows) {
-          // every non-recent key precedes every window row, so causality holds for all of them
-          const float lse = __ldg(lse2 + ((int64_t)r * n_q_heads + g * G + row / w) * window + row % w);
+          const float lse = __ldg(lse2 + ((int64_t)r * n_q_heads + g * G + row / wo) * obs + row % wo);
+          if (wo == w) {
+            // every non-recent key precedes every window row, so causality holds for all of them
 #pragma unroll
-          for (int nb = 0; nb < 8; ++nb) {
-            col[nb][0] += exp2f(fmaf(acc[mb][nb][2 * h], scale_log2, -lse));
-            col[nb][1] += exp2f(fmaf(acc[mb][nb][2 * h + 1], scale_log2, -lse));
+            for (int nb = 0; nb < 8; ++nb) {
+              col[nb][0] += exp2f(fmaf(acc[mb][nb][2 * h], scale_log2, -lse));
+              col[nb][1] += exp2f(fmaf(acc[mb][nb][2 * h + 1], scale_log2, -lse));
+            }
+          } else {
+            // a longer observation reaches rows that lie before some keys: a row only counts for the keys it sees
+            const int32_t i = len - wo + row % wo, jb = j0 + 64 * wc + 2 * (lane & 3);
+#pragma unroll
+            for (int nb = 0; nb < 8; ++nb) {
+              if (jb + 8 * nb <= i) col[nb][0] += exp2f(fmaf(acc[mb][nb][2 * h], scale_log2, -lse));
+              if (jb + 8 * nb + 1 <= i) col[nb][1] += exp2f(fmaf(acc[mb][nb][2 * h + 1], scale_log2, -lse));
+            }
           }
         }
       }
@@ -488,13 +503,16 @@ __global__ void __launch_bounds__(kMmaThreads) score_mma_colsum_kernel(
   }
 }
 
+// `obs` = accumulated rows per request and head (Eq. 2: the window itself); the first pass and the merge see only
+// rows, so they take it in place of the window.
 static purekv_status launch_score_mma(const void* q, const void* k, float* c_out, const purekv_batch* b, int32_t window,
-                                      int32_t H, int32_t Hkv, int32_t d, float scale, float* ws_f, cudaStream_t sm) {
+                                      int32_t obs, int32_t H, int32_t Hkv, int32_t d, float scale, float* ws_f,
+                                      cudaStream_t sm) {
   const int32_t ml = max_len(b);
-  const int32_t n_kb = (ml + kMmaKeys - 1) / kMmaKeys, rows_max = (H / Hkv) * window;
-  float* lse2 = ws_f;                                                             // [n_req][H][window]
+  const int32_t n_kb = (ml + kMmaKeys - 1) / kMmaKeys, rows_max = (H / Hkv) * obs;
+  float* lse2 = ws_f;                                                             // [n_req][H][obs]
   // the pairs start on a 256-byte boundary behind the log-sum-exp values
-  float2* partial = reinterpret_cast<float2*>(ws_f + (((int64_t)b->n_req * H * window + 63) & ~(int64_t)63));  // [n_req][Hkv][n_kb][rows_max]
+  float2* partial = reinterpret_cast<float2*>(ws_f + (((int64_t)b->n_req * H * obs + 63) & ~(int64_t)63));  // [n_req][Hkv][n_kb][rows_max]
   const size_t smem = (size_t)(kCtaKeys + 2 * kMmaRows) * (d + 8) * sizeof(__nv_bfloat16);  // K block + two Q blocks
   {
     static std::atomic<uint64_t> smem_allowed{0};
@@ -509,23 +527,24 @@ static purekv_status launch_score_mma(const void* q, const void* k, float* c_out
   const float scale_log2 = scale * 1.4426950408889634f;
   dim3 grid((unsigned)((ml + kCtaKeys - 1) / kCtaKeys), (unsigned)Hkv, (unsigned)b->n_req);
   score_mma_partial_kernel<<<grid, kMmaThreads, smem, sm>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, b->cu_seqlens,
-                                                            window, H, Hkv, d, scale_log2, n_kb, rows_max, partial);
+                                                            obs, H, Hkv, d, scale_log2, n_kb, rows_max, partial);
   PK_CUDA(cudaGetLastError());
-  const int64_t n_lse = (int64_t)b->n_req * H * window;
-  score_lse_merge_kernel<<<(unsigned)((n_lse + 255) / 256), 256, 0, sm>>>(partial, b->cu_seqlens, window, H, Hkv, n_kb,
+  const int64_t n_lse = (int64_t)b->n_req * H * obs;
+  score_lse_merge_kernel<<<(unsigned)((n_lse + 255) / 256), 256, 0, sm>>>(partial, b->cu_seqlens, obs, H, Hkv, n_kb,
                                                                          rows_max, b->n_req, lse2);
   PK_CUDA(cudaGetLastError());
   score_mma_colsum_kernel<<<grid, kMmaThreads, smem, sm>>>((const __nv_bfloat16*)q, (const __nv_bfloat16*)k, b->cu_seqlens,
-                                                           window, H, Hkv, d, scale_log2, lse2, b->total_tokens, c_out);
+                                                           window, obs, H, Hkv, d, scale_log2, lse2, b->total_tokens, c_out);
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
 }
 
 template <typename T>
 static purekv_status launch_score(const void* q, const void* k, float* c_out, const purekv_batch* b, int32_t window,
-                                  int32_t H, int32_t Hkv, int32_t d, float scale, float* lse2, cudaStream_t sm) {
+                                  int32_t obs, int32_t H, int32_t Hkv, int32_t d, float scale, float* lse2,
+                                  cudaStream_t sm) {
   const int32_t ml = max_len(b);
-  const int32_t w = std::min(window, ml);
+  const int32_t w = std::min(obs, ml);  // accumulated rows per head: the row blocks of the first pass
   const int32_t G = H / Hkv;
   const size_t smem = (size_t)(kRB + kKB) * (d + 4) * sizeof(float);
   {
@@ -540,14 +559,45 @@ static purekv_status launch_score(const void* q, const void* k, float* c_out, co
   }
   const float scale_log2 = scale * 1.4426950408889634f;
   dim3 g1((unsigned)((G * w + kRB - 1) / kRB), (unsigned)Hkv, (unsigned)b->n_req);
-  score_lse_kernel<T><<<g1, kThreads, smem, sm>>>((const T*)q, (const T*)k, b->cu_seqlens, window, H, Hkv, d, scale_log2,
+  score_lse_kernel<T><<<g1, kThreads, smem, sm>>>((const T*)q, (const T*)k, b->cu_seqlens, obs, H, Hkv, d, scale_log2,
                                                   lse2);
   PK_CUDA(cudaGetLastError());
   dim3 g2((unsigned)((ml + kKB - 1) / kKB), (unsigned)Hkv, (unsigned)b->n_req);
-  score_colsum_kernel<T><<<g2, kThreads, smem, sm>>>((const T*)q, (const T*)k, b->cu_seqlens, window, H, Hkv, d,
+  score_colsum_kernel<T><<<g2, kThreads, smem, sm>>>((const T*)q, (const T*)k, b->cu_seqlens, window, obs, H, Hkv, d,
                                                      scale_log2, lse2, b->total_tokens, c_out);
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
+}
+
+// Average pooling of the scores along the key axis (the pooled observation window of App. A.1's policies): each
+// non-recent key takes the mean over `pool` positions centred on it, positions outside the non-recent segment
+// counting as zero.  grid (key blocks of 256 over the longest request, n_kv_heads, n_req).
+__global__ void __launch_bounds__(256) score_pool_kernel(const float* __restrict__ c_in, const int32_t* __restrict__ cu_seqlens,
+                                                         int32_t window, int32_t pool, int64_t n_tokens,
+                                                         float* __restrict__ c_out) {
+  const int32_t r = blockIdx.z, g = blockIdx.y, j = blockIdx.x * 256 + threadIdx.x;
+  const int32_t base = cu_seqlens[r], len = cu_seqlens[r + 1] - base;
+  if (j >= len) return;
+  const int32_t nr = len - min(window, len), half = pool / 2;
+  const float* in = c_in + (int64_t)g * n_tokens + base;
+  float sum = 0.f;
+  if (j < nr)
+    for (int32_t jj = max(0, j - half); jj <= min(nr - 1, j + half); ++jj) sum += in[jj];
+  c_out[(int64_t)g * n_tokens + base + j] = sum / (float)(2 * half + 1);
+}
+
+// the last `obs` rows of every request are accumulated; < 0 or beyond the longest request: all rows
+static int32_t obs_stride(const purekv_batch* b, int32_t obs_rows) {
+  const int32_t ml = std::max(max_len(b), 1);
+  return (obs_rows < 0 || obs_rows > ml) ? ml : std::max(obs_rows, 1);
+}
+
+// floats of log-sum-exp values per (request, head, accumulated row), plus (max, sum) pairs per 64-key block for
+// the tensor-core path
+static size_t score_ws_floats(const purekv_batch* batch, int32_t obs, int32_t n_q_heads) {
+  const size_t rows = (size_t)batch->n_req * n_q_heads * (size_t)std::max(obs, 1);
+  const size_t n_kb = ((size_t)max_len(batch) + kMmaKeys - 1) / kMmaKeys;
+  return ((rows + 63) & ~(size_t)63) + rows * 2 * n_kb;
 }
 
 }  // namespace purekv
@@ -556,38 +606,73 @@ using namespace purekv;
 
 extern "C" size_t purekv_score_ws_bytes(const purekv_batch* batch, int32_t window, int32_t n_q_heads) {
   if (!batch || window < 0 || n_q_heads < 0 || !batch->h_cu_seqlens) return 0;
-  // log-sum-exp per (request, head, window row), plus (max, sum) pairs per 64-key block for the tensor-core path
-  const size_t rows = (size_t)batch->n_req * n_q_heads * (size_t)std::max(window, 1);
-  const size_t n_kb = ((size_t)max_len(batch) + kMmaKeys - 1) / kMmaKeys;
-  return (((rows + 63) & ~(size_t)63) + rows * 2 * n_kb) * sizeof(float) + 256;
+  return score_ws_floats(batch, window, n_q_heads) * sizeof(float) + 256;
+}
+
+extern "C" size_t purekv_score_ex_ws_bytes(const purekv_batch* batch, int32_t obs_rows, int32_t pool, int32_t n_q_heads,
+                                           int32_t n_kv_heads) {
+  if (!batch || n_q_heads < 0 || n_kv_heads < 0 || !batch->h_cu_seqlens) return 0;
+  size_t floats = score_ws_floats(batch, obs_stride(batch, obs_rows), n_q_heads);
+  if (pool > 1) floats += (((size_t)n_kv_heads * batch->total_tokens) + 63) & ~(size_t)63;  // the scores before pooling
+  return floats * sizeof(float) + 256;
+}
+
+// Common body of the score entry points: `obs_rows` accumulated rows (Eq. 2: the window), then pooling.
+static purekv_status score_impl(const char* who, const void* q, const void* k, float* c_out, const purekv_batch* batch,
+                                int32_t window, int32_t obs_rows, int32_t pool, int32_t n_q_heads, int32_t n_kv_heads,
+                                int32_t head_dim, purekv_dtype dtype, float softmax_scale, void* ws, size_t ws_bytes,
+                                size_t ws_need, void* stream) {
+  purekv_status st = check_batch(batch, true);
+  if (st != PUREKV_OK) return st;
+  if (batch->total_tokens == 0 || batch->n_req == 0) return PUREKV_OK;  // empty batch: nothing to do
+  PK_REQUIRE(q && k && c_out, PUREKV_ERR_INVALID_ARG, "%s: null pointer", who);
+  PK_REQUIRE(n_q_heads >= 1 && n_kv_heads >= 1 && n_q_heads % n_kv_heads == 0, PUREKV_ERR_INVALID_ARG,
+             "n_q_heads %d must be a positive multiple of n_kv_heads %d", n_q_heads, n_kv_heads);
+  PK_REQUIRE(window >= 1, PUREKV_ERR_INVALID_ARG, "window must be >= 1");
+  PK_REQUIRE(pool >= 1 && pool % 2 == 1, PUREKV_ERR_INVALID_ARG, "pool %d must be odd and >= 1", pool);
+  PK_REQUIRE(head_dim >= 4 && head_dim % 4 == 0 && head_dim <= 256, PUREKV_ERR_UNSUPPORTED,
+             "head_dim %d: need a multiple of 4 up to 256", head_dim);
+  PK_REQUIRE(dtype == PUREKV_BF16 || dtype == PUREKV_FP32, PUREKV_ERR_INVALID_ARG, "unknown dtype");
+  PK_REQUIRE(n_kv_heads <= 65535 && batch->n_req <= 65535, PUREKV_ERR_UNSUPPORTED, "too many heads or requests");
+  PK_REQUIRE(ws && ws_bytes >= ws_need, PUREKV_ERR_WORKSPACE, "%s: workspace of %zu bytes is too small (need %zu)", who,
+             ws_bytes, ws_need);
+  const int32_t obs = obs_stride(batch, obs_rows);
+  float* lse2 = (float*)(((uintptr_t)ws + 255) & ~(uintptr_t)255);
+  float* c_raw = pool > 1 ? lse2 + score_ws_floats(batch, obs, n_q_heads) : c_out;  // scores before pooling
+  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+  cudaStream_t sm = (cudaStream_t)stream;
+  if (dtype == PUREKV_BF16 && head_dim % 16 == 0)
+    st = launch_score_mma(q, k, c_raw, batch, window, obs, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
+  else if (dtype == PUREKV_BF16)
+    st = launch_score<__nv_bfloat16>(q, k, c_raw, batch, window, obs, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
+  else
+    st = launch_score<float>(q, k, c_raw, batch, window, obs, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
+  if (st != PUREKV_OK || pool == 1) return st;
+  dim3 grid((unsigned)((max_len(batch) + 255) / 256), (unsigned)n_kv_heads, (unsigned)batch->n_req);
+  score_pool_kernel<<<grid, 256, 0, sm>>>(c_raw, batch->cu_seqlens, window, pool, batch->total_tokens, c_out);
+  PK_CUDA(cudaGetLastError());
+  return PUREKV_OK;
 }
 
 extern "C" purekv_status purekv_lowlayer_score(const void* q, const void* k, float* c_out, const purekv_batch* batch,
                                                int32_t window, int32_t n_q_heads, int32_t n_kv_heads,
                                                int32_t head_dim, purekv_dtype dtype, float softmax_scale, void* ws,
                                                size_t ws_bytes, void* stream) {
-  purekv_status st = check_batch(batch, true);
-  if (st != PUREKV_OK) return st;
-  if (batch->total_tokens == 0 || batch->n_req == 0) return PUREKV_OK;  // empty batch: nothing to do
-  PK_REQUIRE(q && k && c_out, PUREKV_ERR_INVALID_ARG, "purekv_lowlayer_score: null pointer");
-  PK_REQUIRE(n_q_heads >= 1 && n_kv_heads >= 1 && n_q_heads % n_kv_heads == 0, PUREKV_ERR_INVALID_ARG,
-             "n_q_heads %d must be a positive multiple of n_kv_heads %d", n_q_heads, n_kv_heads);
-  PK_REQUIRE(window >= 1, PUREKV_ERR_INVALID_ARG, "window must be >= 1");
-  PK_REQUIRE(head_dim >= 4 && head_dim % 4 == 0 && head_dim <= 256, PUREKV_ERR_UNSUPPORTED,
-             "head_dim %d: need a multiple of 4 up to 256", head_dim);
-  PK_REQUIRE(dtype == PUREKV_BF16 || dtype == PUREKV_FP32, PUREKV_ERR_INVALID_ARG, "unknown dtype");
-  PK_REQUIRE(n_kv_heads <= 65535 && batch->n_req <= 65535, PUREKV_ERR_UNSUPPORTED, "too many heads or requests");
-  if (batch->n_req == 0 || batch->total_tokens == 0) return PUREKV_OK;
-  PK_REQUIRE(ws && ws_bytes >= purekv_score_ws_bytes(batch, window, n_q_heads), PUREKV_ERR_WORKSPACE,
-             "purekv_lowlayer_score: workspace of %zu bytes is too small", ws_bytes);
-  float* lse2 = (float*)(((uintptr_t)ws + 255) & ~(uintptr_t)255);
-  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
-  cudaStream_t sm = (cudaStream_t)stream;
-  if (dtype == PUREKV_BF16 && head_dim % 16 == 0)
-    return launch_score_mma(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
-  if (dtype == PUREKV_BF16)
-    return launch_score<__nv_bfloat16>(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
-  return launch_score<float>(q, k, c_out, batch, window, n_q_heads, n_kv_heads, head_dim, scale, lse2, sm);
+  if (batch && batch->h_cu_seqlens && window >= 1 && n_q_heads >= 1)
+    return score_impl("purekv_lowlayer_score", q, k, c_out, batch, window, window, 1, n_q_heads, n_kv_heads, head_dim, dtype,
+                      softmax_scale, ws, ws_bytes, purekv_score_ws_bytes(batch, window, n_q_heads), stream);
+  return score_impl("purekv_lowlayer_score", q, k, c_out, batch, window, window, 1, n_q_heads, n_kv_heads, head_dim, dtype,
+                    softmax_scale, ws, ws_bytes, 0, stream);
+}
+
+extern "C" purekv_status purekv_lowlayer_score_ex(const void* q, const void* k, float* c_out, const purekv_batch* batch,
+                                                  int32_t window, int32_t obs_rows, int32_t pool, int32_t n_q_heads,
+                                                  int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                                  float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
+  const size_t need = (batch && batch->h_cu_seqlens && n_q_heads >= 1 && n_kv_heads >= 1)
+                          ? purekv_score_ex_ws_bytes(batch, obs_rows, pool, n_q_heads, n_kv_heads) : 0;
+  return score_impl("purekv_lowlayer_score_ex", q, k, c_out, batch, window, obs_rows, pool, n_q_heads, n_kv_heads, head_dim,
+                    dtype, softmax_scale, ws, ws_bytes, need, stream);
 }
 
 // Device address of the static scratch array on the current device; resolved on the first call per device.

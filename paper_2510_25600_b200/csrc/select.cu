@@ -298,9 +298,45 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   }
 }
 
+// Attention sinks + recent window: one CTA per (request, KV head, layer) writes 0 .. h-1 and l-w .. l-1.
+__global__ void __launch_bounds__(256) sink_recent_kernel(const int32_t* __restrict__ cu_seqlens,
+                                                          const int32_t* __restrict__ cu_kept,
+                                                          const int32_t* __restrict__ keep, int32_t window, int32_t k_tot,
+                                                          int32_t n_kv_heads, int32_t* __restrict__ idx_out) {
+  const int32_t r = blockIdx.x, g = blockIdx.y, layer = blockIdx.z;
+  const int32_t len = cu_seqlens[r + 1] - cu_seqlens[r];
+  const int32_t w = min(window, len), h = keep[r];
+  int32_t* out = idx_out + ((int64_t)layer * n_kv_heads + g) * k_tot + cu_kept[r];
+  for (int32_t t = threadIdx.x; t < h + w; t += 256) out[t] = t < h ? t : len - w + (t - h);
+}
+
 }  // namespace purekv
 
 using namespace purekv;
+
+extern "C" purekv_status purekv_select_sink_recent(const purekv_batch* batch, int32_t window, const int32_t* keep,
+                                                   const int32_t* h_keep, const int32_t* cu_kept, const int32_t* h_cu_kept,
+                                                   int32_t n_layers, int32_t n_kv_heads, int32_t* idx_out, void* stream) {
+  purekv_status st = check_batch(batch, true);
+  if (st != PUREKV_OK) return st;
+  if (batch->total_tokens == 0 || batch->n_req == 0 || n_layers == 0) return PUREKV_OK;
+  PK_REQUIRE(keep && h_keep && cu_kept && h_cu_kept && idx_out, PUREKV_ERR_INVALID_ARG, "purekv_select_sink_recent: null pointer");
+  PK_REQUIRE(n_layers >= 0 && n_layers <= 65535 && n_kv_heads >= 1 && n_kv_heads <= 65535 && window >= 0,
+             PUREKV_ERR_INVALID_ARG, "purekv_select_sink_recent: bad sizes");
+  PK_REQUIRE(h_cu_kept[0] == 0, PUREKV_ERR_INVALID_ARG, "cu_kept[0] must be 0");
+  for (int r = 0; r < batch->n_req; ++r) {
+    const int32_t len = batch->h_cu_seqlens[r + 1] - batch->h_cu_seqlens[r];
+    const int32_t w = std::min(window, len);
+    PK_REQUIRE(h_keep[r] >= 0 && h_keep[r] <= len - w && h_cu_kept[r + 1] - h_cu_kept[r] == h_keep[r] + w,
+               PUREKV_ERR_INVALID_ARG, "request %d: h = %d must lie in [0, %d] and its kept count be h + w", r, h_keep[r],
+               len - w);
+  }
+  dim3 grid((unsigned)batch->n_req, (unsigned)n_kv_heads, (unsigned)n_layers);
+  sink_recent_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>(batch->cu_seqlens, cu_kept, keep, window,
+                                                             h_cu_kept[batch->n_req], n_kv_heads, idx_out);
+  PK_CUDA(cudaGetLastError());
+  return PUREKV_OK;
+}
 
 extern "C" size_t purekv_select_ws_bytes(const purekv_batch* batch, int32_t n_layers, int32_t n_kv_heads) {
   if (!batch || n_layers < 0 || n_kv_heads < 0) return 0;
