@@ -416,6 +416,8 @@ def compression_detail(pipe, wl, d_in, peaks, timer):
                                                   idx_out=pipe.idx, ws=pipe.select_ws))
     t_compact = timer(lambda: P.purekv_compact_kv(k[lo:hi], v[lo:hi], pipe.idx, pipe.batch, pipe.budget,
                                                   k_out=pipe.k_c, v_out=pipe.v_c))
+    t_fused = timer(lambda: P.purekv_select_compact(pipe.c[len(pipe.scored) - 1], k[lo:hi], v[lo:hi], pipe.batch, pipe.budget,
+                                                    idx_out=pipe.idx, k_out=pipe.k_c, v_out=pipe.v_c, ws=pipe.select_ws))
     row = wl.n_kv_heads * wl.head_dim * esz
     kt = pipe.budget.total_kept
     w_rows = sum(min(wl.window, int(l)) for l in b.seq_lens)
@@ -429,6 +431,8 @@ def compression_detail(pipe, wl, d_in, peaks, timer):
                             kernel="one pass, tcgen05, from the prefill's log-sum-exp" if pipe.one_pass_scores else "two passes"),
               "select": hbm_rec(t_select, bytes_select, peaks),
               "compact": hbm_rec(t_compact, bytes_compact, peaks),
+              "select_compact_one_call": dict(hbm_rec(t_fused, bytes_select + bytes_compact - nc * wl.n_kv_heads * kt * 4, peaks),
+                                              separate_calls_ms=t_select + t_compact),
               "hbm_peak_GBps": float(peaks["hbm_gbs"]), "timing": "cold L2 (256 MiB flush before each call), median of 5"}
     # what the compact cache is for: one decode step (one new query per request) over all compacted layers,
     # one call per layer; not part of the timed step or of `value`
@@ -652,6 +656,7 @@ def sub_ragged(reps, peaks, timer):
     t_sel = timer(lambda: P.purekv_select_topk(c, vv, db, bud, idx_out=idx, ws=ws_sel))
     kc, vc = P.purekv_compact_kv(kk, vv, idx, db, bud)
     t_cmp = timer(lambda: P.purekv_compact_kv(kk, vv, idx, db, bud, k_out=kc, v_out=vc))
+    t_fused = timer(lambda: P.purekv_select_compact(c, kk, vv, db, bud, idx_out=idx, k_out=kc, v_out=vc, ws=ws_sel))
     P.purekv_poll_status(status)
     kt = bud.total_kept
     w_rows = sum(min(wl.window, int(l)) for l in b.seq_lens)
@@ -663,6 +668,8 @@ def sub_ragged(reps, peaks, timer):
                          kernel="one pass (tcgen05)" if one_pass else "two passes"),
            "select": hbm_rec(t_sel, nc * (tokens * row + wl.n_kv_heads * tokens * 4 + wl.n_kv_heads * kt * 4), peaks),
            "compact": hbm_rec(t_cmp, nc * (4 * kt * row + wl.n_kv_heads * kt * 4), peaks),
+           "select_compact_one_call": dict(hbm_rec(t_fused, nc * (tokens * row + wl.n_kv_heads * tokens * 4 + 4 * kt * row +
+                                                                   wl.n_kv_heads * kt * 4), peaks), separate_calls_ms=t_sel + t_cmp),
            "compression_clocks": sampler.stop(), "timing": "cold L2 (256 MiB fill before each call), median"}
     return rec
 

@@ -253,6 +253,20 @@ purekv_status purekv_select_topk(const float *c, const void *v, int64_t v_layer_
                                  purekv_dtype dtype, int32_t *idx_out, float *s_out, void *ws,
                                  size_t ws_bytes, void *stream);
 
+/* ---- selection and compaction in one call (Sec. 3.1: the selection feeds the compressed cache directly) ----
+ * purekv_select_topk followed by purekv_compact_kv of the same layers, in the selection's own kernels: the CTA
+ * that has chosen a (request, KV head, layer) segment's positions copies those K and V rows (k and v share
+ * layer_stride) into k_out / v_out [n_layers][K_tot, H_kv, d] (out_layer_stride) -- one launch fewer, and the
+ * indices do not travel through memory between two kernels.  idx_out (and s_out, if given) are written as by
+ * purekv_select_topk; results are bit-identical to the two separate calls. */
+purekv_status purekv_select_compact(const float *c, const void *k, const void *v, int64_t layer_stride,
+                                    int32_t n_layers, const purekv_batch *batch, int32_t window,
+                                    const int32_t *keep /* device [n_req] */, const int32_t *h_keep,
+                                    const int32_t *cu_kept /* device [n_req+1] */, const int32_t *h_cu_kept,
+                                    int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype, int32_t *idx_out,
+                                    float *s_out, void *k_out, void *v_out, int64_t out_layer_stride, void *ws,
+                                    size_t ws_bytes, void *stream);
+
 /* ---- compaction (the compressed cache of Sec. 3.1) -------------------------------------
  * k_out[L, cu_kept[r]+t, g, :] = k[L, cu_seqlens[r] + idx[L, g, cu_kept[r]+t], g, :], same for v.
  * k, v: [n_layers][T, H_kv, d] with layer_stride elements between layers; outputs

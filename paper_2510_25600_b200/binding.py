@@ -31,7 +31,7 @@ EXPORTS = ("purekv_version", "purekv_last_error", "purekv_budget", "purekv_plan_
            "purekv_select_ws_bytes",
            "purekv_select_topk", "purekv_compact_kv", "purekv_decode_ws_bytes", "purekv_decode_attention",
            "purekv_poll_status", "purekv_set_wait_limit_ns", "purekv_score_ex_ws_bytes", "purekv_lowlayer_score_ex",
-           "purekv_select_sink_recent")
+           "purekv_select_sink_recent", "purekv_select_compact")
 
 _i32p = C.POINTER(C.c_int32)
 
@@ -107,6 +107,9 @@ _lib.purekv_select_ws_bytes.argtypes = [C.POINTER(CBatch), C.c_int32, C.c_int32]
 _lib.purekv_select_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.POINTER(CBatch), C.c_int32,
                                     C.c_void_p, _i32p, C.c_void_p, _i32p, C.c_int32, C.c_int32, C.c_int, C.c_void_p,
                                     C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+_lib.purekv_select_compact.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.POINTER(CBatch), C.c_int32,
+                                       C.c_void_p, _i32p, C.c_void_p, _i32p, C.c_int32, C.c_int32, C.c_int, C.c_void_p,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
 _lib.purekv_compact_kv.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.POINTER(CBatch),
                                    C.c_void_p, _i32p, C.c_int32, C.c_int32, C.c_int, C.c_void_p, C.c_void_p,
                                    C.c_int64, C.c_void_p]
@@ -366,6 +369,30 @@ def purekv_select_topk(c: torch.Tensor, v: torch.Tensor, batch: Batch, budget: B
                                    _dtype_code(v), idx_out.data_ptr(), _ptr(s_out), _ptr(ws),
                                    0 if ws is None else ws.numel(), _stream()), "purekv_select_topk")
     return idx_out
+
+
+def purekv_select_compact(c: torch.Tensor, k: torch.Tensor, v: torch.Tensor, batch: Batch, budget: Budget,
+                          idx_out: Optional[torch.Tensor] = None, s_out: Optional[torch.Tensor] = None,
+                          k_out: Optional[torch.Tensor] = None, v_out: Optional[torch.Tensor] = None,
+                          ws: Optional[torch.Tensor] = None):
+    """Selection and compaction in one call.  c [H_kv,T]; k, v [L,T,H_kv,d]; returns (idx, k_c, v_c)."""
+    assert k.dim() == 4 and k[0].is_contiguous() and v[0].is_contiguous() and k.stride(0) == v.stride(0) and c.is_contiguous()
+    n_layers, t, hkv, d = v.shape
+    if idx_out is None:
+        idx_out = torch.empty((n_layers, hkv, budget.total_kept), dtype=torch.int32, device=v.device)
+    if k_out is None:
+        k_out = torch.empty((n_layers, budget.total_kept, hkv, d), dtype=k.dtype, device=k.device)
+    if v_out is None:
+        v_out = torch.empty_like(k_out)
+    if s_out is None and ws is None:
+        ws = torch.empty(purekv_select_ws_bytes(batch, n_layers, hkv), dtype=torch.uint8, device=v.device)
+    _check(_lib.purekv_select_compact(c.data_ptr(), k.data_ptr(), v.data_ptr(), v.stride(0), n_layers, C.byref(batch.c),
+                                      budget.window, budget.keep.data_ptr(), budget.h_keep.ctypes.data_as(_i32p),
+                                      budget.cu_kept.data_ptr(), budget.h_cu_kept.ctypes.data_as(_i32p), hkv, d,
+                                      _dtype_code(v), idx_out.data_ptr(), _ptr(s_out), k_out.data_ptr(), v_out.data_ptr(),
+                                      k_out.stride(0), _ptr(ws), 0 if ws is None else ws.numel(), _stream()),
+           "purekv_select_compact")
+    return idx_out, k_out, v_out
 
 
 def purekv_compact_kv(k: torch.Tensor, v: torch.Tensor, idx: torch.Tensor, batch: Batch, budget: Budget,

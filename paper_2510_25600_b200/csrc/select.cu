@@ -109,11 +109,21 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 constexpr int kSelThreads = 512;
 constexpr int kSelItems = 4;
 
+// What the selecting CTA needs to also gather its segment's kept rows into the compact cache (Sec. 3.1: the selection
+// feeds the compressed cache directly); k_src == nullptr: selection only.  Rows are `cpr` 16-byte chunks; layer
+// strides in chunks.
+struct Gather {
+  const uint4 *k_src, *v_src;
+  uint4 *k_dst, *v_dst;
+  int64_t src_layer_stride_c, dst_layer_stride_c;
+  int32_t cpr;
+};
+
 // One CTA per (request, KV head, layer).  FUSED = false: the scores come from `s` (written by vnorm_score_kernel).
 // FUSED = true: the CTA first streams its own segment of V (256-byte rows), forms S = C * ||V|| into shared memory
 // (and into s_out if asked), and selects from there, so V is the only large read and S never makes a round trip;
 // used when there are enough segments to keep every SM streaming.
-template <bool FUSED, typename T>
+template <bool FUSED, typename T, bool GATHER = false>
 __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __restrict__ s, int64_t n_tokens,
                                                              const int32_t* __restrict__ cu_seqlens,
                                                              const int32_t* __restrict__ cu_kept,
@@ -121,7 +131,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
                                                              int32_t k_tot, int32_t n_kv_heads,
                                                              int32_t* __restrict__ idx_out, const uint4* __restrict__ v,
                                                              int64_t layer_stride_c, const float* __restrict__ c,
-                                                             float* __restrict__ s_out) {
+                                                             float* __restrict__ s_out, Gather ga) {
   extern __shared__ uint32_t skeys[];  // FUSED: order keys of the segment's non-recent scores
   __shared__ int32_t hist[256];
   __shared__ uint32_t sh_prefix;
@@ -194,7 +204,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
     __syncthreads();
   }
   auto key_at = [&](int32_t j) -> uint32_t { return staged ? skeys[j] : order_key(__ldg(seg + j)); };
-  if (h <= 0) return;
+  if (h > 0) {
 
   // ---- radix select: the h-th largest key --------------------------------------------
   uint32_t prefix = 0, mask = 0;
@@ -296,6 +306,44 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
     if (tid == kSelThreads - 1) { carry_gt = pos_gt; carry_eq = pos_eq; }
     __syncthreads();
   }
+  }  // h > 0
+
+  // ---- gather (optional): the CTA copies the rows it has just chosen, K and V, into the compact cache ----------
+  if constexpr (GATHER) {
+    __syncthreads();  // every index of the segment (written above by this CTA's threads) is visible to all of them
+    const int32_t n_keep = h + w, cpr = ga.cpr, rows_per_step = kSelThreads / cpr;
+    const int32_t ch = tid % cpr, r_in = tid / cpr;
+    const uint4* ks = ga.k_src + layer * ga.src_layer_stride_c;
+    const uint4* vs = ga.v_src + layer * ga.src_layer_stride_c;
+    uint4* kd = ga.k_dst + layer * ga.dst_layer_stride_c;
+    uint4* vd = ga.v_dst + layer * ga.dst_layer_stride_c;
+    const int32_t dst0 = cu_kept[r];
+    if (r_in < rows_per_step) {
+      // four rows of K and of V per thread in flight
+      constexpr int kU = 4;
+      for (int32_t t0 = r_in; t0 < n_keep; t0 += kU * rows_per_step) {
+        uint4 kk[kU], vv[kU];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+          const int32_t t = t0 + u * rows_per_step;
+          if (t < n_keep) {
+            const int64_t src = ((int64_t)(base + out[t]) * n_kv_heads + g) * cpr + ch;
+            kk[u] = ks[src];
+            vv[u] = vs[src];
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+          const int32_t t = t0 + u * rows_per_step;
+          if (t < n_keep) {
+            const int64_t dst = ((int64_t)(dst0 + t) * n_kv_heads + g) * cpr + ch;
+            kd[dst] = kk[u];
+            vd[dst] = vv[u];
+          }
+        }
+      }
+    }
+  }
 }
 
 // Attention sinks + recent window: one CTA per (request, KV head, layer) writes 0 .. h-1 and l-w .. l-1.
@@ -343,11 +391,12 @@ extern "C" size_t purekv_select_ws_bytes(const purekv_batch* batch, int32_t n_la
   return (size_t)n_layers * n_kv_heads * batch->total_tokens * sizeof(float) + 256;
 }
 
-extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64_t v_layer_stride, int32_t n_layers,
-                                            const purekv_batch* batch, int32_t window, const int32_t* keep,
-                                            const int32_t* h_keep, const int32_t* cu_kept, const int32_t* h_cu_kept,
-                                            int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
-                                            int32_t* idx_out, float* s_out, void* ws, size_t ws_bytes, void* stream) {
+// Common body of purekv_select_topk and purekv_select_compact (ga.k_src != nullptr: the selecting CTAs also gather).
+static purekv_status select_impl(const float* c, const void* v, int64_t v_layer_stride, int32_t n_layers,
+                                 const purekv_batch* batch, int32_t window, const int32_t* keep, const int32_t* h_keep,
+                                 const int32_t* cu_kept, const int32_t* h_cu_kept, int32_t n_kv_heads, int32_t head_dim,
+                                 purekv_dtype dtype, int32_t* idx_out, float* s_out, void* ws, size_t ws_bytes,
+                                 void* stream, Gather ga) {
   purekv_status st = check_batch(batch, true);
   if (st != PUREKV_OK) return st;
   if (batch->total_tokens == 0 || batch->n_req == 0) return PUREKV_OK;  // empty batch: nothing to do
@@ -385,27 +434,21 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
   const size_t key_bytes = (size_t)longest * sizeof(uint32_t);
   const int64_t segments = (int64_t)batch->n_req * n_kv_heads * n_layers;
   if (cpr == 16 && key_bytes <= 200 * 1024 && segments >= 2 * 148) {
-    if (dtype == PUREKV_BF16) {
-      {
-        static std::atomic<uint64_t> smem_allowed{0};
-        const purekv_status st_smem = allow_max_dynamic_smem(select_kernel<true, __nv_bfloat16>, smem_allowed);
-        if (st_smem != PUREKV_OK) return st_smem;
-      }
-      select_kernel<true, __nv_bfloat16><<<g2, kSelThreads, key_bytes, sm>>>(
-          nullptr, T, batch->cu_seqlens, cu_kept, keep, window, k_tot, n_kv_heads, idx_out, (const uint4*)v,
-          v_layer_stride * esz / 16, c, s_out);
-    } else {
-      {
-        static std::atomic<uint64_t> smem_allowed{0};
-        const purekv_status st_smem = allow_max_dynamic_smem(select_kernel<true, float>, smem_allowed);
-        if (st_smem != PUREKV_OK) return st_smem;
-      }
-      select_kernel<true, float><<<g2, kSelThreads, key_bytes, sm>>>(nullptr, T, batch->cu_seqlens, cu_kept, keep, window,
-                                                                     k_tot, n_kv_heads, idx_out, (const uint4*)v,
-                                                                     v_layer_stride * esz / 16, c, s_out);
-    }
-    PK_CUDA(cudaGetLastError());
-    return PUREKV_OK;
+    auto launch_fused = [&](auto kernel, std::atomic<uint64_t>& smem_allowed) -> purekv_status {
+      const purekv_status st_smem = allow_max_dynamic_smem(kernel, smem_allowed);
+      if (st_smem != PUREKV_OK) return st_smem;
+      kernel<<<g2, kSelThreads, key_bytes, sm>>>(nullptr, T, batch->cu_seqlens, cu_kept, keep, window, k_tot, n_kv_heads,
+                                                 idx_out, (const uint4*)v, v_layer_stride * esz / 16, c, s_out, ga);
+      PK_CUDA(cudaGetLastError());
+      return PUREKV_OK;
+    };
+    static std::atomic<uint64_t> allowed[4] = {{0}, {0}, {0}, {0}};
+    const bool gather = ga.k_src != nullptr;
+    if (dtype == PUREKV_BF16)
+      return gather ? launch_fused(select_kernel<true, __nv_bfloat16, true>, allowed[0])
+                    : launch_fused(select_kernel<true, __nv_bfloat16, false>, allowed[1]);
+    return gather ? launch_fused(select_kernel<true, float, true>, allowed[2])
+                  : launch_fused(select_kernel<true, float, false>, allowed[3]);
   }
   float* s_buf = s_out;
   if (!s_buf) {
@@ -423,12 +466,13 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
                                                   cpr, s_buf);
   PK_CUDA(cudaGetLastError());
   const bool stage_keys = key_bytes <= 200 * 1024;
-  if (stage_keys)
-    {
-      static std::atomic<uint64_t> smem_allowed{0};
-      const purekv_status st_smem = allow_max_dynamic_smem(select_kernel<false, float>, smem_allowed);
-      if (st_smem != PUREKV_OK) return st_smem;
-    }
+  const bool gather = ga.k_src != nullptr;
+  if (stage_keys) {
+    static std::atomic<uint64_t> smem_allowed{0}, smem_allowed_g{0};
+    const purekv_status st_smem = gather ? allow_max_dynamic_smem(select_kernel<false, float, true>, smem_allowed_g)
+                                         : allow_max_dynamic_smem(select_kernel<false, float, false>, smem_allowed);
+    if (st_smem != PUREKV_OK) return st_smem;
+  }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = g2;
   cfg.blockDim = dim3(kSelThreads);
@@ -439,9 +483,50 @@ extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  PK_CUDA(cudaLaunchKernelEx(&cfg, select_kernel<false, float>, (const float*)s_buf, T, batch->cu_seqlens, cu_kept, keep,
-                             window, k_tot, n_kv_heads, idx_out, (const uint4*)nullptr, (int64_t)0, (const float*)nullptr,
-                             stage_keys ? s_buf : (float*)nullptr));
+  if (gather)
+    PK_CUDA(cudaLaunchKernelEx(&cfg, select_kernel<false, float, true>, (const float*)s_buf, T, batch->cu_seqlens, cu_kept,
+                               keep, window, k_tot, n_kv_heads, idx_out, (const uint4*)nullptr, (int64_t)0,
+                               (const float*)nullptr, stage_keys ? s_buf : (float*)nullptr, ga));
+  else
+    PK_CUDA(cudaLaunchKernelEx(&cfg, select_kernel<false, float, false>, (const float*)s_buf, T, batch->cu_seqlens, cu_kept,
+                               keep, window, k_tot, n_kv_heads, idx_out, (const uint4*)nullptr, (int64_t)0,
+                               (const float*)nullptr, stage_keys ? s_buf : (float*)nullptr, ga));
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
+}
+
+extern "C" purekv_status purekv_select_topk(const float* c, const void* v, int64_t v_layer_stride, int32_t n_layers,
+                                            const purekv_batch* batch, int32_t window, const int32_t* keep,
+                                            const int32_t* h_keep, const int32_t* cu_kept, const int32_t* h_cu_kept,
+                                            int32_t n_kv_heads, int32_t head_dim, purekv_dtype dtype,
+                                            int32_t* idx_out, float* s_out, void* ws, size_t ws_bytes, void* stream) {
+  return select_impl(c, v, v_layer_stride, n_layers, batch, window, keep, h_keep, cu_kept, h_cu_kept, n_kv_heads, head_dim,
+                     dtype, idx_out, s_out, ws, ws_bytes, stream, Gather{});
+}
+
+extern "C" purekv_status purekv_select_compact(const float* c, const void* k, const void* v, int64_t layer_stride,
+                                               int32_t n_layers, const purekv_batch* batch, int32_t window,
+                                               const int32_t* keep, const int32_t* h_keep, const int32_t* cu_kept,
+                                               const int32_t* h_cu_kept, int32_t n_kv_heads, int32_t head_dim,
+                                               purekv_dtype dtype, int32_t* idx_out, float* s_out, void* k_out,
+                                               void* v_out, int64_t out_layer_stride, void* ws, size_t ws_bytes,
+                                               void* stream) {
+  PK_REQUIRE(k && k_out && v_out, PUREKV_ERR_INVALID_ARG, "purekv_select_compact: null pointer");
+  PK_REQUIRE(dtype == PUREKV_BF16 || dtype == PUREKV_FP32, PUREKV_ERR_INVALID_ARG, "unknown dtype");
+  const int64_t esz = dtype == PUREKV_BF16 ? 2 : 4;
+  PK_REQUIRE(head_dim >= 1 && (head_dim * esz) % 16 == 0 && head_dim * esz / 16 <= kSelThreads, PUREKV_ERR_UNSUPPORTED,
+             "row of %lld bytes: need a multiple of 16 up to %d", (long long)(head_dim * esz), 16 * kSelThreads);
+  PK_REQUIRE((layer_stride * esz) % 16 == 0 && (out_layer_stride * esz) % 16 == 0 &&
+                 ((uintptr_t)k | (uintptr_t)v | (uintptr_t)k_out | (uintptr_t)v_out) % 16 == 0,
+             PUREKV_ERR_INVALID_ARG, "K/V bases and layer strides must be 16-byte aligned");
+  Gather ga;
+  ga.k_src = (const uint4*)k;
+  ga.v_src = (const uint4*)v;
+  ga.k_dst = (uint4*)k_out;
+  ga.v_dst = (uint4*)v_out;
+  ga.src_layer_stride_c = layer_stride * esz / 16;
+  ga.dst_layer_stride_c = out_layer_stride * esz / 16;
+  ga.cpr = (int32_t)(head_dim * esz / 16);
+  return select_impl(c, v, layer_stride, n_layers, batch, window, keep, h_keep, cu_kept, h_cu_kept, n_kv_heads, head_dim,
+                     dtype, idx_out, s_out, ws, ws_bytes, stream, ga);
 }

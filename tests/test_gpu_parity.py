@@ -170,7 +170,18 @@ def run_compress(wl, layers_x, window, keep):
     idx_ws = P.purekv_select_topk(c, vs, db, bud)          # workspace path must agree
     assert torch.equal(idx, idx_ws)
     kc, vc = P.purekv_compact_kv(ks, vs, idx, db, bud)
+    # selection and compaction in one call: the same indices and the same bytes (checked against the oracle below
+    # through kc / vc), with guard bands around the outputs
+    pad = 64
+    kf = torch.full((len(layers_x), bud.total_kept + 2 * pad, wl.n_kv_heads, wl.head_dim), 3.0, dtype=ks.dtype, device="cuda")
+    vf = torch.full_like(kf, 3.0)
+    idx_f, kc_f, vc_f = P.purekv_select_compact(c, ks, vs, db, bud, k_out=kf[:, pad:pad + bud.total_kept],
+                                                v_out=vf[:, pad:pad + bud.total_kept])
     torch.cuda.synchronize()
+    as_bits = lambda t: t.contiguous().view(torch.int16 if t.element_size() == 2 else torch.int32)
+    assert torch.equal(idx_f, idx) and torch.equal(as_bits(kc_f), as_bits(kc)) and torch.equal(as_bits(vc_f), as_bits(vc))
+    for t in (kf, vf):
+        assert (t[:, :pad] == 3.0).all() and (t[:, pad + bud.total_kept:] == 3.0).all(), "guard bands"
     return c, s, idx, kc, vc, bud
 
 

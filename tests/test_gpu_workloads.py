@@ -73,7 +73,10 @@ def check_scores_selection_compaction(wl, x0, layers_x, groups=None):
     s = torch.empty((len(layers_x), wl.n_kv_heads, db.total_tokens), dtype=torch.float32, device="cuda")
     idx = P.purekv_select_topk(c, vs, db, bud, s_out=s)
     kc, vc = P.purekv_compact_kv(ks, vs, idx, db, bud)
+    idx_f, kc_f, vc_f = P.purekv_select_compact(c, ks, vs, db, bud)      # one call: the same indices and bytes
     torch.cuda.synchronize()
+    assert torch.equal(idx_f, idx) and torch.equal(kc_f.view(torch.int16), kc.view(torch.int16))
+    assert torch.equal(vc_f.view(torch.int16), vc.view(torch.int16))
     c_gpu = c.cpu().numpy()
     hk, ck = po.budgets(b.seq_lens, wl.window, wl.keep_ratio)
     assert np.array_equal(hk, bud.h_keep) and np.array_equal(ck, bud.h_cu_kept)
