@@ -5,8 +5,10 @@
 // A CTA owns 128 keys of one (request, KV head) -- one key per TMEM lane -- and walks the stacked rows in blocks
 // of 128 columns: S^T = K Q_w^T with tcgen05.mma (A = the K tile, B = a block of window rows, both K-major from
 // shared memory, fp32 accumulators in TMEM, two buffers).  Roles:
-//   warp 0      producer: the K tile once, then per block of rows sixteen 8-row boxes per 64-column panel (a block
-//               of stacked rows may span several query heads; an 8-row box never does when w is a multiple of 8)
+//   warp 0      producer: the K tile once, then per block of rows 128 / B boxes of B rows per 64-column panel, B the
+//               largest power of two (at most 128) that divides every request's window: a block of stacked rows
+//               may span several query heads, a box of B rows never does (few large boxes: the copy engine's rate
+//               of small boxes bounded this kernel when the boxes were 8 rows high)
 //   warp 1      owns the TMEM columns; one lane issues the products
 //   warps 2-5   one thread per key: S^T row from TMEM, exp2 against the column's log-sum-exp, running sum
 // bf16, head_dim 128, window a multiple of 8.  Every wait is bounded; on expiry the status word is set.
@@ -35,9 +37,11 @@ struct __align__(8) Barriers {
 __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
     const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_q8, const float* __restrict__ lse,
     float* __restrict__ c_out, const int32_t* __restrict__ cu_seqlens, int32_t window, int32_t n_q_heads,
-    int32_t n_kv_heads, float scale_log2, int64_t n_tokens, int32_t* __restrict__ status, uint64_t wait_ns) {
+    int32_t n_kv_heads, float scale_log2, int64_t n_tokens, int32_t* __restrict__ status, uint64_t wait_ns,
+    int32_t box_rows) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ Barriers bars;
+  __shared__ __align__(16) float lse_s[4][2][kRows];  // per epilogue warp: the log-sum-exp values of two blocks of rows
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
   const int32_t r = blockIdx.z, g = blockIdx.y, j0 = blockIdx.x * kKeys;
@@ -56,6 +60,10 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
   const uint32_t sK = smem0;          // [2 panels][128 keys x 128 B]
   const uint32_t sQ = sK + kTile;     // [kStages][2 panels][128 rows x 128 B]
   const int32_t n_blocks = (n_rows + kRows - 1) / kRows;
+  // Every CTA of a (request, KV head) reads the same blocks of window rows, and CTAs of one wave run in step: started
+  // at the same block they would all pull the same lines from the same L2 slices at the same time.  Each CTA
+  // therefore starts its walk at a different block (the column sums do not depend on the order).
+  const int32_t rot = (int32_t)(blockIdx.x % (uint32_t)n_blocks);
   volatile int* abort_flag = &abort_s;
 
   if (tid == 0) {
@@ -94,15 +102,15 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
         const int32_t s = t % kStages;
         if (t >= kStages && !mbar_wait(smem_u32(&bars.q_empty[s]), ((t / kStages) - 1) & 1, abort_flag, wait_ns)) break;
         mbar_expect_tx(smem_u32(&bars.q_full[s]), kTile);
-        for (int32_t grp = 0; grp < kRows / 8; ++grp) {
-          const int32_t row = t * kRows + 8 * grp;
+        for (int32_t grp = 0; grp < kRows / box_rows; ++grp) {
+          const int32_t row = ((t + rot) % n_blocks) * kRows + box_rows * grp;
           // rows past the stacked list read from beyond the tensor: zero fill
           int32_t tok = (int32_t)n_tokens, head = 0;
           if (row < n_rows) {
             tok = base + len - w + row % w;
             head = g * G + row / w;
           }
-          const uint32_t dst = sQ + s * kTile + grp * 1024;
+          const uint32_t dst = sQ + s * kTile + grp * (box_rows * 128);
           tma_load_3d(dst, &tm_q8, smem_u32(&bars.q_full[s]), 0, head, tok);
           tma_load_3d(dst + kPanel, &tm_q8, smem_u32(&bars.q_full[s]), 64, head, tok);
         }
@@ -151,34 +159,55 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
     const float kLog2e = 1.4426950408889634f;
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     bool ok = true;
-    for (int32_t t = 0; ok && t < n_blocks; ++t) {
-      const int32_t b = t & 1;
-      // the block's log-sum-exp values (log2 units), lane i holding columns i, i+32, i+64, i+96; +inf for absent rows
-      float lv[4];
+    // The log-sum-exp of a block's 128 stacked rows (log2 units; +inf for absent rows): every key needs all of them.
+    // Each warp keeps its own copy in shared memory, fetched one block ahead (lane i loads rows i, i+32, i+64, i+96)
+    // and read back four at a time; no meeting between warps is needed.
+    float (*my_lse)[kRows] = lse_s[warp - 2];
+    auto fetch_lse = [&](int32_t t, float (&lv)[4]) {
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        const int32_t row = t * kRows + 32 * c + lane;
+        const int32_t row = ((t + rot) % n_blocks) * kRows + 32 * c + lane;
         lv[c] = INFINITY;
         if (row < n_rows)
           lv[c] = __ldg(lse + (int64_t)(g * G + row / w) * n_tokens + base + len - w + row % w) * kLog2e;
       }
+    };
+    float lv[4];
+    fetch_lse(0, lv);
+#pragma unroll
+    for (int c = 0; c < 4; ++c) my_lse[0][32 * c + lane] = lv[c];
+    __syncwarp();
+    for (int32_t t = 0; ok && t < n_blocks; ++t) {
+      const int32_t b = t & 1;
+      if (t + 1 < n_blocks) fetch_lse(t + 1, lv);  // in flight while this block is summed
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.d_full[b]), (t >> 1) & 1, abort_flag, wait_ns) ? 1 : 0) != 0;
       if (!ok) break;
       tc_fence_after();
+      const float4* l4 = reinterpret_cast<const float4*>(my_lse[b]);
+      // the next 32 columns are on their way from TMEM while the current ones go through the exponentials
+      uint32_t rr[2][32];
+      tmem_ld32(t_lane + b * kRows, rr[0]);
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
-        uint32_t rr[32];
-        tmem_ld32(t_lane + b * kRows + 32 * c, rr);
         tc_wait_ld();
+        if (c + 1 < 4) tmem_ld32(t_lane + b * kRows + 32 * (c + 1), rr[(c + 1) & 1]);
 #pragma unroll
-        for (int x = 0; x < 32; ++x) {
-          const float l = __shfl_sync(0xffffffffu, lv[c], x);
-          acc[x & 3] += ex2(fmaf(__uint_as_float(rr[x]), scale_log2, -l));
+        for (int x = 0; x < 32; x += 4) {
+          const float4 l = l4[8 * c + (x >> 2)];
+          acc[0] += ex2(fmaf(__uint_as_float(rr[c & 1][x]), scale_log2, -l.x));
+          acc[1] += ex2(fmaf(__uint_as_float(rr[c & 1][x + 1]), scale_log2, -l.y));
+          acc[2] += ex2(fmaf(__uint_as_float(rr[c & 1][x + 2]), scale_log2, -l.z));
+          acc[3] += ex2(fmaf(__uint_as_float(rr[c & 1][x + 3]), scale_log2, -l.w));
         }
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars.d_empty[b]));
+      if (t + 1 < n_blocks) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) my_lse[b ^ 1][32 * c + lane] = lv[c];  // last read two blocks ago by this warp
+        __syncwarp();
+      }
     }
     if (ok) {
       const int32_t j = j0 + key;
@@ -222,14 +251,22 @@ extern "C" purekv_status purekv_lowlayer_score_lse(const void* q, const void* k,
   for (int r = 0; r < batch->n_req; ++r) {
     const int32_t len = batch->h_cu_seqlens[r + 1] - batch->h_cu_seqlens[r];
     ml = std::max(ml, len);
-    // a request shorter than the window clips it; the clipped window must keep the 8-row boxes inside one head
+    // a request shorter than the window clips it; the clipped window must keep the boxes of rows inside one head
     PK_REQUIRE(len >= window || len % 8 == 0, PUREKV_ERR_UNSUPPORTED,
                "request %d: %d tokens, shorter than the window and not a multiple of 8", r, len);
+  }
+  // rows per box: the largest power of two up to 128 that divides the window of every request (clipped ones too)
+  int32_t box_rows = kRows;
+  while (window % box_rows) box_rows >>= 1;
+  for (int r = 0; r < batch->n_req; ++r) {
+    const int32_t len = batch->h_cu_seqlens[r + 1] - batch->h_cu_seqlens[r];
+    if (len > 0 && len < window)
+      while (len % box_rows) box_rows >>= 1;
   }
   const int64_t T = batch->total_tokens;
   CUtensorMap mk, mq8;
   if ((st = make_map(&mk, k, T, n_kv_heads, kKeys)) != PUREKV_OK) return st;
-  if ((st = make_map(&mq8, q, T, n_q_heads, 8)) != PUREKV_OK) return st;
+  if ((st = make_map(&mq8, q, T, n_q_heads, box_rows)) != PUREKV_OK) return st;
   if (!status) {
     const purekv_status st_w = default_status_word(&status);
     if (st_w != PUREKV_OK) return st_w;
@@ -243,7 +280,8 @@ extern "C" purekv_status purekv_lowlayer_score_lse(const void* q, const void* k,
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
   dim3 grid((unsigned)((ml + kKeys - 1) / kKeys), (unsigned)n_kv_heads, (unsigned)batch->n_req);
   score_tc_kernel<<<grid, kThreads, smem, (cudaStream_t)stream>>>(mk, mq8, lse, c_out, batch->cu_seqlens, window, n_q_heads,
-                                                                   n_kv_heads, scale * 1.4426950408889634f, T, status, wait_limit_ns());
+                                                                   n_kv_heads, scale * 1.4426950408889634f, T, status, wait_limit_ns(),
+                                                                   box_rows);
   PK_CUDA(cudaGetLastError());
   return PUREKV_OK;
 }

@@ -183,14 +183,15 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 }
 // 2^x for a pair of values on the FMA pipe (the MUFU unit is the scarce one): round to the nearest integer n with
 // the 1.5 * 2^23 trick, a cubic for 2^f on f = x - n in [-0.5, 0.5] (relative error 7.5e-5, below bf16 rounding),
-// then n is added into the exponent field.  x <= 0 here; inputs below -126 (and -inf) give 2^-126, which is
-// nothing beside the row's largest term (2^0 .. 2^-8 after lazy rescaling).
+// then n is added into the exponent field.  Inputs below -126 (and -inf, a masked entry) give 2^-126, which is
+// nothing beside the row's largest term; inputs above 127 give garbage of huge magnitude or NaN, which the caller's
+// overflow test (row sum finite and below 1e30) catches like an infinity.
 __device__ __forceinline__ float2 exp2_poly2(float2 x) {
   const float kMagic = 12582912.f;  // 1.5 * 2^23
-  x.x = fminf(fmaxf(x.x, -126.f), 128.f);  // 2^128 lands on the bit pattern of +inf, which the caller's overflow test sees
-  x.y = fminf(fmaxf(x.y, -126.f), 128.f);
+  x.x = fmaxf(x.x, -126.f);
+  x.y = fmaxf(x.y, -126.f);
   const float2 r = __fadd2_rn(x, make_float2(kMagic, kMagic));
-  const float2 f = __ffma2_rn(__fadd2_rn(r, make_float2(-kMagic, -kMagic)), make_float2(-1.f, -1.f), x);  // x - n
+  const float2 f = __fadd2_rn(x, __fadd2_rn(make_float2(kMagic, kMagic), make_float2(-r.x, -r.y)));  // x - n
   float2 p = __ffma2_rn(make_float2(0.05517115443944931f, 0.05517115443944931f), f,
                         make_float2(0.2426101416349411f, 0.2426101416349411f));
   p = __ffma2_rn(p, f, make_float2(0.6932609677314758f, 0.6932609677314758f));
