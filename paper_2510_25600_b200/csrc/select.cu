@@ -107,7 +107,7 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 }
 
 constexpr int kSelThreads = 512;
-constexpr int kSelItems = 4;
+constexpr int kSelItems = 8;
 
 // What the selecting CTA needs to also gather its segment's kept rows into the compact cache (Sec. 3.1: the selection
 // feeds the compressed cache directly); k_src == nullptr: selection only.  Rows are `cpr` 16-byte chunks; layer
@@ -132,7 +132,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
                                                              int32_t* __restrict__ idx_out, const uint4* __restrict__ v,
                                                              int64_t layer_stride_c, const float* __restrict__ c,
                                                              float* __restrict__ s_out, Gather ga) {
-  extern __shared__ uint32_t skeys[];  // FUSED: order keys of the segment's non-recent scores
+  extern __shared__ __align__(16) uint32_t skeys[];  // order keys of the segment's non-recent scores
   __shared__ int32_t hist[256];
   __shared__ uint32_t sh_prefix;
   __shared__ int32_t sh_need;
@@ -200,7 +200,8 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   // in this mode and doubles as that flag), so the radix passes do not go back to L2.
   const bool staged = FUSED || s_out != nullptr;
   if (!FUSED && staged) {
-    for (int32_t j = tid; j < nr; j += kSelThreads) skeys[j] = order_key(__ldg(seg + j));
+#pragma unroll 8
+    for (int32_t j = tid; j < nr; j += kSelThreads) skeys[j] = order_key(__ldg(seg + j));  // loads of a trip in flight together
     __syncthreads();
   }
   auto key_at = [&](int32_t j) -> uint32_t { return staged ? skeys[j] : order_key(__ldg(seg + j)); };
@@ -212,6 +213,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   for (int32_t shift = 24; shift >= 0; shift -= 8) {
     if (tid < 256) hist[tid] = 0;
     __syncthreads();
+#pragma unroll 4
     for (int32_t j = tid; j < nr; j += kSelThreads) {
       const uint32_t key = key_at(j);
       if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
@@ -261,9 +263,20 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
     const int32_t j0 = c0 + tid * kSelItems;
     uint32_t keys[kSelItems];
     int32_t n_gt = 0, n_eq = 0;
+    if (staged && j0 + kSelItems <= nr) {
+      // a thread's keys are consecutive words: 128-bit loads, which shared memory serves without bank conflicts
+      // (word-by-word they would collide eight ways)
+#pragma unroll
+      for (int i = 0; i < kSelItems; i += 4) {
+        const uint4 k4 = *reinterpret_cast<const uint4*>(skeys + j0 + i);
+        keys[i] = k4.x; keys[i + 1] = k4.y; keys[i + 2] = k4.z; keys[i + 3] = k4.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < kSelItems; ++i) keys[i] = (j0 + i < nr) ? key_at(j0 + i) : 0u;
+    }
 #pragma unroll
     for (int i = 0; i < kSelItems; ++i) {
-      keys[i] = (j0 + i < nr) ? key_at(j0 + i) : 0u;
       const bool valid = j0 + i < nr;
       n_gt += (valid && keys[i] > thr);
       n_eq += (valid && keys[i] == thr);
