@@ -67,8 +67,8 @@ class PlanHeaderView(C.Structure):
                 ("part_slots", C.c_int64), ("test_flags", C.c_uint32), ("pad_flags", C.c_uint32)]
 
 
-UNIT_INT32S = 12        # a work unit of the tensor-core plan: q_start, q_rows, req_start, ent_begin, ent_count, pair,
-                        # chunk, n_chunks, part_base, counter_base, 2 x padding
+UNIT_INT32S = 16        # a work unit of the tensor-core plan: q_start, q_rows, req_start, ent_begin, ent_count, pair,
+                        # chunk, n_chunks, part_base, counter_base, q_start1, q_rows1 (a twin unit's second tile), 4 x padding
 
 _lib.purekv_version.restype = C.c_char_p
 _lib.purekv_set_wait_limit_ns.restype = None

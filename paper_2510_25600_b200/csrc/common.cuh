@@ -65,10 +65,12 @@ __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162flo
 // ---- plan buffer layout (device memory, written by purekv_plan_build) -------------------
 // [PlanHeader][QTile x n_qtiles][order int32 x n_qtiles][entries int2 x n_entries][masks uint32 x n_mask_words]
 // [Unit x n_units][merge counters int32 x n_counters][scheduling counters int32 x 2]
-// all sections 16-byte aligned.  The last three sections exist only in plans for the tensor-core kernel.
-constexpr uint32_t kPlanMagic = 0x504B5635u;  // "PKV5"
+// all sections 16-byte aligned.  The last three sections exist only in plans for the tensor-core kernel, whose
+// entries section also holds, behind the query tiles' own lists, the merged lists of the twin units (see Unit).
+constexpr uint32_t kPlanMagic = 0x504B5636u;  // "PKV6"
 
-enum TileClass : int32_t { kTileFull = 0, kTileDiag = 1, kTileGeneral = 2 };
+// kTileNone appears only in the merged list of a twin unit: a key tile one of the two query tiles does not keep.
+enum TileClass : int32_t { kTileFull = 0, kTileDiag = 1, kTileGeneral = 2, kTileNone = 3 };
 
 struct PlanHeader {
   uint32_t magic;
@@ -111,6 +113,14 @@ struct QTile {
 // the second counts finished CTAs, and the last of them sets both back to zero.
 // A list split into n_chunks > 1 chunks leaves one partial result per chunk and head in the
 // workspace; the chunk that arrives last (merge counter) combines them.
+//
+// Twin units (q_rows1 > 0).  With an odd number G of query heads per KV head the last head of a group has no partner
+// and its unit would leave half of the kernel idle.  Two consecutive query tiles of one request whose lists are
+// not split share such a unit instead: both slots work on that head, slot 0 on the tile at q_start and slot 1 on
+// the tile at q_start1, over the union of the two tiles' lists.  The union is stored as ent_count PAIRS of entries
+// from ent_begin on: entries[ent_begin + 2n + s] is key tile n as slot s sees it, with its own class, half mask and
+// bit mask, or class kTileNone with half mask 0 where that query tile keeps nothing of the key tile (the slot then
+// multiplies by zeros).  The halves loaded and multiplied are the union of the two half masks.
 struct __align__(16) Unit {
   int32_t q_start, q_rows, req_start;
   int32_t ent_begin, ent_count;  // into entries[]
@@ -118,8 +128,10 @@ struct __align__(16) Unit {
   int32_t chunk, n_chunks;
   int32_t part_base;             // workspace slot of (chunk 0, head 0) = part_base; slot(chunk, hq) = (part_base + chunk) * H + hq
   int32_t counter_base;          // merge counter of head hq = counters[counter_base + hq]
-  int32_t pad[2];
+  int32_t q_start1, q_rows1;     // a twin unit's second query tile (q_rows1 == 0: an ordinary unit)
+  int32_t pad[4];
 };
+static_assert(sizeof(Unit) == 64, "the plan's unit record is 16 words");
 
 // Partial result of one (chunk, head): 128 x 128 fp32 unnormalised output laid out [col/4][row][col%4],
 // then 128 reference maxima (log2 domain) and 128 row sums.

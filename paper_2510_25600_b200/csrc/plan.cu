@@ -138,27 +138,71 @@ purekv_status purekv_budget(int32_t len, int32_t window, double keep_ratio, int3
 // long lists are cut.  They are in quarters of a 64-key half of a list entry, fitted
 // to measured unit times: 4 per present half (5 when the entry carries a bit mask), 6 per unit (query load, pipeline
 // fill, epilogue) and 14 more for a chunk of a split list (fp32 partial result written out, and the merge).
-static void schedule_units(const std::vector<QTile>& qtiles, const std::vector<int2>& entries, int32_t H, int32_t Hkv,
+//
+// With an odd group size the group's last head has no partner; a unit for it alone takes as long as a unit for two
+// heads.  Consecutive query tiles of a request whose lists are not split therefore share that head's unit (a twin
+// unit, see Unit): the merged lists are appended to `entries`.
+static void schedule_units(const std::vector<QTile>& qtiles, std::vector<int2>& entries, int32_t H, int32_t Hkv,
                            int32_t n_ctas,
                            std::vector<Unit>& units, int32_t* n_counters,
                            int64_t* part_slots, int32_t* max_chunks) {
   const int32_t G = H / Hkv, ppg = (G + 1) / 2, n_pairs = Hkv * ppg;
+  const bool odd = (G & 1) != 0;
   const int32_t overhead = 6, split_extra = 14;
+  const int32_t nq = (int32_t)qtiles.size();
   auto halves = [&](int32_t first, int32_t last) {  // cost of entries [first, last)
     int32_t c = 0;
     for (int32_t i = first; i < last; ++i)
       c += ((((entries[i].x >> 2) & 3) == 3) ? 2 : 1) * ((entries[i].x & 3) == kTileGeneral ? 5 : 4);
     return c;
   };
+  // The union of two query tiles' lists in key-tile order: its cost and length; the entry pairs go to `out` if given.
+  auto merge_lists = [&](const QTile& a, const QTile& b, std::vector<int2>* out, int32_t* count) {
+    int32_t ia = a.entry_begin, ib = b.entry_begin, cost = 0, n = 0;
+    const int32_t ea = ia + a.entry_count, eb = ib + b.entry_count;
+    while (ia < ea || ib < eb) {
+      const int32_t ka = ia < ea ? (entries[ia].x >> 4) : INT32_MAX, kb = ib < eb ? (entries[ib].x >> 4) : INT32_MAX;
+      const int32_t kt = std::min(ka, kb);
+      const int2 none = make_int2((kt << 4) | kTileNone, -1);
+      const int2 xa = ka == kt ? entries[ia++] : none, xb = kb == kt ? entries[ib++] : none;
+      const bool both = (((xa.x | xb.x) >> 2) & 3) == 3;
+      const bool bits = (xa.x & 3) == kTileGeneral || (xb.x & 3) == kTileGeneral;
+      cost += (both ? 2 : 1) * (bits ? 5 : 4);
+      if (out) { out->push_back(xa); out->push_back(xb); }
+      ++n;
+    }
+    *count = n;
+    return cost;
+  };
+  // partner[i]: the tile that shares tile i's odd-head unit (i leads the twin), -2 if tile i is the second of a
+  // twin, -1 if it stays alone.  A merged list may be a quarter longer than the cap on a chunk.
+  std::vector<int32_t> partner;
+  auto find_twins = [&](int32_t l_max) {
+    partner.assign((size_t)nq, -1);
+    if (!odd) return;
+    for (int32_t i = 0; i + 1 < nq; ++i) {
+      const QTile &a = qtiles[i], &b = qtiles[i + 1];
+      if (partner[i] != -1 || a.req_start != b.req_start || a.entry_count > l_max || b.entry_count > l_max) continue;
+      int32_t n = 0;
+      merge_lists(a, b, nullptr, &n);
+      if (n > l_max + l_max / 4) continue;
+      partner[i] = i + 1;
+      partner[i + 1] = -2;
+    }
+  };
   struct Item { Unit u; int32_t cost; };
   std::vector<Item> items;
+  std::vector<int2> twin_entries;
   int32_t counters = 0, mc = 1;
   int64_t slots = 0;
   // the units when no chunk of a list may be longer than l_max entries
   auto make_items = [&](int32_t l_max) {
     items.clear();
+    twin_entries.clear();
     counters = 0; mc = 1; slots = 0;
-    for (const QTile& q : qtiles) {
+    find_twins(l_max);
+    for (int32_t qi = 0; qi < nq; ++qi) {
+      const QTile& q = qtiles[qi];
       const int32_t nch = std::max(1, (q.entry_count + l_max - 1) / l_max);
       mc = std::max(mc, nch);
       const int32_t part_base = nch > 1 ? (int32_t)slots : -1, counter_base = nch > 1 ? counters : -1;
@@ -167,12 +211,27 @@ static void schedule_units(const std::vector<QTile>& qtiles, const std::vector<i
         const int32_t a = (int32_t)((int64_t)q.entry_count * c / nch), e = (int32_t)((int64_t)q.entry_count * (c + 1) / nch);
         const int32_t cost = halves(q.entry_begin + a, q.entry_begin + e) + overhead + (nch > 1 ? split_extra : 0);
         for (int32_t pr = 0; pr < n_pairs; ++pr) {
-          Unit u;
+          if (partner[qi] != -1 && pr % ppg == ppg - 1) continue;  // the odd head goes into a twin unit
+          Unit u = {};
           u.q_start = q.q_start; u.q_rows = q.q_rows; u.req_start = q.req_start;
           u.ent_begin = q.entry_begin + a; u.ent_count = e - a;
           u.pair = pr; u.chunk = c; u.n_chunks = nch;
           u.part_base = part_base; u.counter_base = counter_base;
-          u.pad[0] = u.pad[1] = 0;
+          items.push_back({u, cost});
+        }
+      }
+      if (partner[qi] >= 0) {
+        const QTile& q1 = qtiles[partner[qi]];
+        const int32_t at = (int32_t)(entries.size() + twin_entries.size());
+        int32_t n = 0;
+        const int32_t cost = merge_lists(q, q1, &twin_entries, &n) + overhead;
+        for (int32_t g = 0; g < Hkv; ++g) {
+          Unit u = {};
+          u.q_start = q.q_start; u.q_rows = q.q_rows; u.req_start = q.req_start;
+          u.q_start1 = q1.q_start; u.q_rows1 = q1.q_rows;
+          u.ent_begin = at; u.ent_count = n;
+          u.pair = g * ppg + ppg - 1; u.chunk = 0; u.n_chunks = 1;
+          u.part_base = -1; u.counter_base = -1;
           items.push_back({u, cost});
         }
       }
@@ -183,12 +242,18 @@ static void schedule_units(const std::vector<QTile>& qtiles, const std::vector<i
   std::vector<int32_t> costs;
   auto makespan = [&](int32_t l_max) {
     costs.clear();
-    for (const QTile& q : qtiles) {
+    find_twins(l_max);
+    for (int32_t qi = 0; qi < nq; ++qi) {
+      const QTile& q = qtiles[qi];
       const int32_t nch = std::max(1, (q.entry_count + l_max - 1) / l_max);
       for (int32_t c = 0; c < nch; ++c) {
         const int32_t a = (int32_t)((int64_t)q.entry_count * c / nch), e = (int32_t)((int64_t)q.entry_count * (c + 1) / nch);
-        costs.insert(costs.end(), (size_t)n_pairs,
+        costs.insert(costs.end(), (size_t)(partner[qi] != -1 ? n_pairs - Hkv : n_pairs),
                      halves(q.entry_begin + a, q.entry_begin + e) + overhead + (nch > 1 ? split_extra : 0));
+      }
+      if (partner[qi] >= 0) {
+        int32_t n = 0;
+        costs.insert(costs.end(), (size_t)Hkv, merge_lists(q, qtiles[partner[qi]], nullptr, &n) + overhead);
       }
     }
     std::sort(costs.begin(), costs.end(), std::greater<int32_t>());
@@ -215,6 +280,7 @@ static void schedule_units(const std::vector<QTile>& qtiles, const std::vector<i
     }
   }
   make_items(l_best);
+  entries.insert(entries.end(), twin_entries.begin(), twin_entries.end());
   units.clear();
   for (const Item& it : items) units.push_back(it.u);
   *n_counters = counters;

@@ -3,7 +3,9 @@
 // Persistent kernel: one CTA per SM walks the list of work units the plan assigned to it.  A unit is a
 // 128-row query tile of a PAIR of query heads that share a KV head ("slots") and a chunk of that tile's
 // list of kept key tiles, so every K/V tile staged in shared memory feeds two heads and key blocks the
-// mask removes are never read.  Roles:
+// mask removes are never read.  With an odd number of heads per KV head the group's last head is worked on by both
+// slots for two consecutive query tiles over the union of their lists (a twin unit), each slot with its own tile
+// classes and bit masks.  Roles:
 //   warp 8      producer: per unit Q of both slots, then per key tile the tile's class word and, for
 //               general tiles, its bit mask (bulk copy) into a small ring, and K and V (TMA, 128-byte
 //               swizzle, two 64-column panels each) into a ring of stages.  It runs ahead across units.
@@ -80,7 +82,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
   constexpr uint32_t kMaskBytes = Cfg<BK>::kMaskBytes;
   extern __shared__ uint8_t smem_raw[];
   __shared__ Barriers<BK> bars;
-  __shared__ int2 meta_s[MR];
+  __shared__ int2 meta_s[MR][2];  // per slot: the entry word, and the byte offset in shared memory of the slot's bit mask
   __shared__ Unit unit_s[kUnitRing];
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
@@ -91,7 +93,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
   const uint32_t sQ = smem0;                 // [2 slots][2 panels][128 rows x 128 B]
   const uint32_t sK = sQ + 2 * kTileQ;       // [ST][2 panels][BK rows x 128 B]
   const uint32_t sV = sK + ST * kTileKV;
-  const uint32_t sM = sV + ST * kTileKV;     // [MR][128 rows x BK/8 B]
+  const uint32_t sM = sV + ST * kTileKV;     // [MR][2 slots][128 rows x BK/8 B]
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // Programmatic dependent launch: the next kernel in the stream may start its CTAs as ours retire and set up its
@@ -195,11 +197,15 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       if (idx < n_units) {
         uu = units[idx];
         const int32_t n_pairs = n_kv_heads * ppg;
-        const bool split = uu.n_chunks > 1;
-        const bool good = uu.ent_count >= 1 && uu.ent_begin >= 0 && (int64_t)uu.ent_begin + uu.ent_count <= n_entries &&
+        const bool split = uu.n_chunks > 1, twin = uu.q_rows1 != 0;
+        const bool good = uu.ent_count >= 1 && uu.ent_begin >= 0 &&
+                          (int64_t)uu.ent_begin + (int64_t)uu.ent_count * (twin ? 2 : 1) <= n_entries &&
                           uu.q_rows >= 1 && uu.q_rows <= kBQ && uu.req_start >= 0 && uu.q_start >= uu.req_start &&
                           (int64_t)uu.q_start + uu.q_rows <= total_tokens && uu.pair >= 0 && uu.pair < n_pairs &&
                           uu.n_chunks >= 1 && uu.chunk >= 0 && uu.chunk < uu.n_chunks &&
+                          (!twin || (uu.q_rows1 >= 1 && uu.q_rows1 <= kBQ && uu.q_start1 >= uu.req_start &&
+                                     (int64_t)uu.q_start1 + uu.q_rows1 <= total_tokens && !split && (G & 1) != 0 &&
+                                     uu.pair % ppg == ppg - 1)) &&
                           (!split || (uu.part_base >= 0 && ((int64_t)uu.part_base + uu.n_chunks) * n_q_heads <= part_slots &&
                                       uu.counter_base >= 0 && (int64_t)uu.counter_base + n_q_heads <= n_counters));
         if (!good) {
@@ -243,44 +249,68 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       int32_t idx_next = 0;
       const int32_t nt = u.ent_count;
       const int32_t g = u.pair / ppg, hq0 = g * G + 2 * (u.pair % ppg);
-      const int32_t n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
+      const bool twin = u.q_rows1 != 0;  // both slots on head hq0, slot 1 on the query tile at q_start1
+      const int32_t n_slots = (twin || 2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
       if (lane == 0) {
         if (uo > 0) ok = mbar_wait(smem_u32(&bars.q_empty), (uo - 1u) & 1u, abort_flag, wait_ns);
         if (ok) {
           mbar_expect_tx(smem_u32(&bars.q_full), n_slots * kTileQ);
           for (int sl = 0; sl < n_slots; ++sl) {
-            tma_load_3d(sQ + sl * kTileQ, &tm_q, smem_u32(&bars.q_full), 0, hq0 + sl, u.q_start);
-            tma_load_3d(sQ + sl * kTileQ + kPanelQ, &tm_q, smem_u32(&bars.q_full), 64, hq0 + sl, u.q_start);
+            const int32_t hq = twin ? hq0 : hq0 + sl, qs = (twin && sl) ? u.q_start1 : u.q_start;
+            tma_load_3d(sQ + sl * kTileQ, &tm_q, smem_u32(&bars.q_full), 0, hq, qs);
+            tma_load_3d(sQ + sl * kTileQ + kPanelQ, &tm_q, smem_u32(&bars.q_full), 64, hq, qs);
           }
         }
       }
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       for (int32_t n0 = 0; ok && n0 < nt; n0 += 32) {
-        int2 e_l = make_int2(0, -1);
-        if (n0 + lane < nt) e_l = __ldg(entries + u.ent_begin + n0 + lane);
+        int2 e_l = make_int2(0, -1), f_l = e_l;  // the tile's entry as slot 0 and as slot 1 see it
+        if (n0 + lane < nt) {
+          if (twin) {
+            e_l = __ldg(entries + u.ent_begin + 2 * (n0 + lane));
+            f_l = __ldg(entries + u.ent_begin + 2 * (n0 + lane) + 1);
+          } else {
+            e_l = f_l = __ldg(entries + u.ent_begin + n0 + lane);
+          }
+        }
         const int32_t n1 = min(nt, n0 + 32);
         for (int32_t n = n0; ok && n < n1; ++n) {
-          int2 e;
+          int2 e, f;
           e.x = __shfl_sync(0xffffffffu, e_l.x, n - n0);
           e.y = __shfl_sync(0xffffffffu, e_l.y, n - n0);
+          f.x = __shfl_sync(0xffffffffu, f_l.x, n - n0);
+          f.y = __shfl_sync(0xffffffffu, f_l.y, n - n0);
           if (lane == 0) {
             if (n == nt - 1) idx_next = atomicAdd(sched, 1) + (int32_t)gridDim.x;  // used after the loop
             const uint32_t s = it % ST, par = ((it / ST) - 1u) & 1u, ms = it % MR;
             const int32_t tok = u.req_start + (e.x >> 4) * BK;
-            const uint32_t hm = (uint32_t)(e.x >> 2) & 3u;  // which 64-key halves of the tile are present
-            // the entry is checked before its mask offset or key-tile index is used for a copy
-            if (e.x < 0 || hm == 0u || (e.x & 3) > kTileGeneral || (int64_t)tok >= total_tokens ||
-                ((e.x & 3) == kTileGeneral && (e.y < 0 || (int64_t)e.y + (int64_t)(kMaskBytes / 4) > n_mask_words || (e.y & 3) != 0))) {
+            const uint32_t hm = (uint32_t)((e.x | f.x) >> 2) & 3u;  // which 64-key halves of the tile are present
+            // the entry is checked before its mask offset or key-tile index is used for a copy: a class the slot
+            // knows (none only in a twin unit, and then without halves), a bit mask inside the table
+            auto entry_ok = [&](const int2& x) {
+              const int32_t c = x.x & 3;
+              const uint32_t h = (uint32_t)(x.x >> 2) & 3u;
+              if (x.x < 0 || (c == kTileNone ? (!twin || h != 0u) : h == 0u)) return false;
+              return c != kTileGeneral ||
+                     (x.y >= 0 && (int64_t)x.y + (int64_t)(kMaskBytes / 4) <= n_mask_words && (x.y & 3) == 0);
+            };
+            if (!entry_ok(e) || !entry_ok(f) || (e.x >> 4) != (f.x >> 4) || hm == 0u || (int64_t)tok >= total_tokens) {
               abort_code_s = (int)PUREKV_ERR_BAD_PLAN;
               *abort_flag = 1;
               ok = false;
             }
             if (ok && it >= (uint32_t)ST) ok = mbar_wait(smem_u32(&bars.k_empty[s]), par, abort_flag, wait_ns);
             if (ok) {
-              meta_s[ms] = e;
-              if ((e.x & 3) == kTileGeneral) {
-                mbar_expect_tx(smem_u32(&bars.m_full[ms]), kMaskBytes);
-                bulk_load(sM + ms * kMaskBytes, masks + e.y, kMaskBytes, smem_u32(&bars.m_full[ms]));
+              // a slot's bit mask goes to its own buffer; outside twin units both slots read the first one
+              const uint32_t m_off = (sM - smem_u32(smem_raw)) + ms * 2u * kMaskBytes;
+              const bool mask0 = (e.x & 3) == kTileGeneral, mask1 = twin && (f.x & 3) == kTileGeneral;
+              meta_s[ms][0] = make_int2(e.x, (int32_t)m_off);
+              meta_s[ms][1] = make_int2(f.x, (int32_t)(m_off + (twin ? kMaskBytes : 0u)));
+              if (mask0 || mask1) {
+                mbar_expect_tx(smem_u32(&bars.m_full[ms]), (mask0 && mask1) ? 2u * kMaskBytes : kMaskBytes);
+                if (mask0) bulk_load(sM + ms * 2u * kMaskBytes, masks + e.y, kMaskBytes, smem_u32(&bars.m_full[ms]));
+                if (mask1)
+                  bulk_load(sM + ms * 2u * kMaskBytes + kMaskBytes, masks + f.y, kMaskBytes, smem_u32(&bars.m_full[ms]));
               } else {
                 mbar_arrive(smem_u32(&bars.m_full[ms]));
               }
@@ -357,7 +387,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         // the stage was already awaited for slot 0 of the same tile
         if (sl == 0 && !mbar_wait(smem_u32(&bars.k_full[s]), (it / ST) & 1u, abort_flag, wait_ns)) return false;
         tc_fence_after();
-        const uint32_t hm = (uint32_t)(meta_s[it % MR].x >> 2) & 3u;  // written before the stage's barrier was armed
+        const uint32_t hm = (uint32_t)((meta_s[it % MR][0].x | meta_s[it % MR][1].x) >> 2) & 3u;  // written before the stage's barrier was armed
         const uint32_t q_lo = q_lo0 + (uint32_t)sl * (kTileQ >> 4);
         if (hm == 3u) {
           const uint32_t d_addr = tmem + sl * 128 + b * BK, k_lo = k_lo0 + s * (kTileKV >> 4);
@@ -401,7 +431,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         const uint32_t p_addr = tmem + sl * 128 + b * BK, o_addr = tmem + kColO + sl * 128;
         // B = V tile, MN-major: per K step 16 key rows (2 groups of 8, 1024 B apart) x 128 dims (2 panels)
         const uint32_t v_lo = v_lo0 + s * (kTileKV >> 4);
-        const uint32_t hm = (uint32_t)(meta_s[it % MR].x >> 2) & 3u;
+        const uint32_t hm = (uint32_t)((meta_s[it % MR][0].x | meta_s[it % MR][1].x) >> 2) & 3u;
         const uint32_t acc0 = n > 0 ? 1u : 0u;  // the unit's first product overwrites O
         if (hm == 3u) {
 #pragma unroll
@@ -431,7 +461,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         mbar_arrive(smem_u32(&bars.u_empty[us]));
         if (u.ent_count == 0) break;
         nt = u.ent_count;
-        n_slots = (2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
+        n_slots = (u.q_rows1 != 0 || 2 * (u.pair % ppg) + 1 < G) ? 2 : 1;
         ok = mbar_wait(smem_u32(&bars.q_full), uo & 1u, abort_flag, wait_ns);
         constexpr std::integral_constant<int, 0> s0{};
         constexpr std::integral_constant<int, 1> s1{};
@@ -494,7 +524,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       const int32_t nt = u.ent_count;
       if (nt == 0) break;
       const int32_t pr = u.pair % ppg, g = u.pair / ppg;
-      const int32_t n_slots = (2 * pr + 1 < G) ? 2 : 1;
+      const bool twin = u.q_rows1 != 0;
+      const int32_t n_slots = (twin || 2 * pr + 1 < G) ? 2 : 1;
       if (sl >= n_slots) {
         // A single-head unit: this slot sits it out.  It takes no part in the tile ring meanwhile: a parity wait only
         // tells a barrier's current phase from the one before, and a slot with nothing to deliver is held back by
@@ -505,20 +536,23 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         release_unit();
         continue;
       }
-      const int32_t hq = g * G + 2 * pr + sl;
-      const bool row_valid = row < u.q_rows;
-      const int32_t i_rel = u.q_start - u.req_start + row;
+      const int32_t hq = g * G + 2 * pr + (twin ? 0 : sl);
+      const bool second = twin && sl == 1;  // this slot works on the unit's second query tile
+      const bool row_valid = row < (second ? u.q_rows1 : u.q_rows);
+      const int32_t i_rel = (second ? u.q_start1 : u.q_start) - u.req_start + row;
       float m_ref = 0.f, l_sum = 0.f;
       for (int32_t n = 0; n < nt; ++n) {
         const uint32_t it = it_base + (uint32_t)n, ms = it % MR, b = t % SB;
         if (!wait_w(smem_u32(&bars.m_full[ms]), (it / MR) & 1u)) { ok = false; break; }
-        const int2 e = meta_s[ms];
+        const int2 e = meta_s[ms][sl];
         const int32_t cls = e.x & 3, j0 = (e.x >> 4) * BK;
-        const uint32_t hm = (uint32_t)(e.x >> 2) & 3u;  // present 64-key halves; chunk c belongs to half c / 2
+        // hm: the 64-key halves that were loaded and multiplied (chunk c belongs to half c / 2); hm_own: those in which
+        // this slot's query tile keeps anything (they differ in twin units only)
+        const uint32_t hm_own = (uint32_t)(e.x >> 2) & 3u;
+        const uint32_t hm = (uint32_t)((e.x | meta_s[ms][sl ^ 1].x) >> 2) & 3u;
         uint32_t keep[BK / 32];
         if (cls == kTileGeneral) {  // this row's bits of the tile's mask
-          const uint32_t* mrow = reinterpret_cast<const uint32_t*>(smem_raw + (sM - smem_u32(smem_raw)) + ms * kMaskBytes) +
-                                 row * (BK / 32);
+          const uint32_t* mrow = reinterpret_cast<const uint32_t*>(smem_raw + e.y) + row * (BK / 32);
           static_assert(BK == 128, "a mask row is four 32-bit words");
           const uint4 w4 = *reinterpret_cast<const uint4*>(mrow);
           keep[0] = w4.x; keep[1] = w4.y; keep[2] = w4.z; keep[3] = w4.w;
@@ -533,10 +567,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
 #pragma unroll
           for (int c = 0; c < BK / 32; ++c) keep[c] = 0xFFFFFFFFu;
         }
-        if (hm != 3u) {  // columns of an absent half hold nothing: treat them as masked and leave them alone
+        if (hm_own != 3u) {  // columns of a half the slot keeps nothing of (or that is absent altogether): masked
 #pragma unroll
           for (int c = 0; c < BK / 32; ++c)
-            if (!((hm >> (c >> 1)) & 1u)) keep[c] = 0u;
+            if (!((hm_own >> (c >> 1)) & 1u)) keep[c] = 0u;
         }
         if (!wait_w(smem_u32(&bars.s_full[sl][b]), (t / SB) & 1u)) { ok = false; break; }
         tc_fence_after();
@@ -591,7 +625,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
             else half_exp(r, std::integral_constant<int, 1>{});
           }
           l_tile = (ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y);
-          bool has_kept = cls == kTileFull;
+          bool has_kept = cls == kTileFull;  // (a full tile has both halves)
 #pragma unroll
           for (int c = 0; c < BK / 32; ++c) has_kept |= keep[c] != 0u;
           // overflow (inf or NaN), or kept keys and still nothing representable: redo against the true maximum
@@ -667,9 +701,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
       if (!wait_w(smem_u32(&bars.o_final[sl]), slot_units & 1u)) { ok = false; break; }
       ++slot_units;
       tc_fence_after();
+      const int32_t q_first = (u.q_rows1 != 0 && sl == 1) ? u.q_start1 : u.q_start;  // the slot's query tile
       if (u.n_chunks == 1) {
         const float inv = 1.f / l_sum;
-        __nv_bfloat16* dst = o + ((int64_t)(u.q_start + row) * n_q_heads + hq) * kD;
+        __nv_bfloat16* dst = o + ((int64_t)(q_first + row) * n_q_heads + hq) * kD;
 #pragma unroll
         for (int c = 0; c < kD / 32; ++c) {
           uint32_t tt[32];
@@ -687,7 +722,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
           }
         }
         if (lse && row_valid)
-          lse[(int64_t)hq * total_tokens + u.q_start + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+          lse[(int64_t)hq * total_tokens + q_first + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
       } else {
         // one chunk of a split list: leave the unnormalised result for whoever arrives last
         float* part = ws + ((int64_t)(u.part_base + u.chunk) * n_q_heads + hq) * kPartFloats;
@@ -730,7 +765,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
             if (lc > 0.f) l_all += lc * ex2(mc - m_all);
           }
           const float inv = 1.f / l_all;
-          __nv_bfloat16* dst = o + ((int64_t)(u.q_start + row) * n_q_heads + hq) * kD;
+          __nv_bfloat16* dst = o + ((int64_t)(q_first + row) * n_q_heads + hq) * kD;
 #pragma unroll 1
           for (int cc = 0; cc < kD / 32; ++cc) {
             float acc[32];
@@ -763,7 +798,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
             }
           }
           if (lse && row_valid)
-            lse[(int64_t)hq * total_tokens + u.q_start + row] = (m_all + log2f(l_all)) * 0.6931471805599453f;
+            lse[(int64_t)hq * total_tokens + q_first + row] = (m_all + log2f(l_all)) * 0.6931471805599453f;
         }
       }
       release_unit();
@@ -784,7 +819,7 @@ static purekv_status launch(const PrefillArgs& a, const CUtensorMap& mq, const C
                             const CUtensorMap& mk64, const CUtensorMap& mv64, int32_t* status) {
   constexpr int BK = 128;
   const size_t smem = 1024 + 2 * 2 * (size_t)kBQ * 128 + 2 * (size_t)Cfg<BK>::kStages * 2 * BK * 128 +
-                      (size_t)Cfg<BK>::kMeta * Cfg<BK>::kMaskBytes;
+                      2 * (size_t)Cfg<BK>::kMeta * Cfg<BK>::kMaskBytes;
   static std::atomic<int> launch_regs{0};  // the compiled register count: the same on every device, read once
   int regs = launch_regs.load(std::memory_order_relaxed);
   if (regs == 0) {

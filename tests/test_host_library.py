@@ -36,12 +36,12 @@ def parse_plan(buf: np.ndarray):
     raw = buf.tobytes()
     (magic, tq, tk, nq, T, ne, nm, oq, oo, oe, om, wpr, n_ctas, n_units, n_counters, o_units, o_counters, H, Hkv,
      part_slots) = struct.unpack_from("<Iiiiqqqqqqqiiiiqqiiq", raw, 0)
-    assert magic == 0x504B5635
+    assert magic == 0x504B5636
     qt = np.frombuffer(raw, dtype=np.int32, count=nq * 8, offset=oq).reshape(nq, 8)
     order = np.frombuffer(raw, dtype=np.int32, count=nq, offset=oo)
     entries = np.frombuffer(raw, dtype=np.int32, count=2 * ne, offset=oe).reshape(ne, 2)
     masks = np.frombuffer(raw, dtype=np.uint32, count=nm, offset=om)
-    units = np.frombuffer(raw, dtype=np.int32, count=12 * n_units, offset=o_units).reshape(n_units, 12)
+    units = np.frombuffer(raw, dtype=np.int32, count=16 * n_units, offset=o_units).reshape(n_units, 16)
     counters = np.frombuffer(raw, dtype=np.int32, count=n_counters, offset=o_counters)
     sched = np.frombuffer(raw, dtype=np.int32, count=2 if n_units else 0, offset=o_counters + 4 * n_counters)
     return dict(tq=tq, tk=tk, nq=nq, T=T, qt=qt, order=order, entries=entries, masks=masks, wpr=wpr, n_ctas=n_ctas,
@@ -52,25 +52,56 @@ def check_schedule(p, info, H, Hkv, n_ctas):
     """The persistent kernel's schedule: every (query tile, head pair, list entry) is covered exactly once, chunks
     of a split list are contiguous and complete, workspace slots and merge counters do not collide, the units
     come in order of decreasing cost, and handing them out in that order to whichever CTA is free first leaves no CTA
-    with much more than its share."""
+    with much more than its share.  A twin unit (two consecutive query tiles sharing the unit of a group's odd
+    head) carries the union of the two tiles' lists as entry pairs: each tile's own entries in order, and the
+    "none" class with no halves where a tile does not keep the key tile."""
     G = H // Hkv
-    n_pairs = Hkv * ((G + 1) // 2)
+    ppg = (G + 1) // 2
+    n_pairs = Hkv * ppg
     units = p["units"]
+    ent = p["entries"]
     assert p["n_ctas"] == n_ctas == info.n_ctas and len(units) == info.n_units
     assert (p["counters"] == 0).all() and (p["sched"] == 0).all()
     by_start = {int(r[0]): r for r in p["qt"]}
+    n_own = int(p["qt"][:, 5].sum())                      # the tiles' own lists come first in the entries section
     covered = {}
     chunks = {}
+    n_twin = 0
     for u in units:
-        q_start, q_rows, req_start, eb, ec, pair, chunk, nch, part_base, counter_base = (int(x) for x in u[:10])
+        q_start, q_rows, req_start, eb, ec, pair, chunk, nch, part_base, counter_base, q_start1, q_rows1 = (int(x) for x in u[:12])
+        assert (u[12:] == 0).all()
         qt = by_start[q_start]
         assert q_rows == qt[1] and req_start == qt[2] and 0 <= pair < n_pairs and 0 <= chunk < nch and ec >= 1
-        assert qt[4] <= eb and eb + ec <= qt[4] + qt[5]
-        for e in range(eb, eb + ec):
-            assert (q_start, pair, e) not in covered
-            covered[(q_start, pair, e)] = chunk
-        chunks.setdefault((q_start, pair), []).append((chunk, eb, ec, nch, part_base, counter_base))
-    assert len(covered) == n_pairs * int(p["qt"][:, 5].sum())
+        if q_rows1 == 0:
+            assert q_start1 == 0
+            assert qt[4] <= eb and eb + ec <= qt[4] + qt[5]
+            for e in range(eb, eb + ec):
+                assert (q_start, pair, e) not in covered
+                covered[(q_start, pair, e)] = chunk
+            chunks.setdefault((q_start, pair), []).append((chunk, eb, ec, nch, part_base, counter_base))
+            continue
+        n_twin += 1
+        qt1 = by_start[q_start1]
+        assert G % 2 == 1 and pair % ppg == ppg - 1 and nch == 1 and chunk == 0 and part_base == -1 and counter_base == -1
+        assert q_rows1 == qt1[1] and req_start == qt1[2] and q_start1 == q_start + q_rows    # the next tile of the request
+        assert eb >= n_own and eb + 2 * ec <= len(ent)
+        pairs = ent[eb:eb + 2 * ec].reshape(ec, 2, 2)
+        kts = pairs[:, 0, 0] >> 4
+        assert (kts == pairs[:, 1, 0] >> 4).all() and (np.diff(kts) > 0).all()
+        for s, t in enumerate((qt, qt1)):
+            own = ent[t[4]:t[4] + t[5]]
+            mine = pairs[:, s]
+            kept = (mine[:, 0] & 3) != 3
+            assert np.array_equal(mine[kept], own)                                         # its own list, in order
+            assert ((mine[~kept, 0] & 15) == 3).all() and (mine[~kept, 1] == -1).all()     # none: no class, no halves
+            for e in range(int(t[4]), int(t[4] + t[5])):
+                assert (int(t[0]), pair, e) not in covered
+                covered[(int(t[0]), pair, e)] = 0
+            chunks.setdefault((int(t[0]), pair), []).append((0, int(t[4]), int(t[5]), 1, -1, -1))
+        assert set(kts.tolist()) == set((ent[qt[4]:qt[4] + qt[5], 0] >> 4).tolist()) | set((ent[qt1[4]:qt1[4] + qt1[5], 0] >> 4).tolist())
+    assert len(covered) == n_pairs * n_own
+    if G % 2 == 0:
+        assert n_twin == 0 and len(ent) == n_own
     slots_used, counters_used = set(), set()
     for (q_start, pair), lst in chunks.items():
         lst.sort()
@@ -95,10 +126,16 @@ def check_schedule(p, info, H, Hkv, n_ctas):
                     counters_used.add(cnt)
     assert len(slots_used) == p["part_slots"] and len(counters_used) == len(p["counters"])
     assert info.ws_bytes == p["part_slots"] * (128 * 128 + 256) * 4
-    ent = p["entries"]
     def cost(u):                                          # the scheduler's cost model
-        e = ent[u[3]:u[3] + u[4], 0]
-        c = np.where(((e >> 2) & 3) == 3, 2, 1) * np.where((e & 3) == 2, 5, 4)
+        if u[11] == 0:
+            e = ent[u[3]:u[3] + u[4], 0]
+            both = ((e >> 2) & 3) == 3
+            bits = (e & 3) == 2
+        else:                                             # a twin unit: the halves and bit masks of either tile
+            e = ent[u[3]:u[3] + 2 * u[4], 0].reshape(-1, 2)
+            both = (((e[:, 0] | e[:, 1]) >> 2) & 3) == 3
+            bits = ((e[:, 0] & 3) == 2) | ((e[:, 1] & 3) == 2)
+        c = np.where(both, 2, 1) * np.where(bits, 5, 4)
         return int(c.sum()) + 6 + (14 if u[7] > 1 else 0)
     costs = [cost(u) for u in units]
     assert all(a >= b for a, b in zip(costs, costs[1:]))
@@ -203,9 +240,15 @@ def test_plan_matches_oracle_for_the_named_variants_and_their_block_level_wideni
 def test_plan_for_tensor_core_shapes_and_workload_counts():
     batch = inputs.make_batch([64, 3], [5, 2], [64, 130], 12, 12)
     for tile in (64, 128):
-        for H, Hkv, n_ctas in ((4, 2, 0), (7, 1, 5), (6, 2, 3), (2, 2, 400)):
-            info = check_plan(batch, inputs.STMask(12, 12, tile=tile), pk.BF16, 128, H, Hkv, n_ctas)
-            assert info.tile_q == 128 and info.tile_k == tile
+        for H, Hkv, n_ctas in ((4, 2, 0), (7, 1, 5), (6, 2, 3), (2, 2, 400), (3, 3, 4), (9, 3, 0)):
+            for dense in (False, True):
+                info = check_plan(batch, inputs.STMask(12, 12, tile=tile, dense_causal=dense), pk.BF16, 128, H, Hkv, n_ctas)
+                assert info.tile_q == 128 and info.tile_k == tile
+    # an odd group size: the odd head of consecutive unsplit query tiles shares twin units (none with an even one)
+    b = pk.Batch(batch.seq_lens, batch.n_prefix, batch.n_frames, device=None)
+    for H, Hkv, want in ((7, 1, True), (3, 3, True), (6, 2, True), (8, 2, False)):
+        buf, info = pk.purekv_plan_build_host(b, pk.st_params(inputs.STMask(12, 12, tile=64)), pk.BF16, 128, H, Hkv, 0)
+        assert bool((parse_plan(buf)["units"][:, 11] > 0).any()) == want
     # many CTAs and one long request: its lists (text rows see every key) are cut into chunks
     long_batch = inputs.make_batch([4], [40], [20], 12, 12)
     for n_ctas in (0, 400):
