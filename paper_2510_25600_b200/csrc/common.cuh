@@ -116,8 +116,9 @@ struct QTile {
 //
 // Twin units (q_rows1 > 0).  With an odd number G of query heads per KV head the last head of a group has no partner
 // and its unit would leave half of the kernel idle.  Two consecutive query tiles of one request whose lists are
-// not split share such a unit instead: both slots work on that head, slot 0 on the tile at q_start and slot 1 on
-// the tile at q_start1, over the union of the two tiles' lists.  The union is stored as ent_count PAIRS of entries
+// cut into the same number of chunks share such a unit instead: both slots work on that head, slot 0 on the tile at
+// q_start and slot 1 on the tile at q_start1, over the union of the two tiles' lists (of their chunks number
+// `chunk`, when the lists are split; each tile keeps its own partial results and merge counters).  The union is stored as ent_count PAIRS of entries
 // from ent_begin on: entries[ent_begin + 2n + s] is key tile n as slot s sees it, with its own class, half mask and
 // bit mask, or class kTileNone with half mask 0 where that query tile keeps nothing of the key tile (the slot then
 // multiplies by zeros).  The halves loaded and multiplied are the union of the two half masks.
@@ -129,7 +130,8 @@ struct __align__(16) Unit {
   int32_t part_base;             // workspace slot of (chunk 0, head 0) = part_base; slot(chunk, hq) = (part_base + chunk) * H + hq
   int32_t counter_base;          // merge counter of head hq = counters[counter_base + hq]
   int32_t q_start1, q_rows1;     // a twin unit's second query tile (q_rows1 == 0: an ordinary unit)
-  int32_t pad[4];
+  int32_t part_base1, counter_base1;  // ... and that tile's workspace slots and merge counters when the lists are split
+  int32_t pad[2];
 };
 static_assert(sizeof(Unit) == 64, "the plan's unit record is 16 words");
 

@@ -156,10 +156,10 @@ static void schedule_units(const std::vector<QTile>& qtiles, std::vector<int2>& 
       c += ((((entries[i].x >> 2) & 3) == 3) ? 2 : 1) * ((entries[i].x & 3) == kTileGeneral ? 5 : 4);
     return c;
   };
-  // The union of two query tiles' lists in key-tile order: its cost and length; the entry pairs go to `out` if given.
-  auto merge_lists = [&](const QTile& a, const QTile& b, std::vector<int2>* out, int32_t* count) {
-    int32_t ia = a.entry_begin, ib = b.entry_begin, cost = 0, n = 0;
-    const int32_t ea = ia + a.entry_count, eb = ib + b.entry_count;
+  // The union of two runs of entries (of two query tiles' lists) in key-tile order: its cost and length; the entry
+  // pairs go to `out` if given.
+  auto merge_lists = [&](int32_t ia, int32_t ea, int32_t ib, int32_t eb, std::vector<int2>* out, int32_t* count) {
+    int32_t cost = 0, n = 0;
     while (ia < ea || ib < eb) {
       const int32_t ka = ia < ea ? (entries[ia].x >> 4) : INT32_MAX, kb = ib < eb ? (entries[ib].x >> 4) : INT32_MAX;
       const int32_t kt = std::min(ka, kb);
@@ -174,18 +174,32 @@ static void schedule_units(const std::vector<QTile>& qtiles, std::vector<int2>& 
     *count = n;
     return cost;
   };
-  // partner[i]: the tile that shares tile i's odd-head unit (i leads the twin), -2 if tile i is the second of a
-  // twin, -1 if it stays alone.  A merged list may be a quarter longer than the cap on a chunk.
+  auto chunks_of = [&](const QTile& q, int32_t l_max) { return std::max(1, (q.entry_count + l_max - 1) / l_max); };
+  // chunk c of nch of a tile's list, as a range of entries[]
+  auto chunk_range = [&](const QTile& q, int32_t c, int32_t nch, int32_t* first, int32_t* last) {
+    *first = q.entry_begin + (int32_t)((int64_t)q.entry_count * c / nch);
+    *last = q.entry_begin + (int32_t)((int64_t)q.entry_count * (c + 1) / nch);
+  };
+  // partner[i]: the tile that shares tile i's odd-head units (i leads the twin), -2 if tile i is the second of a
+  // twin, -1 if it stays alone.  Twins have the same number of chunks, and a merged chunk may be a quarter longer
+  // than the cap on a chunk.
   std::vector<int32_t> partner;
   auto find_twins = [&](int32_t l_max) {
     partner.assign((size_t)nq, -1);
     if (!odd) return;
     for (int32_t i = 0; i + 1 < nq; ++i) {
       const QTile &a = qtiles[i], &b = qtiles[i + 1];
-      if (partner[i] != -1 || a.req_start != b.req_start || a.entry_count > l_max || b.entry_count > l_max) continue;
-      int32_t n = 0;
-      merge_lists(a, b, nullptr, &n);
-      if (n > l_max + l_max / 4) continue;
+      const int32_t nch = chunks_of(a, l_max);
+      if (partner[i] != -1 || a.req_start != b.req_start || nch != chunks_of(b, l_max)) continue;
+      bool fits = true;
+      for (int32_t c = 0; c < nch && fits; ++c) {
+        int32_t a0, a1, b0, b1, n = 0;
+        chunk_range(a, c, nch, &a0, &a1);
+        chunk_range(b, c, nch, &b0, &b1);
+        merge_lists(a0, a1, b0, b1, nullptr, &n);
+        fits = n <= l_max + l_max / 4;
+      }
+      if (!fits) continue;
       partner[i] = i + 1;
       partner[i + 1] = -2;
     }
@@ -193,6 +207,7 @@ static void schedule_units(const std::vector<QTile>& qtiles, std::vector<int2>& 
   struct Item { Unit u; int32_t cost; };
   std::vector<Item> items;
   std::vector<int2> twin_entries;
+  std::vector<int32_t> part_of, counter_of;  // per query tile: first workspace slot and merge counter, -1 if unsplit
   int32_t counters = 0, mc = 1;
   int64_t slots = 0;
   // the units when no chunk of a list may be longer than l_max entries
@@ -201,38 +216,51 @@ static void schedule_units(const std::vector<QTile>& qtiles, std::vector<int2>& 
     twin_entries.clear();
     counters = 0; mc = 1; slots = 0;
     find_twins(l_max);
+    part_of.assign((size_t)nq, -1);
+    counter_of.assign((size_t)nq, -1);
+    for (int32_t qi = 0; qi < nq; ++qi) {
+      const int32_t nch = chunks_of(qtiles[qi], l_max);
+      mc = std::max(mc, nch);
+      if (nch > 1) {
+        part_of[qi] = (int32_t)slots;
+        counter_of[qi] = counters;
+        slots += nch;
+        counters += H;
+      }
+    }
     for (int32_t qi = 0; qi < nq; ++qi) {
       const QTile& q = qtiles[qi];
-      const int32_t nch = std::max(1, (q.entry_count + l_max - 1) / l_max);
-      mc = std::max(mc, nch);
-      const int32_t part_base = nch > 1 ? (int32_t)slots : -1, counter_base = nch > 1 ? counters : -1;
-      if (nch > 1) { slots += nch; counters += H; }
+      const int32_t nch = chunks_of(q, l_max);
       for (int32_t c = 0; c < nch; ++c) {
-        const int32_t a = (int32_t)((int64_t)q.entry_count * c / nch), e = (int32_t)((int64_t)q.entry_count * (c + 1) / nch);
-        const int32_t cost = halves(q.entry_begin + a, q.entry_begin + e) + overhead + (nch > 1 ? split_extra : 0);
+        int32_t a, e;
+        chunk_range(q, c, nch, &a, &e);
+        const int32_t cost = halves(a, e) + overhead + (nch > 1 ? split_extra : 0);
         for (int32_t pr = 0; pr < n_pairs; ++pr) {
           if (partner[qi] != -1 && pr % ppg == ppg - 1) continue;  // the odd head goes into a twin unit
           Unit u = {};
           u.q_start = q.q_start; u.q_rows = q.q_rows; u.req_start = q.req_start;
-          u.ent_begin = q.entry_begin + a; u.ent_count = e - a;
+          u.ent_begin = a; u.ent_count = e - a;
           u.pair = pr; u.chunk = c; u.n_chunks = nch;
-          u.part_base = part_base; u.counter_base = counter_base;
+          u.part_base = part_of[qi]; u.counter_base = counter_of[qi];
+          u.part_base1 = u.counter_base1 = -1;
           items.push_back({u, cost});
         }
-      }
-      if (partner[qi] >= 0) {
-        const QTile& q1 = qtiles[partner[qi]];
-        const int32_t at = (int32_t)(entries.size() + twin_entries.size());
-        int32_t n = 0;
-        const int32_t cost = merge_lists(q, q1, &twin_entries, &n) + overhead;
-        for (int32_t g = 0; g < Hkv; ++g) {
-          Unit u = {};
-          u.q_start = q.q_start; u.q_rows = q.q_rows; u.req_start = q.req_start;
-          u.q_start1 = q1.q_start; u.q_rows1 = q1.q_rows;
-          u.ent_begin = at; u.ent_count = n;
-          u.pair = g * ppg + ppg - 1; u.chunk = 0; u.n_chunks = 1;
-          u.part_base = -1; u.counter_base = -1;
-          items.push_back({u, cost});
+        if (partner[qi] >= 0) {
+          const QTile& q1 = qtiles[partner[qi]];
+          int32_t a1, e1, n = 0;
+          chunk_range(q1, c, nch, &a1, &e1);
+          const int32_t at = (int32_t)(entries.size() + twin_entries.size());
+          const int32_t cost2 = merge_lists(a, e, a1, e1, &twin_entries, &n) + overhead + (nch > 1 ? split_extra : 0);
+          for (int32_t g = 0; g < Hkv; ++g) {
+            Unit u = {};
+            u.q_start = q.q_start; u.q_rows = q.q_rows; u.req_start = q.req_start;
+            u.q_start1 = q1.q_start; u.q_rows1 = q1.q_rows;
+            u.ent_begin = at; u.ent_count = n;
+            u.pair = g * ppg + ppg - 1; u.chunk = c; u.n_chunks = nch;
+            u.part_base = part_of[qi]; u.counter_base = counter_of[qi];
+            u.part_base1 = part_of[partner[qi]]; u.counter_base1 = counter_of[partner[qi]];
+            items.push_back({u, cost2});
+          }
         }
       }
     }
@@ -245,15 +273,17 @@ static void schedule_units(const std::vector<QTile>& qtiles, std::vector<int2>& 
     find_twins(l_max);
     for (int32_t qi = 0; qi < nq; ++qi) {
       const QTile& q = qtiles[qi];
-      const int32_t nch = std::max(1, (q.entry_count + l_max - 1) / l_max);
+      const int32_t nch = chunks_of(q, l_max);
       for (int32_t c = 0; c < nch; ++c) {
-        const int32_t a = (int32_t)((int64_t)q.entry_count * c / nch), e = (int32_t)((int64_t)q.entry_count * (c + 1) / nch);
-        costs.insert(costs.end(), (size_t)(partner[qi] != -1 ? n_pairs - Hkv : n_pairs),
-                     halves(q.entry_begin + a, q.entry_begin + e) + overhead + (nch > 1 ? split_extra : 0));
-      }
-      if (partner[qi] >= 0) {
-        int32_t n = 0;
-        costs.insert(costs.end(), (size_t)Hkv, merge_lists(q, qtiles[partner[qi]], nullptr, &n) + overhead);
+        int32_t a, e;
+        chunk_range(q, c, nch, &a, &e);
+        const int32_t extra = overhead + (nch > 1 ? split_extra : 0);
+        costs.insert(costs.end(), (size_t)(partner[qi] != -1 ? n_pairs - Hkv : n_pairs), halves(a, e) + extra);
+        if (partner[qi] >= 0) {
+          int32_t a1, e1, n = 0;
+          chunk_range(qtiles[partner[qi]], c, nch, &a1, &e1);
+          costs.insert(costs.end(), (size_t)Hkv, merge_lists(a, e, a1, e1, nullptr, &n) + extra);
+        }
       }
     }
     std::sort(costs.begin(), costs.end(), std::greater<int32_t>());

@@ -204,8 +204,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
                           (int64_t)uu.q_start + uu.q_rows <= total_tokens && uu.pair >= 0 && uu.pair < n_pairs &&
                           uu.n_chunks >= 1 && uu.chunk >= 0 && uu.chunk < uu.n_chunks &&
                           (!twin || (uu.q_rows1 >= 1 && uu.q_rows1 <= kBQ && uu.q_start1 >= uu.req_start &&
-                                     (int64_t)uu.q_start1 + uu.q_rows1 <= total_tokens && !split && (G & 1) != 0 &&
-                                     uu.pair % ppg == ppg - 1)) &&
+                                     (int64_t)uu.q_start1 + uu.q_rows1 <= total_tokens && (G & 1) != 0 &&
+                                     uu.pair % ppg == ppg - 1 &&
+                                     (!split || (uu.part_base1 >= 0 && ((int64_t)uu.part_base1 + uu.n_chunks) * n_q_heads <= part_slots &&
+                                                 uu.counter_base1 >= 0 && (int64_t)uu.counter_base1 + n_q_heads <= n_counters)))) &&
                           (!split || (uu.part_base >= 0 && ((int64_t)uu.part_base + uu.n_chunks) * n_q_heads <= part_slots &&
                                       uu.counter_base >= 0 && (int64_t)uu.counter_base + n_q_heads <= n_counters));
         if (!good) {
@@ -725,7 +727,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
           lse[(int64_t)hq * total_tokens + q_first + row] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
       } else {
         // one chunk of a split list: leave the unnormalised result for whoever arrives last
-        float* part = ws + ((int64_t)(u.part_base + u.chunk) * n_q_heads + hq) * kPartFloats;
+        const bool second_tile = u.q_rows1 != 0 && sl == 1;  // a twin unit's second tile has slots and counters of its own
+        const int32_t part_base = second_tile ? u.part_base1 : u.part_base;
+        float* part = ws + ((int64_t)(part_base + u.chunk) * n_q_heads + hq) * kPartFloats;
 #pragma unroll
         for (int c = 0; c < kD / 32; ++c) {
           uint32_t tt[32];
@@ -743,14 +747,14 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_tc_kernel(
         // ordered before it, so no thread needs a fence of its own.
         if (!sync_rows()) { ok = false; break; }
         if (row == 0) {
-          int32_t* cnt = counters + u.counter_base + hq;
+          int32_t* cnt = counters + (second_tile ? u.counter_base1 : u.counter_base) + hq;
           const int last = atom_add_acq_rel(cnt, 1) == u.n_chunks - 1;
           if (last) *cnt = 0;  // every chunk has arrived: ready for the next launch (nobody touches it before then)
           merge_s[sl] = last;
         }
         if (!sync_rows()) { ok = false; break; }
         if (merge_s[sl]) {
-          const float* p0 = ws + ((int64_t)u.part_base * n_q_heads + hq) * kPartFloats;
+          const float* p0 = ws + ((int64_t)part_base * n_q_heads + hq) * kPartFloats;
           const int64_t cstride = (int64_t)n_q_heads * kPartFloats;
           float m_all = -INFINITY;
           for (int32_t c = 0; c < u.n_chunks; ++c) {

@@ -69,11 +69,11 @@ def check_schedule(p, info, H, Hkv, n_ctas):
     n_twin = 0
     for u in units:
         q_start, q_rows, req_start, eb, ec, pair, chunk, nch, part_base, counter_base, q_start1, q_rows1 = (int(x) for x in u[:12])
-        assert (u[12:] == 0).all()
+        assert (u[14:] == 0).all()
         qt = by_start[q_start]
         assert q_rows == qt[1] and req_start == qt[2] and 0 <= pair < n_pairs and 0 <= chunk < nch and ec >= 1
         if q_rows1 == 0:
-            assert q_start1 == 0
+            assert q_start1 == 0 and u[12] == -1 and u[13] == -1
             assert qt[4] <= eb and eb + ec <= qt[4] + qt[5]
             for e in range(eb, eb + ec):
                 assert (q_start, pair, e) not in covered
@@ -81,28 +81,37 @@ def check_schedule(p, info, H, Hkv, n_ctas):
             chunks.setdefault((q_start, pair), []).append((chunk, eb, ec, nch, part_base, counter_base))
             continue
         n_twin += 1
+        part_base1, counter_base1 = int(u[12]), int(u[13])
         qt1 = by_start[q_start1]
-        assert G % 2 == 1 and pair % ppg == ppg - 1 and nch == 1 and chunk == 0 and part_base == -1 and counter_base == -1
+        assert G % 2 == 1 and pair % ppg == ppg - 1
         assert q_rows1 == qt1[1] and req_start == qt1[2] and q_start1 == q_start + q_rows    # the next tile of the request
         assert eb >= n_own and eb + 2 * ec <= len(ent)
         pairs = ent[eb:eb + 2 * ec].reshape(ec, 2, 2)
         kts = pairs[:, 0, 0] >> 4
         assert (kts == pairs[:, 1, 0] >> 4).all() and (np.diff(kts) > 0).all()
-        for s, t in enumerate((qt, qt1)):
-            own = ent[t[4]:t[4] + t[5]]
+        both = set()
+        for s, (t, pb, cb) in enumerate(((qt, part_base, counter_base), (qt1, part_base1, counter_base1))):
+            first = int(t[4]) + int(t[5]) * chunk // nch                                   # chunk number `chunk` of its own list
+            last = int(t[4]) + int(t[5]) * (chunk + 1) // nch
+            own = ent[first:last]
             mine = pairs[:, s]
             kept = (mine[:, 0] & 3) != 3
-            assert np.array_equal(mine[kept], own)                                         # its own list, in order
+            assert last > first and np.array_equal(mine[kept], own)                        # its own chunk, in order
             assert ((mine[~kept, 0] & 15) == 3).all() and (mine[~kept, 1] == -1).all()     # none: no class, no halves
-            for e in range(int(t[4]), int(t[4] + t[5])):
+            for e in range(first, last):
                 assert (int(t[0]), pair, e) not in covered
-                covered[(int(t[0]), pair, e)] = 0
-            chunks.setdefault((int(t[0]), pair), []).append((0, int(t[4]), int(t[5]), 1, -1, -1))
-        assert set(kts.tolist()) == set((ent[qt[4]:qt[4] + qt[5], 0] >> 4).tolist()) | set((ent[qt1[4]:qt1[4] + qt1[5], 0] >> 4).tolist())
+                covered[(int(t[0]), pair, e)] = chunk
+            chunks.setdefault((int(t[0]), pair), []).append((chunk, first, last - first, nch, pb, cb))
+            both |= set((own[:, 0] >> 4).tolist())
+        assert set(kts.tolist()) == both
     assert len(covered) == n_pairs * n_own
     if G % 2 == 0:
         assert n_twin == 0 and len(ent) == n_own
     slots_used, counters_used = set(), set()
+    bases = {}
+    for (q_start, pair), lst in chunks.items():
+        bases.setdefault(q_start, set()).update((c[4], c[5]) for c in lst)
+    assert all(len(v) == 1 for v in bases.values())       # every head pair of a tile uses the tile's slots and counters
     for (q_start, pair), lst in chunks.items():
         lst.sort()
         qt = by_start[q_start]
