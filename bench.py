@@ -42,7 +42,7 @@ NOMINAL_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 8000.0   # B200 dense bf16 and HBM3e f
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one ST-SpAttn launch of the tensor-core prefill
 # kernel, from the ncu capture summarised under profiles/.  It is reported only while the kernel and planner
 # sources are the ones the capture was taken from (sha1 of their text); otherwise the roofline's traffic is null.
-NCU_TRAFFIC = {"cfg1_videollama2": {"bytes_per_launch": 31.0e6, "source_sha1": "6c7e587a4c974b32291d8bee206eaa2ce03d012b"}}
+NCU_TRAFFIC = {"cfg2_qwen25vl": {"bytes_per_launch": 113.0e6, "source_sha1": "3f5bace0115fe546dd4006c15381e73169a4d358"}}
 KERNEL_SOURCES = ("prefill_tc.cu", "tc_util.cuh", "plan.cu", "common.cuh", "prefill.cuh")
 
 
@@ -383,7 +383,7 @@ def time_pipeline(pipe, wl, d_in, steps, warmup, local, world, peaks, sync_all):
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                 "peak_kind": f"measured {which} cuBLAS bf16 ({why})" if "bf16_tflops_sustained" in peaks else f"fallback {which}",
                 **tensor_fracs(achieved, peaks), "traffic": ncu_traffic(wl.name),
-                "traffic_note": "ncu capture summarised in profiles/; null when the kernel sources changed since",
+                "traffic_note": "dram read + write of one launch under the paper mask (26 of the 28 launches of a step), from the ncu capture summarised in profiles/; null when the kernel sources changed since",
                 "algorithmic_bytes_per_launch": wl.batch.total_tokens * wl.head_dim * 2 * (2 * wl.n_q_heads + 2 * wl.n_kv_heads),
                 "flops_per_step": fl_dense + fl_st, "launches_per_step": wl.n_layers,
                 "avg_launch_ms": ms_prefill / wl.n_layers,
