@@ -107,7 +107,6 @@ __device__ __forceinline__ uint32_t order_key(float f) {
 }
 
 constexpr int kSelThreads = 512;
-constexpr int kSelItems = 8;
 
 // What the selecting CTA needs to also gather its segment's kept rows into the compact cache (Sec. 3.1: the selection
 // feeds the compressed cache directly); k_src == nullptr: selection only.  Rows are `cpr` 16-byte chunks; layer
@@ -137,7 +136,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   __shared__ uint32_t sh_prefix;
   __shared__ int32_t sh_need;
   __shared__ int32_t warp_gt[32], warp_eq[32];
-  __shared__ int32_t carry_gt, carry_eq;
+  __shared__ int32_t carry_eq;
 
   const int32_t r = blockIdx.x, g = blockIdx.y, layer = blockIdx.z;
   // launched with programmatic stream serialization behind vnorm_score_kernel, which releases its dependents only
@@ -154,7 +153,6 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   const int32_t tid = threadIdx.x;
 
   for (int32_t t = tid; t < w; t += kSelThreads) out[h + t] = nr + t;  // the recent window
-  if (tid < 32) { warp_gt[tid] = 0; warp_eq[tid] = 0; }  // entries past the CTA's warps stay zero
   if constexpr (FUSED) {
     // a half-warp reads one 256-byte row per step (16 x 16 bytes), 16 rows in flight per thread
     const uint4* vl = v + layer * layer_stride_c;
@@ -199,125 +197,180 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   // Not fused: the keys are copied into shared memory once when the launch provided room for them (s_out is unused
   // in this mode and doubles as that flag), so the radix passes do not go back to L2.
   const bool staged = FUSED || s_out != nullptr;
+  // the range of the keys, taken along the way: the radix select only has to resolve the bits in which they differ
+  uint32_t kmin = 0xFFFFFFFFu, kmax = 0u;
   if (!FUSED && staged) {
 #pragma unroll 8
-    for (int32_t j = tid; j < nr; j += kSelThreads) skeys[j] = order_key(__ldg(seg + j));  // loads of a trip in flight together
-    __syncthreads();
+    for (int32_t j = tid; j < nr; j += kSelThreads) {  // loads of a trip in flight together
+      const uint32_t key = order_key(__ldg(seg + j));
+      skeys[j] = key;
+      kmin = min(kmin, key);
+      kmax = max(kmax, key);
+    }
   }
   auto key_at = [&](int32_t j) -> uint32_t { return staged ? skeys[j] : order_key(__ldg(seg + j)); };
+  const int32_t lane = tid & 31, warp = tid >> 5;
   if (h > 0) {
 
-  // ---- radix select: the h-th largest key --------------------------------------------
-  uint32_t prefix = 0, mask = 0;
-  int32_t need = h;  // rank still to find among keys matching the prefix
-  for (int32_t shift = 24; shift >= 0; shift -= 8) {
-    if (tid < 256) hist[tid] = 0;
-    __syncthreads();
+  if (FUSED || !staged) {
 #pragma unroll 4
     for (int32_t j = tid; j < nr; j += kSelThreads) {
       const uint32_t key = key_at(j);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+      kmin = min(kmin, key);
+      kmax = max(kmax, key);
     }
-    __syncthreads();
-    if (tid < 32) {
-      // which bin holds the need-th largest key: bins taken from the top, 8 per lane, a warp scan over the lane sums
-      int32_t cnt[8], lane_sum = 0;
+  }
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        cnt[i] = hist[255 - 8 * tid - i];
-        lane_sum += cnt[i];
-      }
-      int32_t inc = lane_sum;
+  for (int d = 16; d >= 1; d >>= 1) {
+    kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, d));
+    kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, d));
+  }
+  if (lane == 0) { warp_gt[warp] = (int32_t)kmin; warp_eq[warp] = (int32_t)kmax; }
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t a = lane < kSelThreads / 32 ? (uint32_t)warp_gt[lane] : 0xFFFFFFFFu;
+    uint32_t b = lane < kSelThreads / 32 ? (uint32_t)warp_eq[lane] : 0u;
 #pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const int32_t x = __shfl_up_sync(0xffffffffu, inc, d);
-        if (tid >= d) inc += x;
+    for (int d = 16; d >= 1; d >>= 1) {
+      a = min(a, __shfl_xor_sync(0xffffffffu, a, d));
+      b = max(b, __shfl_xor_sync(0xffffffffu, b, d));
+    }
+    if (lane == 0) { sh_prefix = a; sh_need = (int32_t)b; }
+  }
+  __syncthreads();
+  kmin = sh_prefix;
+  kmax = (uint32_t)sh_need;
+  if (tid < 256) hist[tid] = 0;
+  __syncthreads();  // sh_prefix / sh_need and the two warp arrays are reused below
+
+  // ---- radix select: the h-th largest key --------------------------------------------
+  // MSB first over the bits below the keys' common prefix, 8 at a time (scores of one segment share their sign and
+  // most of their exponent: starting at bit 31 would throw nearly every key into one or two bins of the first pass,
+  // which the shared-memory atomics would serialise).  The search ends early when the bin that holds the h-th largest
+  // key is taken whole: every key of that bin and above is then selected and nothing has to be told apart inside it.
+  uint32_t thr;      // keys above thr are selected ...
+  int32_t need_eq;   // ... and this many keys equal to thr, lowest positions first
+  const uint32_t diff = kmin ^ kmax;
+  if (diff == 0u) {
+    thr = kmax;
+    need_eq = h;
+  } else {
+    const int32_t nbits = 32 - __clz(diff);  // the keys agree above bit nbits - 1
+    uint32_t mask = nbits == 32 ? 0u : ~((1u << nbits) - 1u);
+    uint32_t prefix = kmax & mask;
+    int32_t need = h;  // rank still to find among keys matching the prefix
+    // two block barriers per pass: the warp that reads the bins also clears them for the next pass, and what it
+    // publishes is read by everybody before anybody can reach the next pass's first barrier
+    for (int32_t shift = max(nbits - 8, 0);; shift = max(shift - 8, 0)) {
+#pragma unroll 4
+      for (int32_t j = tid; j < nr; j += kSelThreads) {
+        const uint32_t key = key_at(j);
+        if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
       }
-      int32_t acc = inc - lane_sum;  // keys in the bins above this lane's
-      if (acc < need && need <= inc) {
+      __syncthreads();
+      if (tid < 32) {
+        // which bin holds the need-th largest key: bins taken from the top, 8 per lane, a warp scan over the lane sums
+        int32_t cnt[8], lane_sum = 0;
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-          if (acc + cnt[i] >= need) {
-            sh_prefix = prefix | ((uint32_t)(255 - 8 * tid - i) << shift);
-            sh_need = need - acc;
-            break;
+          cnt[i] = hist[255 - 8 * tid - i];
+          hist[255 - 8 * tid - i] = 0;
+          lane_sum += cnt[i];
+        }
+        int32_t inc = lane_sum;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+          const int32_t x = __shfl_up_sync(0xffffffffu, inc, d);
+          if (tid >= d) inc += x;
+        }
+        int32_t acc = inc - lane_sum;  // keys in the bins above this lane's
+        if (acc < need && need <= inc) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            if (acc + cnt[i] >= need) {
+              // (a digit that overlaps bits already resolved repeats them: or-ing it in changes nothing)
+              sh_prefix = prefix | ((uint32_t)(255 - 8 * tid - i) << shift);
+              sh_need = need - acc;
+              carry_eq = cnt[i];  // size of the chosen bin
+              break;
+            }
+            acc += cnt[i];
           }
-          acc += cnt[i];
         }
       }
-    }
-    __syncthreads();
-    prefix = sh_prefix;
-    need = sh_need;
-    mask |= 255u << shift;
-    __syncthreads();
-  }
-  const uint32_t thr = prefix;  // key of the h-th largest score
-  const int32_t need_eq = need; // how many keys equal to thr are taken (lowest positions first)
-
-  // ---- ordered compaction --------------------------------------------------------------
-  if (tid == 0) { carry_gt = 0; carry_eq = 0; }
-  __syncthreads();
-  const int32_t lane = tid & 31, warp = tid >> 5;
-  for (int32_t c0 = 0; c0 < nr; c0 += kSelThreads * kSelItems) {
-    const int32_t j0 = c0 + tid * kSelItems;
-    uint32_t keys[kSelItems];
-    int32_t n_gt = 0, n_eq = 0;
-    if (staged && j0 + kSelItems <= nr) {
-      // a thread's keys are consecutive words: 128-bit loads, which shared memory serves without bank conflicts
-      // (word-by-word they would collide eight ways)
-#pragma unroll
-      for (int i = 0; i < kSelItems; i += 4) {
-        const uint4 k4 = *reinterpret_cast<const uint4*>(skeys + j0 + i);
-        keys[i] = k4.x; keys[i + 1] = k4.y; keys[i + 2] = k4.z; keys[i + 3] = k4.w;
+      __syncthreads();
+      prefix = sh_prefix;
+      need = sh_need;
+      const int32_t bin = carry_eq;
+      mask |= 255u << shift;
+      if (bin == need && prefix != 0u) {  // the whole bin: everything at or above its lowest possible key
+        thr = prefix - 1u;
+        need_eq = 0;
+        break;
       }
+      if (shift == 0) {
+        thr = prefix;  // key of the h-th largest score
+        need_eq = need;
+        break;
+      }
+    }
+  }
+
+  // ---- ordered compaction: one contiguous run of keys per thread, one block scan ---------------------------------
+  // runs of a multiple of 4 keys (128-bit loads) whose number of 16-byte words is odd, so that the quarter-warps'
+  // loads fall into different banks
+  const int32_t per = 4 * (((nr + kSelThreads * 4 - 1) / (kSelThreads * 4)) | 1);
+  const int32_t j0 = min(nr, tid * per), j1 = min(nr, j0 + per);
+  int32_t n_gt = 0, n_eq = 0;
+  for (int32_t j = j0; j < j1; j += 4) {
+    uint32_t k4[4];
+    if (staged && j + 4 <= j1) {
+      const uint4 q = *reinterpret_cast<const uint4*>(skeys + j);
+      k4[0] = q.x; k4[1] = q.y; k4[2] = q.z; k4[3] = q.w;
     } else {
 #pragma unroll
-      for (int i = 0; i < kSelItems; ++i) keys[i] = (j0 + i < nr) ? key_at(j0 + i) : 0u;
+      for (int i = 0; i < 4; ++i) k4[i] = j + i < j1 ? key_at(j + i) : 0u;
     }
 #pragma unroll
-    for (int i = 0; i < kSelItems; ++i) {
-      const bool valid = j0 + i < nr;
-      n_gt += (valid && keys[i] > thr);
-      n_eq += (valid && keys[i] == thr);
+    for (int i = 0; i < 4; ++i) {
+      const bool valid = j + i < j1;
+      n_gt += (valid && k4[i] > thr);
+      n_eq += (valid && k4[i] == thr);
     }
-    int32_t inc_gt = n_gt, inc_eq = n_eq;
+  }
+  int32_t inc_gt = n_gt, inc_eq = n_eq;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const int32_t a = __shfl_up_sync(0xffffffffu, inc_gt, d), b = __shfl_up_sync(0xffffffffu, inc_eq, d);
+    if (lane >= d) { inc_gt += a; inc_eq += b; }
+  }
+  if (lane == 31) { warp_gt[warp] = inc_gt; warp_eq[warp] = inc_eq; }
+  __syncthreads();
+  if (warp == 0) {
+    int32_t a = lane < kSelThreads / 32 ? warp_gt[lane] : 0, b = lane < kSelThreads / 32 ? warp_eq[lane] : 0;
+    const int32_t ta = a, tb = b;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) {
-      const int32_t a = __shfl_up_sync(0xffffffffu, inc_gt, d), b = __shfl_up_sync(0xffffffffu, inc_eq, d);
-      if (lane >= d) { inc_gt += a; inc_eq += b; }
+      const int32_t x = __shfl_up_sync(0xffffffffu, a, d), y = __shfl_up_sync(0xffffffffu, b, d);
+      if (lane >= d) { a += x; b += y; }
     }
-    if (lane == 31) { warp_gt[warp] = inc_gt; warp_eq[warp] = inc_eq; }
-    __syncthreads();
-    if (warp == 0) {
-      int32_t a = warp_gt[lane], b = warp_eq[lane];
-      const int32_t ta = a, tb = b;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) {
-        const int32_t x = __shfl_up_sync(0xffffffffu, a, d), y = __shfl_up_sync(0xffffffffu, b, d);
-        if (lane >= d) { a += x; b += y; }
-      }
-      warp_gt[lane] = a - ta;  // exclusive
-      warp_eq[lane] = b - tb;
-    }
-    __syncthreads();
-    int32_t pos_gt = carry_gt + warp_gt[warp] + inc_gt - n_gt;  // exclusive counts before this thread
-    int32_t pos_eq = carry_eq + warp_eq[warp] + inc_eq - n_eq;
-#pragma unroll
-    for (int i = 0; i < kSelItems; ++i) {
-      if (j0 + i < nr) {
-        if (keys[i] > thr) {
-          out[pos_gt + min(pos_eq, need_eq)] = j0 + i;
-          ++pos_gt;
-        } else if (keys[i] == thr) {
-          if (pos_eq < need_eq) out[pos_gt + pos_eq] = j0 + i;
-          ++pos_eq;
-        }
+    warp_gt[lane] = a - ta;  // exclusive
+    warp_eq[lane] = b - tb;
+  }
+  __syncthreads();
+  int32_t pos_gt = warp_gt[warp] + inc_gt - n_gt;  // exclusive counts before this thread's run
+  int32_t pos_eq = warp_eq[warp] + inc_eq - n_eq;
+  if (n_gt > 0 || (n_eq > 0 && pos_eq < need_eq)) {
+    for (int32_t j = j0; j < j1; ++j) {
+      const uint32_t key = key_at(j);
+      if (key > thr) {
+        out[pos_gt + min(pos_eq, need_eq)] = j;
+        ++pos_gt;
+      } else if (key == thr) {
+        if (pos_eq < need_eq) out[pos_gt + pos_eq] = j;
+        ++pos_eq;
       }
     }
-    __syncthreads();
-    if (tid == kSelThreads - 1) { carry_gt = pos_gt; carry_eq = pos_eq; }
-    __syncthreads();
   }
   }  // h > 0
 
