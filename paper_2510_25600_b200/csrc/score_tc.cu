@@ -10,7 +10,10 @@
 //               may span several query heads, a box of B rows never does (few large boxes: the copy engine's rate
 //               of small boxes bounded this kernel when the boxes were 8 rows high)
 //   warp 1      owns the TMEM columns; one lane issues the products
-//   warps 2-5   one thread per key: S^T row from TMEM, exp2 against the column's log-sum-exp, running sum
+//   warps 2-9   two groups of four warps, one thread per key in each; a group takes every other block of rows (always
+//               the same accumulator): S^T row from TMEM, exp2 against the column's log-sum-exp, running sum; the
+//               groups' sums meet at the end.  Two CTAs per SM give each scheduler four such warps: with two the
+//               kernel was bound by the latencies of the TMEM loads and of the exponentials, not by any unit's rate.
 // bf16, head_dim 128, window a multiple of 8.  Every wait is bounded; on expiry the status word is set.
 #include <algorithm>
 
@@ -28,7 +31,7 @@ constexpr int kScorePoly = PUREKV_SCORE_POLY;
 using namespace tc;
 
 constexpr int kKeys = 128, kRows = 128;
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr int kStages = 2;         // Q-row blocks in flight
 constexpr uint32_t kTmemCols = 256;  // two 128-column accumulators
 constexpr uint32_t kPanel = kRows * 128;  // bytes of one 64-column panel of a 128-row tile
@@ -48,7 +51,8 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
     int32_t box_rows) {
   extern __shared__ uint8_t smem_raw[];
   __shared__ Barriers bars;
-  __shared__ __align__(16) float lse_s[4][2][kRows];  // per epilogue warp: the log-sum-exp values of two blocks of rows
+  __shared__ __align__(16) float lse_s[8][2][kRows];  // per epilogue warp: the log-sum-exp values of two blocks of rows
+  __shared__ float comb_s[kKeys];                     // the second group's column sums, for the first to add
   __shared__ uint32_t tmem_base_s;
   __shared__ int abort_s;
   const int32_t r = blockIdx.z, g = blockIdx.y, j0 = blockIdx.x * kKeys;
@@ -97,6 +101,7 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
   tc_fence_after();
   const uint32_t tmem = tmem_base_s;
   const bool start_ok = abort_s == 0;
+  float col_sum = 0.f;  // an epilogue thread's column sum over its group's blocks
 
   if (start_ok && warp == 0) {
     // ---------------- producer ----------------
@@ -161,6 +166,7 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
   } else if (start_ok && warp >= 2) {
     // ---------------- column sums: one thread per key ----------------
     const int quad = warp & 3;  // TMEM lane quadrant this warp may access
+    const int32_t wg = (warp - 2) >> 2;  // this warp's group takes blocks wg, wg + 2, ...: always accumulator wg
     const int key = quad * 32 + lane;
     const uint32_t t_lane = tmem + ((uint32_t)(quad * 32) << 16);
     const float kLog2e = 1.4426950408889634f;
@@ -180,17 +186,19 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
       }
     };
     float lv[4];
-    fetch_lse(0, lv);
+    if (wg < n_blocks) {
+      fetch_lse(wg, lv);
 #pragma unroll
-    for (int c = 0; c < 4; ++c) my_lse[0][32 * c + lane] = lv[c];
+      for (int c = 0; c < 4; ++c) my_lse[0][32 * c + lane] = lv[c];
+    }
     __syncwarp();
-    for (int32_t t = 0; ok && t < n_blocks; ++t) {
-      const int32_t b = t & 1;
-      if (t + 1 < n_blocks) fetch_lse(t + 1, lv);  // in flight while this block is summed
+    for (int32_t t = wg, n = 0; ok && t < n_blocks; t += 2, ++n) {
+      const int32_t b = wg, lb = n & 1;
+      if (t + 2 < n_blocks) fetch_lse(t + 2, lv);  // in flight while this block is summed
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.d_full[b]), (t >> 1) & 1, abort_flag, wait_ns) ? 1 : 0) != 0;
       if (!ok) break;
       tc_fence_after();
-      const float4* l4 = reinterpret_cast<const float4*>(my_lse[b]);
+      const float4* l4 = reinterpret_cast<const float4*>(my_lse[lb]);
       // the next 32 columns are on their way from TMEM while the current ones go through the exponentials
       uint32_t rr[2][32];
       tmem_ld32(t_lane + b * kRows, rr[0]);
@@ -219,16 +227,15 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars.d_empty[b]));
-      if (t + 1 < n_blocks) {
+      if (t + 2 < n_blocks) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) my_lse[b ^ 1][32 * c + lane] = lv[c];  // last read two blocks ago by this warp
+        for (int c = 0; c < 4; ++c) my_lse[lb ^ 1][32 * c + lane] = lv[c];  // last read two of this warp's blocks ago
         __syncwarp();
       }
     }
-    if (ok) {
-      const int32_t j = j0 + key;
-      if (j < len) cg[j] = j < nr ? ((acc[0] + acc[1]) + (acc[2] + acc[3])) / (float)G : 0.f;
-    }
+    // the two groups' sums meet after the CTA's closing barrier
+    col_sum = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    if (wg == 1) comb_s[key] = col_sum;
   }
 
   tc_fence_before();
@@ -236,6 +243,10 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
+  }
+  if (start_ok && warp >= 2 && warp < 6 && abort_s == 0) {
+    const int32_t j = j0 + (warp & 3) * 32 + lane;
+    if (j < len) cg[j] = j < nr ? (col_sum + comb_s[(warp & 3) * 32 + lane]) / (float)G : 0.f;
   }
   if (tid == 0 && abort_s && start_ok) atomicExch(status, (int32_t)PUREKV_ERR_TIMEOUT);
 }
