@@ -176,13 +176,19 @@ __global__ void __launch_bounds__(kThreads, 2) score_tc_kernel(
     // Each warp keeps its own copy in shared memory, fetched one block ahead (lane i loads rows i, i+32, i+64, i+96)
     // and read back four at a time; no meeting between warps is needed.
     float (*my_lse)[kRows] = lse_s[warp - 2];
+    const uint32_t w_inv = (uint32_t)(0x100000000ull / (uint32_t)w);  // floor(2^32 / w): the quotient estimate is low by at most 1
     auto fetch_lse = [&](int32_t t, float (&lv)[4]) {
 #pragma unroll
+      const int32_t blk = t + rot < n_blocks ? t + rot : t + rot - n_blocks;  // t and rot are both below n_blocks
       for (int c = 0; c < 4; ++c) {
-        const int32_t row = ((t + rot) % n_blocks) * kRows + 32 * c + lane;
+        const int32_t row = blk * kRows + 32 * c + lane;
         lv[c] = INFINITY;
-        if (row < n_rows)
-          lv[c] = __ldg(lse + (int64_t)(g * G + row / w) * n_tokens + base + len - w + row % w) * kLog2e;
+        if (row < n_rows) {
+          // row / w by a multiplication (a division per row and block is a tenth of this warp's instructions)
+          int32_t head = (int32_t)__umulhi((uint32_t)row, w_inv);
+          head += (head + 1) * w <= row;
+          lv[c] = __ldg(lse + (int64_t)(g * G + head) * n_tokens + base + len - w + (row - head * w)) * kLog2e;
+        }
       }
     };
     float lv[4];
