@@ -258,6 +258,34 @@ def test_scores_from_prefill_lse(window, H, Hkv):
     assert gc.score_error(c.cpu().numpy(), c_two_pass.cpu().numpy().astype(np.float64)) <= gc.SCORE_RTOL
 
 
+@pytest.mark.parametrize("window", [16, 64])
+def test_scores_from_prefill_lse_many_requests(window):
+    # 45 requests, some empty, some shorter than the window, some of several key blocks: the persistent form of the
+    # one-pass kernel numbers its items through a table of the requests' running block counts (scanned 32 requests at a
+    # time) and carries its pipeline from item to item
+    P = gc.pk()
+    H, Hkv = 6, 2
+    pre = [(0, 8, 0, 24, 3, 0, 16, 5, 40)[i % 9] for i in range(45)]
+    frames = [(0, 0, 1, 0, 4, 0, 0, 9, 0)[i % 9] for i in range(45)]
+    suf = [(0, 0, 2, 0, 5, 0, 0, 7, 0)[i % 9] for i in range(45)]         # lengths 0, 8, 32, 24, 128, 0, 16, 282, 40
+    wl = make_wl("bf16", H, Hkv, 128, pre, frames, suf, 5, 6, 64)
+    x = inputs.make_qkv(wl, 0)
+    db = gc.device_batch(wl)
+    q, k, v = (gc.upload(x, n, "bf16") for n in "qkv")
+    dense = inputs.STMask(5, 6, tile=64, dense_causal=True)
+    plan = P.purekv_plan_build(db, P.st_params(dense), P.BF16, 128, H, Hkv)
+    lse = torch.empty((H, db.total_tokens), dtype=torch.float32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    P.purekv_st_sparse_prefill(q, k, v, db, plan, lse=lse, status=status)
+    c = torch.full((Hkv, db.total_tokens), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):                                               # twice: nothing is left behind between calls
+        P.purekv_lowlayer_score_lse(q, k, lse, db, window, c_out=c, status=status)
+    assert P.purekv_poll_status(status) == 0
+    c_ref = po.lowlayer_score(x["q"], x["k"], wl.batch.cu_seqlens, window)
+    assert np.isfinite(c.cpu().numpy()).all()
+    assert gc.score_error(c.cpu().numpy(), c_ref) <= gc.SCORE_RTOL
+
+
 def test_compress_cfg0():
     wl = inputs.workload(0)
     check_compress(wl, 1, wl.window, wl.keep_ratio)
