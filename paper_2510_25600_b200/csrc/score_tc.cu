@@ -649,13 +649,25 @@ extern "C" purekv_status purekv_lowlayer_score_lse(const void* q, const void* k,
   }
   const size_t smem = 1024 + (size_t)(1 + kStages) * kTile;
   const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
-  // Two forms.  Long lists of rows per item (about eight blocks of 128 stacked rows or more): one CTA per key block,
-  // handed out by the hardware as CTAs retire -- the fixed costs of a CTA are small beside its item, and a retiring
-  // CTA's successor starts while the SM's other CTA is in mid-item.  Short lists (a small window), where those fixed
-  // costs were most of the time: two persistent CTAs per SM take the items in turn and overlap an item's loads and
-  // first product with the previous item's sums.
+  // Two forms.  One CTA per key block, handed out by the hardware over the grid (longest request's key blocks) x
+  // heads x requests: a retiring CTA's successor starts while the SM's other CTA is in mid-item, which hides a CTA's
+  // fixed costs well once an item has a few blocks of rows.  Two persistent CTAs per SM that take the items in turn
+  // over the key blocks the requests really have: measured faster when an item is one or two blocks of rows (the
+  // fixed costs were most of a CTA's time) and when the requests' lengths differ (the rectangular grid then launches
+  // many CTAs that find nothing to do) unless the items are very long.
   const int64_t blocks_per_item = ((int64_t)(n_q_heads / n_kv_heads) * window + kRows - 1) / kRows;
-  if (blocks_per_item >= 8 || batch->n_req > kMaxReq) {
+  int64_t n_items = 0;  // the key blocks of every (request, KV head)
+  for (int r = 0; r < batch->n_req; ++r)
+    n_items += (int64_t)((batch->h_cu_seqlens[r + 1] - batch->h_cu_seqlens[r] + kKeys - 1) / kKeys) * n_kv_heads;
+  if (n_items == 0) return PUREKV_OK;
+  const int64_t n_rect = (int64_t)((ml + kKeys - 1) / kKeys) * n_kv_heads * batch->n_req;
+  int dev = 0, n_sm = 0;
+  PK_CUDA(cudaGetDevice(&dev));
+  PK_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+  // (with no more than two items per persistent CTA there is nothing to overlap)
+  const bool persistent = batch->n_req <= kMaxReq && n_items > 4 * (int64_t)n_sm &&
+                          (blocks_per_item <= 2 || (n_items * 100 < n_rect * 85 && blocks_per_item < 20));
+  if (!persistent) {
     static std::atomic<uint64_t> smem_allowed{0};
     const purekv_status st_smem = allow_max_dynamic_smem(score_tc_kernel, smem_allowed);
     if (st_smem != PUREKV_OK) return st_smem;
@@ -667,15 +679,8 @@ extern "C" purekv_status purekv_lowlayer_score_lse(const void* q, const void* k,
     static std::atomic<uint64_t> smem_allowed{0};
     const purekv_status st_smem = allow_max_dynamic_smem(score_tc_items_kernel, smem_allowed);
     if (st_smem != PUREKV_OK) return st_smem;
-    int64_t n_items = 0;  // the key blocks of every (request, KV head)
-    for (int r = 0; r < batch->n_req; ++r)
-      n_items += (int64_t)((batch->h_cu_seqlens[r + 1] - batch->h_cu_seqlens[r] + kKeys - 1) / kKeys) * n_kv_heads;
-    if (n_items == 0) return PUREKV_OK;
     PK_REQUIRE(n_items < (int64_t)1 << 30, PUREKV_ERR_UNSUPPORTED, "purekv_lowlayer_score_lse: %lld key blocks",
                (long long)n_items);
-    int dev = 0, n_sm = 0;
-    PK_CUDA(cudaGetDevice(&dev));
-    PK_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
     dim3 grid((unsigned)std::min<int64_t>(n_items, 2 * (int64_t)n_sm));
     score_tc_items_kernel<<<grid, kThreads, smem, (cudaStream_t)stream>>>(
         mk, mq8, lse, c_out, batch->cu_seqlens, window, n_q_heads, n_kv_heads, scale * 1.4426950408889634f, T, status,

@@ -260,14 +260,15 @@ def test_scores_from_prefill_lse(window, H, Hkv):
 
 @pytest.mark.parametrize("window", [16, 64])
 def test_scores_from_prefill_lse_many_requests(window):
-    # 45 requests, some empty, some shorter than the window, some of several key blocks: the persistent form of the
-    # one-pass kernel numbers its items through a table of the requests' running block counts (scanned 32 requests at a
-    # time) and carries its pipeline from item to item
+    # 99 requests, some empty, some shorter than the window, some of several key blocks -- 660 key blocks over the 4 KV
+    # heads, one block of rows each: enough items of few rows for the persistent form of the one-pass kernel, which
+    # numbers its items through a table of the requests' running block counts (scanned 32 requests at a time) and
+    # carries its pipeline from item to item
     P = gc.pk()
-    H, Hkv = 6, 2
-    pre = [(0, 8, 0, 24, 3, 0, 16, 5, 40)[i % 9] for i in range(45)]
-    frames = [(0, 0, 1, 0, 4, 0, 0, 9, 0)[i % 9] for i in range(45)]
-    suf = [(0, 0, 2, 0, 5, 0, 0, 7, 0)[i % 9] for i in range(45)]         # lengths 0, 8, 32, 24, 128, 0, 16, 282, 40
+    H, Hkv = 8, 4
+    pre = [(0, 8, 10, 24, 30, 0, 16, 40, 40)[i % 9] for i in range(99)]
+    frames = [(0, 0, 5, 0, 9, 0, 0, 22, 0)[i % 9] for i in range(99)]
+    suf = [(0, 0, 0, 0, 0, 0, 0, 0, 0)[i % 9] for i in range(99)]         # lengths 0, 8, 160, 24, 300, 0, 16, 700, 40
     wl = make_wl("bf16", H, Hkv, 128, pre, frames, suf, 5, 6, 64)
     x = inputs.make_qkv(wl, 0)
     db = gc.device_batch(wl)
